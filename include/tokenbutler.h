@@ -1,0 +1,181 @@
+/*
+ * tokenbutler.h -- C ABI of the B200 (sm_100a) decode hot path of TokenButler.
+ *
+ * The path, per layer, per KV head and per decode step (paper Sec. 3.1, 3.3, 3.4, Sec. 4
+ * "Token Selection Policy"):
+ *   append_kv / project_keys   keep the full, never-evicted KV cache and, beside it, the cache of
+ *                              keys projected to the low "interaction" dimension d'
+ *   score_tokens               dot product of the importance query with every projected key
+ *   select_topk                top-B of the candidates (everything but S sink and W recent tokens),
+ *                              optional neighbour fetching, reuse of a selection for P steps
+ *   sparse_decode_attention    softmax attention over sinks + selected rows + recent window only
+ *
+ * Conventions
+ *   - Every pointer named *_dev is DEVICE memory, every other pointer is HOST memory that is read
+ *     before the call returns.  The library never allocates or frees device memory: the caller
+ *     allocates the four regions sized by tb_query_sizes() (256-byte aligned) and binds them with
+ *     tb_create().  `stream` is a cudaStream_t passed as void*; all work is enqueued on it and the
+ *     call returns without synchronising (tb_get_status is the one exception).
+ *   - Errors are return codes only.  A call that returns anything but TB_OK has changed no state and
+ *     launched nothing.  Problems only the device can see (an out-of-range entry in a caller-supplied
+ *     index list, an internal wait that ran out) set a device status word, skip the offending access
+ *     and let the kernel finish; tb_get_status() reads and clears that word.
+ *   - Shapes: B sequences, Hq query heads, Hkv KV heads, g = Hq/Hkv, D = head_dim (128),
+ *     d' = imp_dim (16 or 32).  kv_dtype is the storage type of K, V, K_imp, W_K and q; importance
+ *     queries, scores, outputs and log-sum-exps are fp32.  All arithmetic accumulates in fp32.
+ *
+ * Device layouts (row-major, element = kv_dtype)
+ *   kv    [n_layers][max_batch][Hkv][max_seq_len][2][D]   K row then V row of a token, adjacent
+ *   kimp  [n_layers][max_batch][Hkv][max_seq_len][d']
+ *   W_K   [Hkv][D][d'] per layer (one D x d' matrix per layer AND per KV head)
+ *   index lists: int32 rows of tb_index_capacity() entries, ascending token positions
+ */
+#ifndef TOKENBUTLER_H_
+#define TOKENBUTLER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TB_OK = 0,
+    TB_ERR_INVALID_ARG = -1,  /* null pointer, index out of range, empty problem               */
+    TB_ERR_UNSUPPORTED = -2,  /* shape / mode outside the compiled set                         */
+    TB_ERR_CAPACITY = -3,     /* append beyond max_seq_len, budget beyond max_budget, ...      */
+    TB_ERR_UNPROJECTED = -4,  /* selection asked over keys that have not been projected yet    */
+    TB_ERR_STATE = -5,        /* attention from the stored list before any selection           */
+    TB_ERR_CUDA = -6,         /* a CUDA runtime call failed                                    */
+    TB_ERR_TIMEOUT = -7,      /* device status: an internal bounded wait ran out               */
+    TB_ERR_BAD_INDEX = -8     /* device status: caller-supplied index outside [0, L)           */
+} tb_status;
+
+typedef enum { TB_F32 = 0, TB_BF16 = 1 } tb_dtype;
+/* How the g importance queries of a GQA group become one ranking per KV head. */
+typedef enum { TB_GROUP_SUM = 0, TB_GROUP_MAX = 1, TB_PER_QHEAD = 2 } tb_group_reduce;
+/* Neighbour fetching (Sec. 3.4): DILATE = every position within +-radius of a selected one;
+ * CLUSTER = runs of consecutive selected positions get radius*len extra positions just outside the
+ * run (ceil half after it, floor half before it). */
+typedef enum { TB_NEIGHBOR_DILATE = 0, TB_NEIGHBOR_CLUSTER = 1 } tb_neighbor_mode;
+
+typedef struct {
+    int32_t n_layers, n_q_heads, n_kv_heads, head_dim, imp_dim;
+    int32_t kv_dtype;      /* tb_dtype                                                       */
+    int32_t max_batch;     /* sequences the caches hold                                      */
+    int32_t max_seq_len;   /* token capacity per sequence                                    */
+    int32_t max_budget;    /* largest `budget` any select call will use                      */
+    int32_t max_radius;    /* largest neighbour radius; lists hold (2*max_radius+1)*max_budget */
+    int32_t device;        /* CUDA device ordinal the regions live on                        */
+} tb_config;
+
+typedef struct {
+    int32_t budget;        /* dynamic tokens kept per KV head; < 0 in attention = dense       */
+    int32_t sinks;         /* S: first S tokens always attended, never candidates             */
+    int32_t recent;        /* W: last W tokens always attended, never candidates              */
+    int32_t radius;        /* neighbour radius r (0 = off)                                    */
+    int32_t nmode;         /* tb_neighbor_mode                                                */
+    int32_t interval;      /* P: selection refreshed iff step % interval == 0                 */
+    int32_t step;          /* decode step counted from the first sparse step                  */
+    int32_t reduce;        /* tb_group_reduce                                                 */
+    float score_scale;     /* positive factor applied to materialised scores only             */
+} tb_select_params;
+
+typedef struct tb_ctx tb_ctx;
+
+/* Sizes (bytes) of the four caller-allocated device regions for this configuration.
+ * Errors: TB_ERR_INVALID_ARG (null, non-positive sizes, Hq % Hkv != 0),
+ * TB_ERR_UNSUPPORTED (head_dim != 128, imp_dim not in {16,32}, group size > 8). */
+tb_status tb_query_sizes(const tb_config* cfg, size_t* kv_bytes, size_t* kimp_bytes,
+                         size_t* state_bytes, size_t* workspace_bytes);
+
+/* Bind the four regions (256-byte aligned device pointers; contents of kv/kimp may be anything,
+ * state and workspace are cleared here with a synchronous memset).  The context owns nothing on the
+ * device; tb_destroy frees only host memory.  All sequences start empty. */
+tb_status tb_create(const tb_config* cfg, void* kv_dev, void* kimp_dev, void* state_dev,
+                    void* workspace_dev, tb_ctx** out);
+tb_status tb_destroy(tb_ctx* ctx);
+
+/* Entries per index-list row: (2*max_radius+1)*max_budget rounded up to a multiple of 4. */
+int32_t tb_index_capacity(const tb_ctx* ctx);
+
+/* Copy one layer's key projection W_K [Hkv][D][d'] (kv_dtype, device) into the context's state
+ * (Sec. 3.1: learned matrix of the key-cache projection). */
+tb_status tb_set_projection(tb_ctx* ctx, int32_t layer, const void* W_dev, void* stream);
+
+/* Forget a sequence in every layer: length and projected length 0, stored selections dropped. */
+tb_status tb_reset_sequence(tb_ctx* ctx, int32_t seq);
+
+/* Host-side view of a sequence: tokens cached and tokens whose keys are projected. */
+tb_status tb_get_length(const tb_ctx* ctx, int32_t layer, int32_t seq, int32_t* len, int32_t* len_projected);
+
+/* Sec. 3.3: write new tokens' K and V rows at the end of each listed sequence, for layers
+ * [layer_begin, layer_begin+layer_count).  k_dev, v_dev: [layer_count][sum(n_new)][Hkv][D], the
+ * tokens of the listed sequences concatenated in list order.  seq_ids == NULL means 0..n_seq-1.
+ * TB_ERR_CAPACITY if any sequence would exceed max_seq_len (nothing is written). */
+tb_status tb_append_kv(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, const int32_t* seq_ids,
+                       const int32_t* n_new, int32_t n_seq, const void* k_dev, const void* v_dev, void* stream);
+
+/* Sec. 3.1 "Key-cache projection" K_imp = K W_K for token positions [pos_begin[i], pos_end[i]) of
+ * each listed sequence (fp32 accumulation over channels in ascending order, one rounding to
+ * kv_dtype).  Eager (one token) or deferred batches (Sec. 3.3) are both just ranges.  Ranges must
+ * lie inside the cached tokens and start at or before the sequence's projected length (no holes). */
+tb_status tb_project_keys(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, const int32_t* seq_ids,
+                          const int32_t* pos_begin, const int32_t* pos_end, int32_t n_seq, void* stream);
+
+/* Sec. 3.4 / App. E importance scores of ALL projected tokens, materialised:
+ * scores_dev[i][h][t] = score_scale * sum_j qr[i][h][j] * K_imp[seq_i][h][t][j], t < projected length,
+ * row stride max_seq_len, entries past the projected length untouched.  q_imp_dev [n_seq][Hq][d'] fp32;
+ * qr = sum of the g importance queries that share KV head h (TB_GROUP_SUM; the other modes return
+ * TB_ERR_UNSUPPORTED).  The fast path (tb_select_topk) never materialises scores. */
+tb_status tb_score_tokens(tb_ctx* ctx, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
+                          const float* q_imp_dev, int32_t reduce, float score_scale, float* scores_dev, void* stream);
+
+/* Sec. 4 "Token Selection Policy" + Sec. 3.4 interval / neighbour fetching, fused with scoring, for
+ * layers [layer_begin, layer_begin+layer_count) (Sec. 3.3: predictor work is batched over the
+ * consumer layers of a producer).  If params->step % params->interval != 0 nothing is launched and
+ * the stored lists stay (stale reuse).  Otherwise, per (layer, sequence, KV head): candidates are
+ * positions [min(S,L), max(min(S,L), L-W)); the `budget` highest scores are kept (all candidates if
+ * fewer), equal scores resolved toward the LOWER position, -0.0 == +0.0; the list is expanded by the
+ * neighbour rule, clipped to the candidates, and stored ascending in the context.
+ * q_imp_dev: [layer_count][n_seq][Hq][d'] fp32.  idx_out_dev / cnt_out_dev (optional, may be NULL):
+ * copies of the stored lists, [layer_count][n_seq][Hkv][tb_index_capacity()] and [..][Hkv].
+ * TB_ERR_UNPROJECTED if a candidate range is not fully projected; TB_ERR_CAPACITY if budget or radius
+ * exceed the configured maxima. */
+tb_status tb_select_topk(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, const int32_t* seq_ids,
+                         int32_t n_seq, const float* q_imp_dev, const tb_select_params* params,
+                         int32_t* idx_out_dev, int32_t* cnt_out_dev, void* stream);
+
+/* Sec. 3.3 attention of one decode token per listed sequence over
+ * sinks [0,min(S,L)) + index list + window [max(min(S,L),L-W), L) of the full cache, each gathered
+ * K/V row shared by the g query heads of its KV head; split over the rows with a fixed partition and
+ * merged in a fixed order (bit-reproducible).  q_dev [layer_count][n_seq][Hq][D] kv_dtype;
+ * out_dev [layer_count][n_seq][Hq][D] fp32; lse_dev (optional) [layer_count][n_seq][Hq] natural-log
+ * sum-exp of the scaled logits.  idx_dev/cnt_dev: caller lists laid out like tb_select_topk's
+ * outputs, or both NULL to use the lists stored by the last selection (TB_ERR_STATE if none).
+ * params->budget < 0 selects the dense rule (every cached token; sinks/recent/lists ignored).
+ * sm_scale <= 0 means 1/sqrt(D). */
+tb_status tb_sparse_decode_attention(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count,
+                                     const int32_t* seq_ids, int32_t n_seq, const void* q_dev,
+                                     const tb_select_params* params, const int32_t* idx_dev,
+                                     const int32_t* cnt_dev, float sm_scale, float* out_dev, float* lse_dev,
+                                     void* stream);
+
+/* Synchronise `stream`, return the device status word (TB_OK, TB_ERR_TIMEOUT or TB_ERR_BAD_INDEX)
+ * in *device_status and clear it. */
+tb_status tb_get_status(tb_ctx* ctx, void* stream, int32_t* device_status);
+
+/* Algorithmic bytes (projected keys scanned + K/V rows gathered, upper bound from host-known sizes)
+ * of the most recent select or attention call. */
+uint64_t tb_last_step_bytes(const tb_ctx* ctx);
+
+/* Kernels launched by this context since it was created. */
+uint64_t tb_launch_count(const tb_ctx* ctx);
+
+const char* tb_status_string(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOKENBUTLER_H_ */

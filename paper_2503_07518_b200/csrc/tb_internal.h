@@ -1,0 +1,113 @@
+// Host-side context and the launch interfaces between the C ABI (tb_api.cu) and the kernel files.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/tokenbutler.h"
+
+namespace tb {
+
+constexpr int kMaxLaunchSeq = 64;     // sequences per launch (larger batches are chunked on the host)
+constexpr int kMaxLaunchUnits = 256;  // (layer, sequence) pairs per launch
+constexpr int kMaxSplits = 32;        // split-K partitions per (sequence, KV head)
+constexpr int kMaxGroup = 8;          // query heads per KV head
+
+// Geometry every kernel needs; passed by value.
+struct Geom {
+    int n_layers, Hq, Hkv, g, D, dp;
+    int max_batch, max_seq_len;
+    int idx_cap;       // entries per index-list row
+    int dtype;         // tb_dtype
+};
+
+// Per-launch table of (layer-local, sequence) pairs: which cache slot and how many tokens.
+struct UnitTable {
+    int layer_begin, layer_count, n_seq;
+    int seq_id[kMaxLaunchSeq];
+    int len[kMaxLaunchUnits];   // [layer_local * n_seq + s]
+};
+
+struct SelectArgs {
+    const float* q_imp;   // [layer_count][n_seq][Hq][dp]
+    int32_t* idx_dst;     // rows of `idx_stride` entries, indexed like the stored lists (see below)
+    int32_t* cnt_dst;
+    int dst_is_state;     // 1: rows indexed by (layer, seq_id, head) in the context's lists; 0: by launch unit
+    int idx_stride;
+    int budget, sinks, recent;
+};
+
+struct NeighborArgs {
+    const int32_t* idx_src;  // launch-unit indexed rows of `src_stride`
+    const int32_t* cnt_src;
+    int src_stride;
+    int radius, nmode, sinks, recent;
+};
+
+struct AttnArgs {
+    const void* q;          // [layer_count][n_seq][Hq][D]
+    const int32_t* idx;     // caller lists (launch-unit indexed) or NULL = stored lists
+    const int32_t* cnt;
+    float* out;             // [layer_count][n_seq][Hq][D]
+    float* lse;             // optional
+    int dense, sinks, recent, nsplit;
+    int list_bound;         // host-known upper bound of the list length (sizes the split count)
+    float sm_scale;
+};
+
+struct DevState {
+    void* W;              // [n_layers][Hkv][D][dp] kv_dtype
+    int32_t* idx;         // [n_layers][max_batch][Hkv][idx_cap]
+    int32_t* cnt;         // [n_layers][max_batch][Hkv]
+    int32_t* status;      // device status word
+    uint32_t* attn_counter;  // [n_layers*max_batch*Hkv] split arrival counters (self-resetting)
+};
+
+struct DevWork {
+    float* part_o;        // [units_q][kMaxSplits][D]
+    float* part_ml;       // [units_q][kMaxSplits][2]
+    int32_t* sel_idx;     // [n_layers*max_batch*Hkv][max_budget rounded]  pre-expansion selection
+    int32_t* sel_cnt;
+    int sel_stride;
+};
+
+}  // namespace tb
+
+struct tb_ctx {
+    tb_config cfg;
+    tb::Geom geom;
+    void* kv;
+    void* kimp;
+    tb::DevState st;
+    tb::DevWork wk;
+    size_t state_bytes, work_bytes;
+    std::vector<int> len, len_proj;       // [n_layers * max_batch]
+    std::vector<int> has_sel;             // [n_layers * max_batch]
+    CUtensorMap kimp_map;                 // 2-D view of kimp: rows = all token slots, cols = d'
+    int tile_rows;                        // rows per TMA box of the score pass
+    int sm_count;
+    uint64_t last_bytes, launches;
+};
+
+namespace tb {
+
+// tb_cache.cu
+cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new, const int* tok_off, int total_new,
+                          const void* k, const void* v, cudaStream_t s);
+cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, cudaStream_t s);
+
+// tb_select.cu
+cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, float scale, float* scores,
+                         cudaStream_t s);
+cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
+cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s);
+cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s);
+size_t select_smem_bytes(const tb_ctx* c, int chunk_tokens);
+
+// tb_attention.cu
+cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArgs& a, cudaStream_t s);
+
+}  // namespace tb

@@ -1,0 +1,304 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Sizes span several 256-row tiles, ragged tails and thread-block clusters."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2503_07518_b200 import workloads as wl  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def H():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from oracle import tb_oracle
+    tb_oracle.build()
+    from paper_2503_07518_b200 import build
+    build.build()
+    import gpu_harness
+    return gpu_harness
+
+
+def tb():
+    from paper_2503_07518_b200 import binding
+    return binding
+
+
+def full_pipeline_check(H, case, p, step=0, dense_too=False):
+    """select (vs oracle, with the near-tie rule) then attention from the stored lists (vs oracle on
+    the GPU's own list, and end to end when the sets agree)."""
+    w = case.w
+    q, qi = H.queries(w, step)
+    lists = H.gpu_select(case, qi, p)
+    assert case.ctx.get_status() == 0
+    swaps = 0
+    for l in range(w.n_layers):
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                base, full, s = case.oracle_select(l, b, h, qi[l, b], p)
+                if p.radius == 0:
+                    swaps += H.check_selection(lists[l][b][h], full, s, "layer %d seq %d head %d" % (l, b, h))
+                else:
+                    # neighbour lists follow from the base selection; compare exactly when the base sets agree
+                    if np.array_equal(lists[l][b][h], full):
+                        continue
+                    lo, hi = H.orc.candidate_range(case.cur[b], p.sinks, p.recent)
+                    assert np.all((lists[l][b][h] >= lo) & (lists[l][b][h] < hi))
+                    swaps += 1
+    out, lse = H.gpu_attention(case, q, p)
+    assert case.ctx.get_status() == 0
+    worst = 0.0
+    for l in range(w.n_layers):
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                ref, ref_lse = case.oracle_attention(l, b, h, q[l, b], lists[l][b][h], p)
+                got = out[l, b, h * w.group:(h + 1) * w.group]
+                worst = max(worst, np.abs(got - ref).max())
+                assert np.allclose(lse[l, b, h * w.group:(h + 1) * w.group], ref_lse, atol=2e-3 if w.dtype == wl.BF16 else 1e-5, rtol=1e-5)
+    assert worst <= H.ATTN_TOL[w.dtype], worst
+    if dense_too:
+        pd = tb().select_params(-1)
+        outd, _ = H.gpu_attention(case, q, pd)
+        for l in range(w.n_layers):
+            for b in range(w.batch):
+                for h in range(w.n_kv_heads):
+                    ref, _ = case.oracle_attention(l, b, h, q[l, b], None, p, dense=True)
+                    assert np.abs(outd[l, b, h * w.group:(h + 1) * w.group] - ref).max() <= H.ATTN_TOL[w.dtype]
+    return swaps, worst
+
+
+def test_cfg1_fp32_full_size(H):
+    # configs[0]: single layer, 8 = 8 heads, fp32, 4096 tokens, budget 256 + 4 sinks + 64 recent
+    w = wl.workload(1)
+    case = H.Case(w)
+    p = tb().select_params(w.budget, w.sinks, w.recent)
+    swaps, worst = full_pipeline_check(H, case, p, dense_too=True)
+    assert swaps == 0
+
+
+def test_bf16_gqa_ragged_batch(H):
+    # Llama-shaped heads (32 query / 8 KV), two layers, ragged lengths that end mid-tile
+    w = wl.workload(2, n_layers=2, batch=3, lengths=[5000, 3333, 257], budget=300, sinks=3, recent=17, outlier_channels=4)
+    case = H.Case(w)
+    p = tb().select_params(w.budget, w.sinks, w.recent)
+    full_pipeline_check(H, case, p, dense_too=True)
+
+
+def test_cluster_path_long_sequence(H):
+    # one sequence, two KV heads: the selection is spread over a thread-block cluster of 8
+    w = wl.workload(4, n_layers=1, n_q_heads=8, n_kv_heads=2, lengths=[20011], budget=777, sinks=16, recent=256, planted=0)
+    case = H.Case(w)
+    p = tb().select_params(w.budget, w.sinks, w.recent)
+    full_pipeline_check(H, case, p)
+
+
+def test_imp_dim_16_and_fp32_gqa(H):
+    w = wl.workload(1, n_q_heads=4, n_kv_heads=2, imp_dim=16, lengths=[1500], budget=100, sinks=2, recent=5)
+    full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, w.sinks, w.recent))
+    w = wl.workload(2, n_layers=1, n_q_heads=16, n_kv_heads=2, imp_dim=16, lengths=[3000], budget=64)
+    full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, 0, 0))
+
+
+def test_scores_match_oracle_and_selection_is_exact_topk_of_them(H):
+    w = wl.workload(2, n_layers=1, batch=2, lengths=[4100, 900], budget=200, sinks=1, recent=9)
+    case = H.Case(w)
+    q, qi = H.queries(w)
+    scores = torch.full((w.batch, w.n_kv_heads, case.cap), float("nan"), device="cuda")
+    case.ctx.score_tokens(0, None, w.batch, torch.from_numpy(qi[0]).cuda(), scores, scale=0.5)
+    p = tb().select_params(w.budget, w.sinks, w.recent)
+    lists = H.gpu_select(case, qi, p)
+    sc = scores.cpu().numpy()
+    for b in range(w.batch):
+        L = case.cur[b]
+        for h in range(w.n_kv_heads):
+            _, _, s = case.oracle_select(0, b, h, qi[0, b], p)
+            assert np.allclose(sc[b, h, :L], 0.5 * s, rtol=1e-5, atol=1e-5)
+            assert np.all(np.isnan(sc[b, h, L:]))                       # tail untouched
+            # the fused kernel ranks by these very fp32 values: exact top-k, ties to the lower index
+            lo, hi = H.orc.candidate_range(L, p.sinks, p.recent)
+            cand = np.arange(lo, hi)
+            order = np.lexsort((cand, -sc[b, h, lo:hi].astype(np.float64)))
+            assert np.array_equal(lists[0][b][h], np.sort(cand[order[:w.budget]]))
+
+
+def test_exact_ties_keep_lower_positions(H):
+    w = wl.workload(2, n_layers=1, n_q_heads=4, n_kv_heads=1, lengths=[3000], budget=50)
+    case = H.Case(w)
+    q, qi = H.queries(w)
+    p = tb().select_params(w.budget, 0, 0)
+    _, _, s = case.oracle_select(0, 0, 0, qi[0, 0], p)
+    order = np.argsort(-s)
+    # duplicate the projected key of the token ranked 49th (boundary) at five later and earlier positions
+    src = order[48]
+    dup = [int(x) for x in order[200:205]]
+    for t in dup:
+        case.Kimp[0][0][0, t] = case.Kimp[0][0][0, src]
+    case.ctx.kimp[0, 0, 0, :3000] = H.to_dev(case.Kimp[0][0][0, :3000], w.dtype)
+    lists = H.gpu_select(case, qi, p)
+    _, full, s2 = case.oracle_select(0, 0, 0, qi[0, 0], p)
+    assert np.array_equal(lists[0][0][0], full)                            # bit-equal scores: no tolerance
+    tied = sorted(dup + [int(src)])
+    assert set(tied[:2]) <= set(full.tolist()) and not (set(tied[2:]) & set(full.tolist()))
+    # all scores equal (zero query): the first `budget` candidates win; -0.0 and +0.0 tie
+    zero = np.zeros_like(qi)
+    zero[0, 0, 0, 0] = -0.0
+    lists = H.gpu_select(case, zero, tb().select_params(50, 7, 3))
+    assert np.array_equal(lists[0][0][0], np.arange(7, 57))
+
+
+def test_edge_cases(H):
+    w = wl.workload(2, n_layers=1, batch=4, n_q_heads=8, n_kv_heads=2, lengths=[1, 40, 300, 513], budget=64)
+    case = H.Case(w, max_budget=1024)
+    q, qi = H.queries(w)
+    # L <= S + W for the two short sequences (no candidates -> dense); budget > candidates for the others
+    p = tb().select_params(1000, 8, 32)
+    lists = H.gpu_select(case, qi, p)
+    for h in range(2):
+        assert len(lists[0][0][h]) == 0 and len(lists[0][1][h]) == 0
+        assert np.array_equal(lists[0][2][h], np.arange(8, 300 - 32))
+        assert np.array_equal(lists[0][3][h], np.arange(8, 513 - 32))
+    out, _ = H.gpu_attention(case, q, p)
+    for b in range(4):
+        for h in range(2):
+            ref, _ = case.oracle_attention(0, b, h, q[0, b], None, p, dense=True)   # everything attended
+            assert np.abs(out[0, b, h * 4:(h + 1) * 4] - ref).max() <= 2e-3
+    # budget 0: sinks + window only
+    p0 = tb().select_params(0, 8, 32)
+    full_pipeline_check(H, case, p0)
+    # budget 1
+    full_pipeline_check(H, case, tb().select_params(1, 0, 0))
+
+
+@pytest.mark.parametrize("nmode", [0, 1])
+@pytest.mark.parametrize("radius", [1, 2])
+def test_neighbor_modes(H, nmode, radius):
+    w = wl.workload(5, n_layers=1, batch=2, n_q_heads=8, n_kv_heads=2, lengths=[2500, 1800], budget=120, recent=16,
+                    radius=radius, nmode=nmode, decode_steps=0)
+    case = H.Case(w)
+    q, qi = H.queries(w)
+    p = tb().select_params(w.budget, 0, w.recent, radius, nmode)
+    lists = H.gpu_select(case, qi, p)
+    for b in range(2):
+        for h in range(2):
+            base, full, s = case.oracle_select(0, b, h, qi[0, b], p)
+            assert np.array_equal(lists[0][b][h], full)
+    full_pipeline_check(H, case, p)
+
+
+def test_interval_trajectory_with_appends(H):
+    # configs[4] in miniature: selection refreshed every P steps, +-1 neighbours, one token appended
+    # per step, keys projected in deferred batches of W tokens
+    P, Wn, steps = 4, 8, 10
+    w = wl.workload(5, n_layers=2, batch=2, n_q_heads=8, n_kv_heads=2, lengths=[1200, 700], budget=90, recent=Wn,
+                    radius=1, interval=P, decode_steps=steps)
+    case = H.Case(w, extra_len=steps)
+    stored = None
+    for t in range(steps):
+        if t > 0:
+            case.append_step(t)
+            if (case.cur[0] - case.proj[0]) >= Wn:                      # the window wrapped: project its tokens
+                case.project_range(list(case.proj), [case.proj[b] + Wn for b in range(w.batch)])
+        p = tb().select_params(w.budget, 0, Wn, 1, 0, P, t)
+        q, qi = H.queries(w, t)
+        lists = H.gpu_select(case, qi, p)
+        if t % P == 0:
+            for l in range(2):
+                for b in range(2):
+                    for h in range(2):
+                        _, full, _ = case.oracle_select(l, b, h, qi[l, b], p)
+                        assert np.array_equal(lists[l][b][h], full)
+            stored = lists
+        else:
+            for l in range(2):
+                for b in range(2):
+                    for h in range(2):
+                        assert np.array_equal(lists[l][b][h], stored[l][b][h])     # stale list reused
+        out, _ = H.gpu_attention(case, q, p)
+        for l in range(2):
+            for b in range(2):
+                for h in range(2):
+                    ref, _ = case.oracle_attention(l, b, h, q[l, b], stored[l][b][h], p)
+                    assert np.abs(out[l, b, h * 4:(h + 1) * 4] - ref).max() <= 2e-3
+
+
+def test_full_budget_equals_dense(H):
+    w = wl.workload(1, lengths=[1111], budget=2000, sinks=4, recent=64, n_q_heads=4, n_kv_heads=4)
+    case = H.Case(w, max_budget=2000)
+    q, qi = H.queries(w)
+    p = tb().select_params(2000, 4, 64)
+    H.gpu_select(case, qi, p)
+    sparse, _ = H.gpu_attention(case, q, p)
+    dense, _ = H.gpu_attention(case, q, tb().select_params(-1))
+    assert np.abs(sparse - dense).max() <= 1e-6
+
+
+def test_caller_lists_and_bad_index_status(H):
+    w = wl.workload(2, n_layers=1, n_q_heads=8, n_kv_heads=2, lengths=[600], budget=32)
+    case = H.Case(w)
+    q, qi = H.queries(w)
+    cap = case.ctx.index_capacity
+    r = np.random.Generator(np.random.PCG64(5))
+    idx = np.zeros((1, 1, 2, cap), np.int32)
+    mine = [np.sort(r.choice(np.arange(5, 590), 20, replace=False)).astype(np.int32) for _ in range(2)]
+    for h in range(2):
+        idx[0, 0, h, :20] = mine[h]
+    cnt = np.full((1, 1, 2), 20, np.int32)
+    p = tb().select_params(32, 5, 10)
+    out, _ = H.gpu_attention(case, q, p, idx=torch.from_numpy(idx).cuda(), cnt=torch.from_numpy(cnt).cuda())
+    for h in range(2):
+        ref, _ = case.oracle_attention(0, 0, h, q[0, 0], mine[h], p)
+        assert np.abs(out[0, 0, h * 4:(h + 1) * 4] - ref).max() <= 2e-3
+    assert case.ctx.get_status() == 0
+    idx[0, 0, 1, 3] = 600                                                # one past the end: skipped and reported
+    out2, _ = H.gpu_attention(case, q, p, idx=torch.from_numpy(idx).cuda(), cnt=torch.from_numpy(cnt).cuda())
+    assert case.ctx.get_status() == tb().TB_ERR_BAD_INDEX
+    assert case.ctx.get_status() == 0                                    # reading clears it
+    ref, _ = case.oracle_attention(0, 0, 1, q[0, 0], np.delete(mine[1], 3), p)
+    assert np.abs(out2[0, 0, 4:8] - ref).max() <= 2e-3
+
+
+def test_error_codes_change_nothing(H):
+    b = tb()
+    w = wl.workload(2, n_layers=1, n_q_heads=8, n_kv_heads=2, lengths=[100], budget=16)
+    case = H.Case(w, extra_len=4, project=None)
+    q, qi = H.queries(w)
+    qi_d = torch.from_numpy(qi).cuda()
+    with pytest.raises(b.TBError) as e:
+        case.ctx.select_topk(0, 1, None, 1, qi_d, b.select_params(16))
+    assert e.value.status == b.TB_ERR_UNPROJECTED
+    out = torch.zeros(1, 1, 8, 128, device="cuda")
+    with pytest.raises(b.TBError) as e:
+        case.ctx.sparse_decode_attention(0, 1, None, 1, H.to_dev(q, w.dtype), b.select_params(16), out)
+    assert e.value.status == b.TB_ERR_STATE
+    with pytest.raises(b.TBError) as e:
+        case.ctx.select_topk(0, 1, None, 1, qi_d, b.select_params(17))
+    assert e.value.status == b.TB_ERR_CAPACITY
+    k = torch.zeros(5, 2, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(b.TBError) as e:
+        case.ctx.append_kv(0, 1, None, [5], k, k)
+    assert e.value.status == b.TB_ERR_CAPACITY
+    assert case.ctx.get_length(0, 0) == (100, 0)
+    with pytest.raises(b.TBError) as e:
+        case.ctx.project_keys(0, 1, None, [10], [20])                    # would leave positions 0..9 unprojected
+    assert e.value.status == b.TB_ERR_INVALID_ARG
+    # the deferred-projection rule: only the candidates need projecting
+    case.project_range([0], [60])
+    case.ctx.select_topk(0, 1, None, 1, qi_d, b.select_params(16, 0, 40))
+    with pytest.raises(b.TBError) as e:
+        case.ctx.select_topk(0, 1, None, 1, qi_d, b.select_params(16, 0, 39))
+    assert e.value.status == b.TB_ERR_UNPROJECTED
+
+
+def test_bit_reproducible(H):
+    w = wl.workload(2, n_layers=2, batch=2, lengths=[9000, 4000], budget=500)
+    case = H.Case(w, project="oracle-only")
+    q, qi = H.queries(w)
+    p = tb().select_params(w.budget, 0, 0)
+    a = H.gpu_select(case, qi, p)
+    oa, la = H.gpu_attention(case, q, p)
+    b = H.gpu_select(case, qi, p)
+    ob, lb = H.gpu_attention(case, q, p)
+    assert all(np.array_equal(x, y) for l in range(2) for s in range(2) for x, y in zip(a[l][s], b[l][s]))
+    assert np.array_equal(oa, ob) and np.array_equal(la, lb)

@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the TokenButler decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+One "step" = one decode step of the whole path over the workload's batch: fused importance scoring +
+top-B selection (launched per group of G=4 consumer layers, as the paper batches predictor work per
+producer), neighbour expansion where the workload has it, and sparse attention per layer, over all
+layers.  Default workload: the Llama-3-8B-shaped decode at 32K context (32 layers, budget 10%).
+The printed JSON line carries the device-timed throughput (inputs resident in HBM), the same metric
+end to end through the public API with pinned host buffers, the roofline of the dominant kernel
+measured live with CUDA events, and the CPU oracle timed on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_07518_b200 import workloads as wl  # noqa: E402
+
+GROUP_LAYERS = 4          # consumer layers served by one producer (paper: G = 4)
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (None until a capture exists for that workload).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+
+def oracle_sample(w: wl.Workload, n_layers: int, passes: int, threads: int):
+    """Times the oracle, as it stands, on all (sequence, KV head) units of `n_layers` layers of the
+    workload, host-generated inputs.  Returns (seconds per pass list, units in the sample)."""
+    from oracle import tb_oracle as orc
+    orc.build()
+    units, qis, qs, Ls = [], [], [], []
+    cap = (2 * w.radius + 1) * w.budget
+    for l in range(n_layers):
+        W = wl.gen_W(w, l)
+        for b in range(w.batch):
+            K, V = wl.gen_KV(w, l, b)
+            q, qi = wl.gen_queries(w, l, b)
+            for h in range(w.n_kv_heads):
+                Kh, Vh = np.ascontiguousarray(K[h]), np.ascontiguousarray(V[h])
+                units.append(orc.Unit(Kh, Vh, orc.project_keys(Kh, np.ascontiguousarray(W[h]), w.dtype), cap))
+                qis.append(qi[h * w.group:(h + 1) * w.group])
+                qs.append(q[h * w.group:(h + 1) * w.group])
+                Ls.append(w.lengths[b])
+    times = []
+    for _ in range(passes):
+        t0 = time.perf_counter()
+        orc.step_units(units, Ls, qis, qs, [1] * len(units), g=w.group, D=w.head_dim, dp=w.imp_dim, dtype=w.dtype,
+                       budget=w.budget, sinks=w.sinks, recent=w.recent, radius=w.radius, nmode=w.nmode, n_threads=threads)
+        times.append(time.perf_counter() - t0)
+    return times, len(units)
+
+
+def cpu_leg(w: wl.Workload, sample_layers: int, passes: int):
+    threads = len(os.sched_getaffinity(0))
+    times, n_units = oracle_sample(w, sample_layers, passes, threads)
+    total_units = w.n_layers * w.batch * w.n_kv_heads
+    step_s = [t * total_units / n_units for t in times]          # units are independent: linear scaling
+    return {"times": step_s, "threads": threads,
+            "sample": "%d of %d layers (%d of %d (sequence, KV head) units) of %s, one refresh step each pass, "
+                      "scaled linearly to the whole step" % (sample_layers, w.n_layers, n_units, total_units, w.name)}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    leg = cpu_leg(w, 1, args.steps + args.warmup)       # one layer per step keeps K steps within minutes
+    t = leg["times"][args.warmup:]
+    ms = 1e3 * float(np.mean(t))
+    val = w.batch / (ms * 1e-3)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": w.name},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": leg["threads"], "kind": "oracle", "sample": leg["sample"]},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------------
+# device leg
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.stop_flag, self.max_mhz = [], set(), False, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def sample(self):
+        if not self.nv:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+            names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                     "hw_power_brake_slowdown": 0x80}
+            for k, bit in names.items():
+                if r & bit:
+                    self.reasons.add(k)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self.stop_flag:
+            self.sample()
+            time.sleep(0.01)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def fill_caches(ctx, w, torch, tbh):
+    """Seeded synthetic K/V drawn on the device (N(0,1), outlier channels x8 where the workload has
+    them), appended and projected through the library's own entry points."""
+    dt = tbh.torch_dtype(w.dtype)
+    gen = torch.Generator(device="cuda")
+    total = sum(w.lengths)
+    for l in range(w.n_layers):
+        gen.manual_seed(wl.seed_for(w.cfg_id, l, 0, wl.TAG_K))
+        Wl = (torch.randn(w.n_kv_heads, w.head_dim, w.imp_dim, generator=gen, device="cuda") / np.sqrt(w.head_dim)).to(dt)
+        ctx.set_projection(l, Wl)
+        k = torch.randn(total, w.n_kv_heads, w.head_dim, generator=gen, device="cuda")
+        if w.outlier_channels:
+            ch = wl.outlier_channels(w, l)
+            for h in range(w.n_kv_heads):
+                k[:, h, torch.from_numpy(ch[h]).cuda()] *= 8.0
+        v = torch.randn(total, w.n_kv_heads, w.head_dim, generator=gen, device="cuda")
+        ctx.append_kv(l, 1, None, w.lengths, k.to(dt), v.to(dt))
+        ctx.project_keys(l, 1, None, [0] * w.batch, w.lengths)
+        del k, v
+    torch.cuda.synchronize()
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2503_07518_b200 import binding as tbh
+    from paper_2503_07518_b200 import build
+    build.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode)
+    ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + 8,
+                      w.budget, w.radius, device=local)
+    fill_caches(ctx, w, torch, tbh)
+    dt = tbh.torch_dtype(w.dtype)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(wl.seed_for(w.cfg_id, 0, 0, wl.TAG_Q))
+    q = torch.randn(w.n_layers, w.batch, w.n_q_heads, w.head_dim, generator=gen, device="cuda").to(dt)
+    qi = torch.randn(w.n_layers, w.batch, w.n_q_heads, w.imp_dim, generator=gen, device="cuda")
+    out = torch.empty(w.n_layers, w.batch, w.n_q_heads, w.head_dim, device="cuda")
+    q_host, qi_host = q.cpu().pin_memory(), qi.cpu().pin_memory()
+    out_host = torch.empty_like(out, device="cpu").pin_memory()
+
+    groups = [(l, min(GROUP_LAYERS, w.n_layers - l)) for l in range(0, w.n_layers, GROUP_LAYERS)]
+    sel_bytes, att_bytes = [], []
+
+    def step_launches(record=False):
+        # model-faithful schedule: at each producer the selections of its consumer layers, then
+        # attention layer by layer
+        for (l0, n) in groups:
+            ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p)
+            if record:
+                sel_bytes.append(ctx.last_step_bytes())
+            for l in range(l0, l0 + n):
+                ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l])
+                if record:
+                    att_bytes.append(ctx.last_step_bytes())
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        n0 = ctx.launch_count()
+        step_launches(record=True)
+        launches_per_step = ctx.launch_count() - n0
+        torch.cuda.synchronize()
+        assert ctx.get_status(stream) == 0, "device status set during warm-up"
+        if args.profile:
+            # plain launches only (no graphs, no extra passes): the command line profilers are given
+            for _ in range(args.warmup + args.steps):
+                step_launches()
+            torch.cuda.synchronize()
+            print(json.dumps({"profile_run": w.name, "layers": w.n_layers, "launches_per_step": int(launches_per_step)}))
+            return
+
+        def capture(fn):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+            return g
+
+        g_step = capture(step_launches)
+        g_sel = capture(lambda: [ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p) for (l0, n) in groups])
+        g_att = capture(lambda: [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)])
+
+        def timed(fn, steps, warmup, sampler=None):
+            for _ in range(warmup):
+                fn()
+            stream.synchronize()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if sampler:
+                sampler.start()
+            e0.record(stream)
+            for _ in range(steps):
+                fn()
+            e1.record(stream)
+            if sampler:
+                while not e1.query():
+                    time.sleep(0.002)
+            torch.cuda.synchronize()
+            if sampler:
+                sampler.sample()
+                sampler.stop_flag = True
+            if world > 1:
+                dist.barrier()
+            ms = e0.elapsed_time(e1)
+            if world > 1:
+                t = torch.tensor([ms], device="cuda")
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ms = float(t.item())
+            return ms / steps
+
+        sampler = ClockSampler(local)
+        ms_step = timed(g_step.replay, args.steps, args.warmup, sampler)
+
+        def e2e_step():
+            q.copy_(q_host, non_blocking=True)
+            qi.copy_(qi_host, non_blocking=True)
+            g_step.replay()
+            out_host.copy_(out, non_blocking=True)
+
+        ms_e2e = timed(e2e_step, args.steps, args.warmup)
+        ms_sel = timed(g_sel.replay, max(20, args.steps // 4), 3) / len(groups)
+        ms_att = timed(g_att.replay, max(20, args.steps // 4), 3) / w.n_layers
+        assert ctx.get_status(stream) == 0, "device status set during the timed region"
+
+    peak, peak_kind = measured_peaks()
+    tokens = w.batch * world
+    sel_b, att_b = float(np.mean(sel_bytes)), float(np.mean(att_bytes))
+    step_bytes = float(np.sum(sel_bytes) + np.sum(att_bytes))
+    dom = ("select_kernel", sel_b, ms_sel) if ms_sel * len(groups) >= ms_att * w.n_layers else ("attn_kernel", att_b, ms_att)
+    achieved = dom[1] / (dom[2] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "q_heads": w.n_q_heads,
+                   "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "imp_dim": w.imp_dim,
+                   "kv_storage": "bf16" if w.dtype == wl.BF16 else "f32", "context": w.lengths if len(set(w.lengths)) > 1 else w.lengths[0],
+                   "budget": w.budget, "sinks": w.sinks, "recent": w.recent, "radius": w.radius, "interval": w.interval,
+                   "schedule": "score+select per %d layers, attention per layer, CUDA-graph replay" % GROUP_LAYERS,
+                   "l2": "inputs larger than L2: %.0f MB touched per step" % (step_bytes / 1e6)},
+        "step_hbm_gbs": step_bytes / (ms_step * 1e-3) / 1e9, "step_bytes": step_bytes,
+        "step_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "gpu_launches": int(launches_per_step * args.steps),
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
+                "h2d_bytes_per_step": q_host.numel() * q_host.element_size() + qi_host.numel() * 4,
+                "d2h_bytes_per_step": out_host.numel() * 4},
+        "roofline": {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom[0])),
+                     "bytes_per_launch": dom[1], "us_per_launch": dom[2] * 1e3},
+        "kernels": {"select_kernel": {"us_per_launch": ms_sel * 1e3, "bytes_per_launch": sel_b,
+                                      "gbs": sel_b / (ms_sel * 1e-3) / 1e9, "launches_per_step": len(groups)},
+                    "attn_kernel": {"us_per_launch": ms_att * 1e3, "bytes_per_launch": att_b,
+                                    "gbs": att_b / (ms_att * 1e-3) / 1e9, "launches_per_step": w.n_layers}},
+        "clocks": sampler.summary(),
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu:
+            leg = cpu_leg(w, args.cpu_layers, 3)
+            best = min(leg["times"])
+            line["cpu_baseline"] = {"value": w.batch / best, "unit": UNIT, "cores": leg["threads"], "kind": "oracle",
+                                    "sample": leg["sample"], "ms_per_step": best * 1e3}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (default: the 32K Llama-3-8B-shaped decode)")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-layers", type=int, default=2, help="layers in the CPU oracle's sample")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--profile", action="store_true", help="only warm-up + steps of plain launches (for ncu)")
+    args = ap.parse_args()
+    w = wl.workload(args.config)
+    if args.layers:
+        w = w.scaled(n_layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -33,6 +33,75 @@ struct RowMap {
     }
 };
 
+// Publishes one split's (m, l, o) per query head and lets the last block to arrive for the
+// (sequence, KV head) merge all splits in split order:  M = max m_j;  l = sum l_j 2^(m_j-M);
+// out = sum o_j 2^(m_j-M) / l;  lse = (M + log2 l) ln 2.  Called by all 128 threads; thread = channel.
+struct SplitSink {
+    float* part_o;
+    float* part_ml;
+    uint32_t* counters;
+    float* out;
+    float* lse;
+    size_t hq0;        // first query head of this (layer, sequence, KV head) in the launch
+    int lu, split, nsplit;
+
+    __device__ __forceinline__ void publish(int u, float M, float lsum, float o) const {
+        const size_t pq = (hq0 + u) * kMaxSplits + split;
+        part_o[pq * 128 + threadIdx.x] = o;
+        if (threadIdx.x == 0) part_ml[pq * 2] = M, part_ml[pq * 2 + 1] = lsum;
+    }
+    __device__ __forceinline__ void merge_if_last(int g, int* sh_last) const {
+        const int tid = threadIdx.x;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            unsigned prev = atomicAdd(&counters[lu], 1u);
+            *sh_last = prev == (unsigned)nsplit - 1u;
+            if (*sh_last) counters[lu] = 0;             // ready for the next launch
+        }
+        __syncthreads();
+        if (!*sh_last) return;
+        __threadfence();
+        // all (head, split) statistics in one round trip, then weights, then 16-byte wide sums
+        __shared__ float mm[kMaxGroup][kMaxSplits], lw[kMaxGroup][kMaxSplits], w[kMaxGroup][kMaxSplits];
+        __shared__ float Lsum[kMaxGroup], Mmax[kMaxGroup];
+        for (int i = tid; i < g * nsplit; i += kAttnThreads) {
+            const int u = i / nsplit, j = i % nsplit;
+            const size_t pq = (hq0 + u) * kMaxSplits + j;
+            mm[u][j] = __ldcg(&part_ml[pq * 2]);
+            lw[u][j] = __ldcg(&part_ml[pq * 2 + 1]);
+        }
+        __syncthreads();
+        if (tid < g) {
+            float M = -INFINITY;
+            for (int j = 0; j < nsplit; ++j) M = fmaxf(M, mm[tid][j]);
+            const float Ms = M == -INFINITY ? 0.f : M;
+            float lsum = 0.f;
+            for (int j = 0; j < nsplit; ++j) {
+                const float e = exp2f(mm[tid][j] - Ms);
+                w[tid][j] = e;
+                lsum += lw[tid][j] * e;
+            }
+            Lsum[tid] = lsum, Mmax[tid] = M;
+            if (lse) lse[hq0 + tid] = (M + log2f(lsum)) * kLn2;
+        }
+        __syncthreads();
+        for (int item = tid; item < g * 32; item += kAttnThreads) {
+            const int u = item >> 5, c4 = item & 31;
+            const float4* src = reinterpret_cast<const float4*>(part_o + (hq0 + u) * kMaxSplits * 128) + c4;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
+            for (int j = 0; j < nsplit; ++j) {
+                const float4 v = __ldcg(src + j * 32);
+                const float e = w[u][j];
+                acc.x = fmaf(v.x, e, acc.x), acc.y = fmaf(v.y, e, acc.y), acc.z = fmaf(v.z, e, acc.z), acc.w = fmaf(v.w, e, acc.w);
+            }
+            const float inv = 1.f / Lsum[u];
+            reinterpret_cast<float4*>(out + (hq0 + u) * 128)[c4] = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        }
+    }
+};
+
 template <typename T>
 struct RowVec;   // the 4 channels of a 128-channel row that one lane owns
 template <>
@@ -168,6 +237,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
         *reinterpret_cast<float4*>(&sh_o[warp][u][lane * 4]) = make_float4(acc[u][0], acc[u][1], acc[u][2], acc[u][3]);
     }
     __syncthreads();
+    SplitSink sink{part_o, part_ml, counters, a.out, a.lse, (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g, lu, split, a.nsplit};
     for (int u = 0; u < g; ++u) {
         float M = -INFINITY;
 #pragma unroll
@@ -180,37 +250,238 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
             lsum += sh_l[w][u] * e;
             o += sh_o[w][u][tid] * e;
         }
-        const size_t pq = ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * g + u) * kMaxSplits + split;
-        part_o[pq * D + tid] = o;
-        if (tid == 0) part_ml[pq * 2] = M, part_ml[pq * 2 + 1] = lsum;
+        sink.publish(u, M, lsum, o);
     }
+    sink.merge_if_last(g, &sh_last);
+}
 
-    // ---- last block of this (sequence, KV head) merges the splits ----------------------------------
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        unsigned prev = atomicAdd(&counters[lu], 1u);
-        sh_last = prev == (unsigned)a.nsplit - 1u;
-        if (sh_last) counters[lu] = 0;                  // ready for the next launch
+// ---------------------------------------------------------------------------------------------------
+// bf16 path: tensor-core tiles of (query heads padded to 16) x (16 gathered tokens).
+//
+// Each warp owns a ring of shared-memory stages; a stage holds 16 gathered K|V row pairs (512 B each,
+// fetched by one bulk copy per row through the TMA engine, completion counted on the stage's
+// mbarrier) at a 528-byte pitch so that ldmatrix reads are bank-conflict free.  S = Q K^T and
+// O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate); P is split into a bf16 high and low
+// part so that the probabilities keep ~16 bits.  The GQA group's heads are the M rows of the tiles,
+// which is where batch x group makes the contraction a real dense tile.
+
+constexpr int kMmaStages = 3;
+constexpr int kTileTok = 16;
+constexpr int kRowPitch = 528;                        // 512 B of K|V + 16 B pad
+constexpr int kStageBytes = kTileTok * kRowPitch;     // 8448
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTable ut, AttnArgs a, const __nv_bfloat16* __restrict__ kv,
+                                                                const int32_t* __restrict__ state_idx,
+                                                                const int32_t* __restrict__ state_cnt, float* __restrict__ part_o,
+                                                                float* __restrict__ part_ml, uint32_t* __restrict__ counters,
+                                                                int32_t* __restrict__ status) {
+    constexpr int D = 128;
+    extern __shared__ __align__(128) unsigned char smem_dyn[];
+    __shared__ uint64_t full[kAttnWarps][kMmaStages];
+    __shared__ float sh_m[kAttnWarps][kMaxGroup], sh_l[kAttnWarps][kMaxGroup];
+    __shared__ int sh_last;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+    const int split = blockIdx.x, h = blockIdx.y;
+    const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq;
+    const int L = ut.len[ll * ut.n_seq + s];
+    const int g = gm.g;
+    const size_t cu = ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h;
+    const int lu = (ll * ut.n_seq + s) * gm.Hkv + h;
+
+    RowMap rm;
+    rm.L = L, rm.dense = a.dense;
+    rm.n_sink = a.dense ? 0 : min(a.sinks, L);
+    rm.w_begin = a.dense ? 0 : max(rm.n_sink, L - a.recent);
+    int n_list = 0;
+    if (!a.dense) {
+        n_list = a.idx ? a.cnt[lu] : state_cnt[cu];
+        n_list = max(0, min(n_list, gm.idx_cap));
     }
-    __syncthreads();
-    if (!sh_last) return;
-    __threadfence();
-    for (int u = 0; u < g; ++u) {
-        const size_t hq = (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g + u;
-        const size_t pq = hq * kMaxSplits;
-        float M = -INFINITY;
-        for (int j = 0; j < a.nsplit; ++j) M = fmaxf(M, __ldcg(&part_ml[(pq + j) * 2]));
-        const float Ms = M == -INFINITY ? 0.f : M;
-        float lsum = 0.f, o = 0.f;
-        for (int j = 0; j < a.nsplit; ++j) {
-            const float e = exp2f(__ldcg(&part_ml[(pq + j) * 2]) - Ms);
-            lsum += __ldcg(&part_ml[(pq + j) * 2 + 1]) * e;
-            o += __ldcg(&part_o[(pq + j) * D + tid]) * e;
+    rm.n_list = n_list;
+    rm.list = a.idx ? a.idx + (size_t)lu * gm.idx_cap : state_idx + cu * gm.idx_cap;
+    const int n_rows = a.dense ? L : rm.n_sink + n_list + (L - rm.w_begin);
+
+    // rows of this split, dealt to the warps in whole tiles of 16
+    const int r_begin = (int)((long long)n_rows * split / a.nsplit);
+    const int r_end = (int)((long long)n_rows * (split + 1) / a.nsplit);
+    const int tiles_all = (r_end - r_begin + kTileTok - 1) / kTileTok;
+    const int tiles_per_warp = (tiles_all + kAttnWarps - 1) / kAttnWarps;
+    const int wb = min(r_end, r_begin + warp * tiles_per_warp * kTileTok);
+    const int we = min(r_end, wb + tiles_per_warp * kTileTok);
+    const int n_tiles = (we - wb + kTileTok - 1) / kTileTok;
+
+    unsigned char* my_stage = smem_dyn + (size_t)warp * kMmaStages * kStageBytes;
+    const unsigned char* kv_unit = reinterpret_cast<const unsigned char*>(kv) + cu * gm.max_seq_len * 2 * D * 2;
+
+    if (lane == 0) {
+        for (int i = 0; i < kMmaStages; ++i) mbar_init(&full[warp][i], 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+
+    bool any_bad = false;
+    // One bulk copy per row; rows past the end of the warp's range repeat its last row (their
+    // probabilities are masked to zero), so a stage always holds finite numbers.
+    auto issue = [&](int tile) {
+        const int st = tile % kMmaStages;
+        const int r0 = wb + tile * kTileTok;
+        if (lane == 0) mbar_arrive_expect_tx(&full[warp][st], kTileTok * 512);
+        __syncwarp();
+        if (lane < kTileTok) {
+            bool bad;
+            const int t = rm.token(min(r0 + lane, we - 1), bad);
+            bulk_copy_g2s(my_stage + st * kStageBytes + lane * kRowPitch, kv_unit + (size_t)t * 512, 512, &full[warp][st]);
         }
-        a.out[hq * D + tid] = o / lsum;
-        if (a.lse && tid == 0) a.lse[hq] = (M + log2f(lsum)) * kLn2;
+    };
+    for (int t = 0; t < kMmaStages && t < n_tiles; ++t) issue(t);
+
+    // Q as the A operand: rows = query heads (gid; rows 8..15 are padding), k = channels
+    uint32_t qa[8][2];
+    {
+        const __nv_bfloat16* qbase = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * g) * D;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qa[ks][0] = qa[ks][1] = 0u;
+            if (gid < g) {
+                qa[ks][0] = __ldg(reinterpret_cast<const uint32_t*>(qbase + gid * D + ks * 16 + tig * 2));
+                qa[ks][1] = __ldg(reinterpret_cast<const uint32_t*>(qbase + gid * D + ks * 16 + 8 + tig * 2));
+            }
+        }
     }
+    const float qscale = a.sm_scale * kLog2e;
+
+    float o[16][4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;             // of head gid, over this thread's token columns
+
+    const uint32_t stage_u32 = smem_u32(my_stage);
+    // per-lane ldmatrix row addresses inside a stage
+    const int mi = lane >> 3, r8 = lane & 7;
+    const uint32_t k_lane_off = ((mi >> 1) * 8 + r8) * kRowPitch + (mi & 1) * 16;          // + ks * 32
+    const uint32_t v_lane_off = ((mi & 1) * 8 + r8) * kRowPitch + 256 + (mi >> 1) * 16;    // + np * 32
+
+    bool timed_out = false;
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        const int st = tile % kMmaStages;
+        const int r0 = wb + tile * kTileTok;
+        // validity of the tile's 16 rows (past-the-end and out-of-range list entries are masked)
+        bool ok = false;
+        if (lane < kTileTok && r0 + lane < we) {
+            bool bad;
+            rm.token(r0 + lane, bad);
+            ok = !bad;
+            any_bad |= bad;
+        }
+        const unsigned vmask = __ballot_sync(0xffffffffu, ok);
+        if (!mbar_wait(&full[warp][st], (tile / kMmaStages) & 1)) timed_out = true;
+        const uint32_t sb = stage_u32 + st * kStageBytes;
+
+        float sc[2][4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(sb + k_lane_off + ks * 32, b0, b1, b2, b3);
+            mma_bf16(sc[0], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+            mma_bf16(sc[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+        }
+        // this thread: head gid, tokens j*8 + tig*2 + {0,1}
+        float x[4];
+        float tmax = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int col = j * 8 + tig * 2 + e;
+                x[j * 2 + e] = (vmask >> col) & 1u ? sc[j][e] * qscale : -INFINITY;
+                tmax = fmaxf(tmax, x[j * 2 + e]);
+            }
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+        const float m_new = fmaxf(m_run, tmax);
+        const float ms = m_new == -INFINITY ? 0.f : m_new;
+        const float corr = exp2f(m_run - ms);
+        m_run = m_new;
+        float p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = exp2f(x[i] - ms);
+        l_run = l_run * corr + (p[0] + p[1] + p[2] + p[3]);
+        const bool rescale = __any_sync(0xffffffffu, corr != 1.f);
+        if (rescale) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i][0] *= corr, o[i][1] *= corr;
+        }
+        // P = P_hi + P_lo in bf16
+        float ph[4], pl[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            ph[i] = __bfloat162float(__float2bfloat16_rn(p[i]));
+            pl[i] = p[i] - ph[i];
+        }
+        const uint32_t pa_hi0 = pack_bf16(ph[0], ph[1]), pa_hi2 = pack_bf16(ph[2], ph[3]);
+        const uint32_t pa_lo0 = pack_bf16(pl[0], pl[1]), pa_lo2 = pack_bf16(pl[2], pl[3]);
+#pragma unroll
+        for (int np = 0; np < 8; ++np) {
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(sb + v_lane_off + np * 32, b0, b1, b2, b3);
+            mma_bf16(o[2 * np], pa_hi0, 0u, pa_hi2, 0u, b0, b1);
+            mma_bf16(o[2 * np], pa_lo0, 0u, pa_lo2, 0u, b0, b1);
+            mma_bf16(o[2 * np + 1], pa_hi0, 0u, pa_hi2, 0u, b2, b3);
+            mma_bf16(o[2 * np + 1], pa_lo0, 0u, pa_lo2, 0u, b2, b3);
+        }
+        __syncwarp();
+        if (tile + kMmaStages < n_tiles) {
+            fence_proxy_async();
+            issue(tile + kMmaStages);
+        }
+    }
+    if ((any_bad || timed_out) && lane < kTileTok) atomicExch(status, timed_out ? kStatusTimeout : kStatusBadIndex);
+
+    // ---- warp result -> shared (reusing the warp's own stages), block combine, publish ------------------
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    __syncwarp();
+    float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][128 channels]
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) *reinterpret_cast<float2*>(&wo[gid * D + nt * 8 + tig * 2]) = make_float2(o[nt][0], o[nt][1]);
+    if (tig == 0) sh_m[warp][gid] = m_run, sh_l[warp][gid] = l_run;
+    __syncthreads();
+    SplitSink sink{part_o, part_ml, counters, a.out, a.lse, (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g, lu, split, a.nsplit};
+    for (int u = 0; u < g; ++u) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, sh_m[w][u]);
+        const float Ms = M == -INFINITY ? 0.f : M;
+        float lsum = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kAttnWarps; ++w) {
+            const float e = exp2f(sh_m[w][u] - Ms);
+            lsum += sh_l[w][u] * e;
+            acc += reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * D + tid] * e;
+        }
+        sink.publish(u, M, lsum, acc);
+    }
+    sink.merge_if_last(g, &sh_last);
 }
 
 static int pick_nsplit(const tb_ctx* c, int units, int max_rows) {
@@ -245,7 +516,19 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         else if (gm.g <= 4) TB_ATTN(T, 4);            \
         else TB_ATTN(T, 8);                           \
     } while (0)
-    if (gm.dtype == TB_BF16) TB_ATTN_G(__nv_bfloat16); else TB_ATTN_G(float);
+    if (gm.dtype == TB_BF16) {
+        static bool configured = false;
+        const size_t smem = (size_t)kAttnWarps * kMmaStages * kStageBytes;
+        if (!configured) {
+            cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        attn_mma_kernel<<<grid, kAttnThreads, smem, s>>>(gm, ut, a, (const __nv_bfloat16*)c->kv, c->st.idx, c->st.cnt,
+                                                         c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
+    } else {
+        TB_ATTN_G(float);
+    }
 #undef TB_ATTN_G
 #undef TB_ATTN
     return cudaGetLastError();

@@ -24,6 +24,24 @@ constexpr int kStages = 3;
 constexpr int kBins = 2048;         // 11-bit digits (the last pass uses 10 bits)
 constexpr int kMaxCluster = 8;
 
+// Optional per-phase timestamps of block (0,0) and of the last block, for tuning builds only
+// (-DTB_PHASE_TIMING); the product build compiles these away.
+#ifdef TB_PHASE_TIMING
+__device__ unsigned long long g_phase_ns[2][16];
+__device__ __forceinline__ void phase_stamp(int i) {
+    if (threadIdx.x == 0 && blockIdx.y == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_phase_ns[blockIdx.x == 0 ? 0 : 1][i] = t;
+    }
+}
+extern "C" int tb_debug_phase_ns(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_phase_ns, sizeof(g_phase_ns));
+}
+#else
+__device__ __forceinline__ void phase_stamp(int) {}
+#endif
+
 // ---- scoring arithmetic shared by the standalone and the fused kernel --------------------------
 
 // Importance query of KV head h: sum over the g query heads of the group, in head order.
@@ -198,6 +216,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     }
 
     // ---- set-up -------------------------------------------------------------------------------
+    phase_stamp(0);
     for (int i = tid; i < 4 * kBins; i += kSelThreads) hist[i] = 0;               // local + 3 merged
     if (tid == 0) {
         prefetch_tmap(&tmap);
@@ -207,6 +226,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     __syncthreads();
     if (C > 1) cluster.sync();                         // every block's merged histograms are zero before any push
 
+    phase_stamp(1);
     const int n_tiles = (ncand + kTileRows - 1) / kTileRows;
     const int tile0 = rank * tiles_per_cta;
     const int my_tiles = max(0, min(tiles_per_cta, n_tiles - tile0));
@@ -251,6 +271,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         }
     }
     if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    phase_stamp(2);
 
     // ---- radix select: three digits (11, 11, 10 bits), histograms merged over the cluster --------
     uint32_t prefix = 0;          // digits fixed so far (value of key >> low_bits)
@@ -293,6 +314,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
         }
         __syncthreads();
+        phase_stamp(3 + pass);
     }
 
     // ---- ordered compaction ------------------------------------------------------------------------
@@ -323,6 +345,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         cluster.sync();
         for (int r = 0; r < rank; ++r) gt_before += sm->tot[r][0], eq_before += sm->tot[r][1];
     }
+    phase_stamp(6);
     int out_pos = gt_before + min(eq_before, krem);
     const unsigned lt_mask = (1u << lane) - 1u;
     for (int i0 = seg_begin; i0 < seg_end; i0 += 32) {
@@ -339,6 +362,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         eq_before += __popc(eq_ballot);
     }
     if (rank == 0 && tid == 0) *cnt_dst = k;
+    phase_stamp(7);
 }
 
 size_t select_smem_bytes(const tb_ctx* c, int tiles_per_cta) {

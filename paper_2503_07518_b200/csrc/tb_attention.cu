@@ -265,6 +265,27 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
 // part so that the probabilities keep ~16 bits.  The GQA group's heads are the M rows of the tiles,
 // which is where batch x group makes the contraction a real dense tile.
 
+#ifdef TB_PHASE_TIMING
+__device__ unsigned long long g_attn_phase_ns[2][16];
+__device__ __forceinline__ void attn_stamp(int i) {
+    if (threadIdx.x == 0 && (i == 0 || i == 6)) {    // slots 8/9 of row 0: earliest start / latest end over all blocks
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        if (i == 0) atomicMin(&g_attn_phase_ns[0][8], t); else atomicMax(&g_attn_phase_ns[0][9], t);
+    }
+    if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_attn_phase_ns[blockIdx.x == 0 ? 0 : 1][i] = t;
+    }
+}
+extern "C" int tb_debug_attn_phase_ns(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_attn_phase_ns, sizeof(g_attn_phase_ns));
+}
+#else
+__device__ __forceinline__ void attn_stamp(int) {}
+#endif
+
 constexpr int kMmaStages = 3;
 constexpr int kTileTok = 16;
 constexpr int kRowPitch = 528;                        // 512 B of K|V + 16 B pad
@@ -297,6 +318,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
     __shared__ float sh_m[kAttnWarps][kMaxGroup], sh_l[kAttnWarps][kMaxGroup];
     __shared__ int sh_last;
 
+    attn_stamp(0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gid = lane >> 2, tig = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y;
@@ -351,7 +373,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
             bulk_copy_g2s(my_stage + st * kStageBytes + lane * kRowPitch, kv_unit + (size_t)t * 512, 512, &full[warp][st]);
         }
     };
+    attn_stamp(1);
     for (int t = 0; t < kMmaStages && t < n_tiles; ++t) issue(t);
+    attn_stamp(2);
 
     // Q as the A operand: rows = query heads (gid; rows 8..15 are padding), k = channels
     uint32_t qa[8][2];
@@ -393,6 +417,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
         }
         const unsigned vmask = __ballot_sync(0xffffffffu, ok);
         if (!mbar_wait(&full[warp][st], (tile / kMmaStages) & 1)) timed_out = true;
+        if (tile == 0) attn_stamp(3);
         const uint32_t sb = stage_u32 + st * kStageBytes;
 
         float sc[2][4];
@@ -458,6 +483,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
     if ((any_bad || timed_out) && lane < kTileTok) atomicExch(status, timed_out ? kStatusTimeout : kStatusBadIndex);
 
     // ---- warp result -> shared (reusing the warp's own stages), block combine, publish ------------------
+    attn_stamp(4);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
     __syncwarp();
@@ -481,7 +507,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
         }
         sink.publish(u, M, lsum, acc);
     }
+    attn_stamp(5);
     sink.merge_if_last(g, &sh_last);
+    attn_stamp(6);
 }
 
 static int pick_nsplit(const tb_ctx* c, int units, int max_rows) {

@@ -162,6 +162,34 @@ tb_status tb_sparse_decode_attention(tb_ctx* ctx, int32_t layer_begin, int32_t l
                                      const int32_t* cnt_dev, float sm_scale, float* out_dev, float* lse_dev,
                                      void* stream);
 
+/* Allocation-free variant of the attention entry point.  (The paper has no counterpart: this exists
+ * for callers that cannot allocate device memory when they need attention -- a plugin inside a
+ * serving process whose memory pool was fixed at start-up, a latency-critical thread on which
+ * cudaMalloc, which may synchronise the device, is forbidden, or a host that has given all free HBM
+ * to its KV cache.)  It needs no tb_ctx and no workspace: the split partials and arrival counters
+ * live in a fixed array inside the library image, about 1.1 MB that every GPU loading the library
+ * holds until the process exits.  The call itself allocates and frees nothing.
+ *
+ *   kv_dev     one layer's cache [slot][Hkv][max_seq_len][2][D] in kv_dtype (same row layout as above)
+ *   seq_slots  (host, NULL = 0..n_seq-1) cache slot of each listed sequence; seq_lens (host) tokens cached
+ *   q_dev      [n_seq][Hq][D] kv_dtype;  out_dev [n_seq][Hq][D] fp32;  lse_dev optional [n_seq][Hq]
+ *   idx_dev / cnt_dev  caller lists [n_seq][Hkv][idx_stride] / [n_seq][Hkv] (ascending positions inside the
+ *              candidate range), or both NULL for dense attention; entries outside [0, len) are skipped
+ *   sinks, recent, sm_scale  as in tb_sparse_decode_attention
+ *
+ * Limits: n_seq * Hq <= TB_STATIC_MAX_QHEADS and n_seq <= 64, otherwise TB_ERR_CAPACITY and nothing is
+ * launched.  The first call on each device looks up the array's device address (that device must be
+ * current) and configures the kernel; make that first call outside any stream capture.  All calls in
+ * the process share the one array: the counters are cleared on `stream` at the start of every call, and
+ * two calls whose kernels overlap on the GPU (different streams, no ordering) race on the partials. */
+#define TB_STATIC_MAX_QHEADS 64
+tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32_t kv_dtype, int32_t n_q_heads, int32_t n_kv_heads,
+                                            int32_t head_dim, int32_t max_seq_len, const int32_t* seq_slots,
+                                            const int32_t* seq_lens, int32_t n_seq, const void* q_dev,
+                                            const int32_t* idx_dev, const int32_t* cnt_dev, int32_t idx_stride,
+                                            int32_t sinks, int32_t recent, float sm_scale, float* out_dev,
+                                            float* lse_dev, void* stream);
+
 /* Synchronise `stream`, return the device status word (TB_OK, TB_ERR_TIMEOUT or TB_ERR_BAD_INDEX)
  * in *device_status and clear it. */
 tb_status tb_get_status(tb_ctx* ctx, void* stream, int32_t* device_status);

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libtokenbutler.so")
 
 EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb_set_projection", "tb_reset_sequence",
            "tb_get_length", "tb_append_kv", "tb_project_keys", "tb_score_tokens", "tb_select_topk",
-           "tb_sparse_decode_attention", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
+           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
 
 
 class tb_config(C.Structure):
@@ -68,6 +68,8 @@ def lib():
         L.tb_select_topk.argtypes = [vp, i32, i32, ip, i32, vp, C.POINTER(tb_select_params), vp, vp, vp]
         L.tb_sparse_decode_attention.argtypes = [vp, i32, i32, ip, i32, vp, C.POINTER(tb_select_params), vp, vp, C.c_float,
                                                  vp, vp, vp]
+        L.tb_sparse_decode_attention_static.argtypes = [vp, i32, i32, i32, i32, i32, ip, ip, i32, vp, vp, vp, i32, i32, i32,
+                                                        C.c_float, vp, vp, vp]
         L.tb_get_status.argtypes = [vp, vp, ip]
         L.tb_last_step_bytes.argtypes = [vp]
         L.tb_launch_count.argtypes = [vp]
@@ -98,6 +100,20 @@ def select_params(budget, sinks=0, recent=0, radius=0, nmode=TB_NEIGHBOR_DILATE,
 
 def torch_dtype(kv_dtype):
     return torch.bfloat16 if kv_dtype == TB_BF16 else torch.float32
+
+
+TB_STATIC_MAX_QHEADS = 64
+
+
+def sparse_decode_attention_static(kv, kv_dtype, n_q_heads, n_kv_heads, head_dim, max_seq_len, seq_slots, seq_lens, q, out,
+                                   idx=None, cnt=None, idx_stride=0, sinks=0, recent=0, sm_scale=0.0, lse=None, stream=None):
+    """Attention without a context or workspace, for callers that cannot allocate device memory
+    (fixed memory pools, threads where cudaMalloc is forbidden): scratch lives inside the library.
+    Only marshals arguments for tb_sparse_decode_attention_static; returns its status code."""
+    return lib().tb_sparse_decode_attention_static(_ptr(kv), kv_dtype, n_q_heads, n_kv_heads, head_dim, max_seq_len,
+                                                   _ints(seq_slots), _ints(seq_lens), len(seq_lens), _ptr(q), _ptr(idx),
+                                                   _ptr(cnt), idx_stride, sinks, recent, sm_scale, _ptr(out), _ptr(lse),
+                                                   _stream(stream))
 
 
 class Context:

@@ -563,3 +563,125 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
 }
 
 }  // namespace tb
+
+// ---------------------------------------------------------------------------------------------------
+// Allocation-free attention entry point.
+//
+// Some callers cannot obtain device memory at the time they need attention: a plugin running inside
+// a serving process whose memory pool is fixed at start-up, code on a latency-critical thread where a
+// cudaMalloc (which may synchronise the whole device) is forbidden, or a host that has already handed
+// all free HBM to its KV cache.  For them the split-K partials and arrival counters live in the
+// file-scope device array below instead of a caller-provided workspace.  The array is part of the
+// library image: every GPU that loads the library holds it (about 1 MB) until the process exits.
+
+namespace {
+
+constexpr int kStaticMaxQHeads = TB_STATIC_MAX_QHEADS;                 // n_seq * n_q_heads per call
+constexpr size_t kStaticPartO = (size_t)kStaticMaxQHeads * tb::kMaxSplits * 128 * sizeof(float);
+constexpr size_t kStaticPartMl = (size_t)kStaticMaxQHeads * tb::kMaxSplits * 2 * sizeof(float);
+constexpr size_t kStaticCounters = (size_t)kStaticMaxQHeads * sizeof(uint32_t);   // one per (sequence, KV head) at most
+constexpr size_t kStaticStatus = 256;
+constexpr size_t kStaticBytes = kStaticPartO + kStaticPartMl + kStaticCounters + kStaticStatus;
+
+// In host code this name is only a handle for the runtime, never a device address: the address a
+// kernel may use comes from cudaGetSymbolAddress, asked once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_scratch_addr[kMaxDevices];     // per device, filled at first use
+int g_sm_count[kMaxDevices];
+
+tb_status static_scratch_for_current_device(unsigned char** out, int* sm_count) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TB_ERR_CUDA;
+    if (!g_scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return TB_ERR_CUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TB_ERR_CUDA;
+        if (cudaFuncSetAttribute(tb::attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 tb::kAttnWarps * tb::kMmaStages * tb::kStageBytes) != cudaSuccess)
+            return TB_ERR_CUDA;
+        g_sm_count[dev] = sms;
+        g_scratch_addr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_scratch_addr[dev];
+    *sm_count = g_sm_count[dev];
+    return TB_OK;
+}
+
+}  // namespace
+
+extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32_t kv_dtype, int32_t n_q_heads, int32_t n_kv_heads,
+                                                       int32_t head_dim, int32_t max_seq_len, const int32_t* seq_slots,
+                                                       const int32_t* seq_lens, int32_t n_seq, const void* q_dev,
+                                                       const int32_t* idx_dev, const int32_t* cnt_dev, int32_t idx_stride,
+                                                       int32_t sinks, int32_t recent, float sm_scale, float* out_dev,
+                                                       float* lse_dev, void* stream) {
+    using namespace tb;
+    if (!kv_dev || !seq_lens || !q_dev || !out_dev || n_seq <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || max_seq_len <= 0)
+        return TB_ERR_INVALID_ARG;
+    if ((idx_dev == nullptr) != (cnt_dev == nullptr) || sinks < 0 || recent < 0) return TB_ERR_INVALID_ARG;
+    if (idx_dev && idx_stride <= 0) return TB_ERR_INVALID_ARG;
+    if (kv_dtype != TB_F32 && kv_dtype != TB_BF16) return TB_ERR_INVALID_ARG;
+    if (n_q_heads % n_kv_heads != 0) return TB_ERR_INVALID_ARG;
+    if (head_dim != 128 || n_q_heads / n_kv_heads > kMaxGroup) return TB_ERR_UNSUPPORTED;
+    // the fixed scratch bounds the problem: refuse anything larger instead of overrunning it
+    if (n_seq > kMaxLaunchSeq || (long long)n_seq * n_q_heads > kStaticMaxQHeads) return TB_ERR_CAPACITY;
+
+    unsigned char* scratch = nullptr;
+    int sm_count = 0;
+    tb_status st = static_scratch_for_current_device(&scratch, &sm_count);
+    if (st != TB_OK) return st;
+    float* part_o = reinterpret_cast<float*>(scratch);
+    float* part_ml = reinterpret_cast<float*>(scratch + kStaticPartO);
+    uint32_t* counters = reinterpret_cast<uint32_t*>(scratch + kStaticPartO + kStaticPartMl);
+    int32_t* status = reinterpret_cast<int32_t*>(scratch + kStaticPartO + kStaticPartMl + kStaticCounters);
+
+    Geom gm;
+    gm.n_layers = 1, gm.Hq = n_q_heads, gm.Hkv = n_kv_heads, gm.g = n_q_heads / n_kv_heads, gm.D = head_dim, gm.dp = 0;
+    gm.max_batch = 1 << 20, gm.max_seq_len = max_seq_len, gm.idx_cap = idx_dev ? idx_stride : 0, gm.dtype = kv_dtype;
+    UnitTable ut;
+    ut.layer_begin = 0, ut.layer_count = 1, ut.n_seq = n_seq;
+    int max_rows = 0;
+    for (int i = 0; i < n_seq; ++i) {
+        const int slot = seq_slots ? seq_slots[i] : i;
+        if (slot < 0 || seq_lens[i] <= 0 || seq_lens[i] > max_seq_len) return TB_ERR_INVALID_ARG;
+        ut.seq_id[i] = slot;
+        ut.len[i] = seq_lens[i];
+        int rows = seq_lens[i];
+        if (idx_dev) {
+            long long r = (long long)(sinks < rows ? sinks : rows) + idx_stride + recent;
+            if (r < rows) rows = (int)r;
+        }
+        if (rows > max_rows) max_rows = rows;
+    }
+    AttnArgs a;
+    a.q = q_dev, a.idx = idx_dev, a.cnt = cnt_dev, a.out = out_dev, a.lse = lse_dev;
+    a.dense = idx_dev ? 0 : 1, a.sinks = idx_dev ? sinks : 0, a.recent = idx_dev ? recent : 0;
+    a.list_bound = idx_dev ? idx_stride : 0;
+    a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim);
+    {   // same split rule as the context path
+        int units = n_seq * n_kv_heads, target = 4 * sm_count;
+        int n = (target + units - 1) / units, by_rows = max_rows / 64;
+        if (n > by_rows) n = by_rows;
+        if (n > kMaxSplits) n = kMaxSplits;
+        if (n < 1) n = 1;
+        a.nsplit = n;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    // the array keeps whatever the previous call left: the arrival counters and the status word must start at zero
+    if (cudaMemsetAsync(counters, 0, kStaticCounters + kStaticStatus, s) != cudaSuccess) return TB_ERR_CUDA;
+    dim3 grid(a.nsplit, n_kv_heads, n_seq);
+    // the stored-list arguments of the kernels are never read here (caller lists or dense)
+    if (kv_dtype == TB_BF16) {
+        attn_mma_kernel<<<grid, kAttnThreads, kAttnWarps * kMmaStages * kStageBytes, s>>>(
+            gm, ut, a, (const __nv_bfloat16*)kv_dev, nullptr, nullptr, part_o, part_ml, counters, status);
+    } else {
+#define TB_ATTN_S(G) attn_kernel<float, G><<<grid, kAttnThreads, 0, s>>>(gm, ut, a, (const float*)kv_dev, nullptr, nullptr, part_o, part_ml, counters, status)
+        if (gm.g == 1) TB_ATTN_S(1); else if (gm.g == 2) TB_ATTN_S(2); else if (gm.g <= 4) TB_ATTN_S(4); else TB_ATTN_S(8);
+#undef TB_ATTN_S
+    }
+    return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
+}
+

@@ -1,30 +1,38 @@
-// Importance scoring and token selection (paper Sec. 3.4 "score computation against all projected
-// keys ... top-B selection", Sec. 4 "Token Selection Policy", Sec. 3.4 "Neighbor fetching").
+// Fused importance scoring + exact top-B selection (paper Sec. 3.4 "score computation against all
+// projected keys ... top-B selection", Sec. 4 "Token Selection Policy").
 //
-//   score_kernel      materialises fp32 scores (standalone API call, not on the fast path)
-//   select_kernel     fused: streams the projected keys of one (layer, sequence, KV head) through
-//                     shared memory with 2-D TMA tiles, scores each row, keeps the scores on chip as
-//                     order-preserving 32-bit keys, and finds the exact top-B with a radix select
-//                     whose histograms are merged across a thread-block cluster through distributed
-//                     shared memory.  Output: ascending positions, ties to the lower position.
-//   neighbor_kernel   expands a selection by the DILATE or CLUSTER rule via a bitmask over the
-//                     candidate range, compacted in order.
+// One thread-block cluster (1..8 blocks) per (layer, sequence, KV head).  Each block streams its share
+// of the candidate rows of the projected-key cache through shared memory with 2-D TMA tiles, scores
+// every row, and keeps the scores on chip as order-preserving 32-bit keys (scores never go to HBM).
+// The exact top-B is a radix select on those keys:
+//   digit 1 (top 11 bits)  histogrammed while streaming; the blocks publish their non-empty bins to
+//                          each other through distributed shared memory, one cluster barrier, and
+//                          every block finds the threshold bin itself;
+//   digits 2, 3            only the keys of the threshold bin matter (a few per cent): they are
+//                          gathered at rank 0, which finishes alone and hands every rank the
+//                          threshold and its output offsets;
+//   compaction             ordered (warp ballots), ties taken in position order, ascending list
+//                          written straight to its destination.
+// Unusual inputs (more non-empty bins than a list holds, a crowded threshold bin) and single-block
+// launches take the general path: every digit through cluster-merged histograms.
 #include <cooperative_groups.h>
 
-#include "tb_common.cuh"
-#include "tb_internal.h"
+#include "tb_select.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace tb {
 
 constexpr int kSelThreads = 256;
+constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kTileRows = 256;      // rows per TMA box = one row per thread
 constexpr int kStages = 3;
-constexpr int kBins = 2048;         // 11-bit digits (the last pass uses 10 bits)
+constexpr int kBins = 2048;         // 11-bit digits (the last digit has 10 bits)
 constexpr int kMaxCluster = 8;
+constexpr int kListCap = 256;       // non-empty first-digit bins a block may publish on the fast path
+constexpr int kCandCap = 4096;      // keys of the threshold bin gathered at rank 0 (aliases merged[1..2])
 
-// Optional per-phase timestamps of block (0,0) and of the last block, for tuning builds only
+// Optional per-phase timestamps of the first and last block of unit 0, for tuning builds only
 // (-DTB_PHASE_TIMING); the product build compiles these away.
 #ifdef TB_PHASE_TIMING
 __device__ unsigned long long g_phase_ns[2][16];
@@ -42,127 +50,79 @@ extern "C" int tb_debug_phase_ns(unsigned long long* out) {
 __device__ __forceinline__ void phase_stamp(int) {}
 #endif
 
-// ---- scoring arithmetic shared by the standalone and the fused kernel --------------------------
-
-// Importance query of KV head h: sum over the g query heads of the group, in head order.
-template <int DP>
-__device__ __forceinline__ void load_group_query(const float* __restrict__ q_imp_unit, int g, float* qr) {
-#pragma unroll
-    for (int j = 0; j < DP; ++j) qr[j] = 0.f;
-    for (int u = 0; u < g; ++u)
-#pragma unroll
-        for (int j = 0; j < DP; ++j) qr[j] += q_imp_unit[u * DP + j];
-}
-
-// Dot product of one projected-key row (NCH 16-byte chunks fetched by `ld(c)`) with qr.  Two FMA
-// chains (even / odd chunks), each in ascending element order, added at the end: the result depends
-// only on the row's bytes, never on where the row sits.
-template <typename T, int DP, typename LoadChunk>
-__device__ __forceinline__ float row_score(const float* qr, LoadChunk ld) {
-    constexpr int P = Elem<T>::kPer16;
-    constexpr int NCH = DP / P;
-    float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-        uint4 v = ld(c);
-        float f[P];
-        Elem<T>::unpack16(v, f);
-        if (c & 1) {
-#pragma unroll
-            for (int e = 0; e < P; ++e) acc1 = fmaf(qr[c * P + e], f[e], acc1);
-        } else {
-#pragma unroll
-            for (int e = 0; e < P; ++e) acc0 = fmaf(qr[c * P + e], f[e], acc0);
-        }
-    }
-    return acc0 + acc1;
-}
-
-__device__ __forceinline__ void decode_unit(const Geom& gm, const UnitTable& ut, int u, int& ll, int& s, int& h) {
-    h = u % gm.Hkv;
-    s = (u / gm.Hkv) % ut.n_seq;
-    ll = u / (gm.Hkv * ut.n_seq);
-}
-__device__ __forceinline__ size_t cache_unit(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
-    return ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h;
-}
-
-// ---- standalone scores ---------------------------------------------------------------------------
-
-template <typename T, int DP>
-__global__ void __launch_bounds__(256) score_kernel(Geom gm, UnitTable ut, const float* __restrict__ q_imp, float scale,
-                                                    const T* __restrict__ kimp, float* __restrict__ scores) {
-    constexpr int NCH = DP / Elem<T>::kPer16;
-    int ll, s, h;
-    decode_unit(gm, ut, blockIdx.y, ll, s, h);
-    const int L = ut.len[ll * ut.n_seq + s];
-    float qr[DP];
-    load_group_query<DP>(q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
-    const uint4* base = reinterpret_cast<const uint4*>(kimp + cache_unit(gm, ut, ll, s, h) * gm.max_seq_len * DP);
-    float* out = scores + ((size_t)(ll * ut.n_seq + s) * gm.Hkv + h) * gm.max_seq_len;
-    for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < L; t += gridDim.x * blockDim.x) {
-        const uint4* row = base + (size_t)t * NCH;
-        float sc = row_score<T, DP>(qr, [&](int c) { return __ldg(row + c); });
-        out[t] = scale * sc;
-    }
-}
-
-cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, float scale, float* scores, cudaStream_t s) {
-    const Geom& gm = c->geom;
-    int maxL = 0;
-    for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) maxL = ut.len[i] > maxL ? ut.len[i] : maxL;
-    if (maxL == 0) return cudaSuccess;
-    dim3 grid((maxL + 255) / 256, ut.layer_count * ut.n_seq * gm.Hkv);
-    if (grid.x > 64) grid.x = 64;
-#define TB_SCORE(T, DP) score_kernel<T, DP><<<grid, 256, 0, s>>>(gm, ut, q_imp, scale, (const T*)c->kimp, scores)
-    if (gm.dtype == TB_BF16) {
-        if (gm.dp == 32) TB_SCORE(__nv_bfloat16, 32); else TB_SCORE(__nv_bfloat16, 16);
-    } else {
-        if (gm.dp == 32) TB_SCORE(float, 32); else TB_SCORE(float, 16);
-    }
-#undef TB_SCORE
-    return cudaGetLastError();
-}
-
-// ---- fused score + exact top-B -------------------------------------------------------------------
-
-struct SelSmem {
+struct __align__(16) SelSmem {
+    int res[8];                         // rank 0's verdict: prefix, low_bits, krem, gt_base, eq_base (16-byte stores)
     uint64_t full[kStages];
-    int warp_a[kSelThreads / 32];
-    int warp_b[kSelThreads / 32];
+    int warp_a[kSelWarps];
+    int warp_b[kSelWarps];
     int tot[kMaxCluster][2];
-    int bc_bin, bc_krem, bc_count;
+    int bc_bin, bc_krem, bc_count, pad0;
+    int list_len[kMaxCluster];          // per rank: entries in lists[rank]
+    int above[kMaxCluster];             // per rank: keys in bins above the threshold bin
+    int inbin[kMaxCluster];             // per rank: keys in the threshold bin
+    uint32_t lists[kMaxCluster][kListCap];   // (bin << 16 | count) of every rank's non-empty bins
 };
 
-// Finds, over `nbins` counters ordered by digit value, the digit b with
-//   count(digits > b) < k <= count(digits >= b)
-// and returns it with k' = k - count(digits > b) and the population of b.  All threads call it and
-// all receive the same answer.  k >= 1 and k <= total count are preconditions.
-__device__ __forceinline__ void find_digit(const int* __restrict__ hist, int nbins, int k, SelSmem* sm, int& bin, int& krem,
-                                           int& bcount) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = nbins / kSelThreads;             // 8 or 4 digits per thread, highest digits first
-    const int top = nbins - 1 - tid * per;
-    int mine = 0;
-    for (int i = 0; i < per; ++i) mine += hist[top - i];
-    int incl = warp_incl_scan(mine, lane);
-    if (lane == 31) sm->warp_a[warp] = incl;
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void smem_add(int* p, int v) {
+    asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
+}
+
+// PER consecutive counters of thread `tid` (16-byte loads, at most 2-way bank conflicts).
+template <int PER>
+__device__ __forceinline__ void load_bins(const int* hist, int tid, int (&b)[PER]) {
+    const int4* p = reinterpret_cast<const int4*>(hist + tid * PER);
+#pragma unroll
+    for (int v = 0; v < PER / 4; ++v) {
+        const int4 x = p[v];
+        b[4 * v] = x.x, b[4 * v + 1] = x.y, b[4 * v + 2] = x.z, b[4 * v + 3] = x.w;
+    }
+}
+
+// Exclusive prefix of `v` over the block in thread order, and the block total.  One barrier; uses
+// `slots` (kSelWarps ints), which must not be reused before the next barrier.
+__device__ __forceinline__ int block_excl_scan(int v, int* slots, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int incl = warp_incl_scan(v, lane);
+    if (lane == 31) slots[warp] = incl;
     __syncthreads();
     int before = 0;
-    for (int w = 0; w < warp; ++w) before += sm->warp_a[w];
-    incl += before;
-    int excl = incl - mine;
-    if (excl < k && k <= incl) {                     // exactly one thread
-        int run = excl;
-        for (int i = 0; i < per; ++i) {
-            int cnt = hist[top - i];
-            if (run + cnt >= k) {
-                sm->bc_bin = top - i;
-                sm->bc_krem = k - run;
-                sm->bc_count = cnt;
-                break;
+    total = 0;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+        const int x = slots[w];
+        total += x;
+        before += w < warp ? x : 0;
+    }
+    return before + incl - v;
+}
+
+// Finds, over PER*256 counters ordered by digit value, the digit b with
+//   count(digits > b) < k <= count(digits >= b)
+// and returns it with k' = k - count(digits > b) and the population of b.  All threads call it and
+// all receive the same answer.  Preconditions: 1 <= k <= total count.
+template <int PER>
+__device__ __forceinline__ void find_digit(const int* hist, int k, SelSmem* sm, int& bin, int& krem, int& bcount) {
+    const int tid = threadIdx.x;
+    int b[PER];
+    load_bins<PER>(hist, tid, b);
+    int mine = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) mine += b[i];
+    int total;
+    const int excl = block_excl_scan(mine, sm->warp_a, total);
+    const int above = total - excl - mine;           // keys in digits above this thread's digits
+    if (above < k && k <= above + mine) {            // exactly one thread
+        int run = above;
+        bool done = false;
+#pragma unroll
+        for (int i = PER - 1; i >= 0; --i) {
+            if (!done && run + b[i] >= k) {
+                sm->bc_bin = tid * PER + i, sm->bc_krem = k - run, sm->bc_count = b[i];
+                done = true;
             }
-            run += cnt;
+            run += b[i];
         }
     }
     __syncthreads();
@@ -190,6 +150,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     const int C = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned lt_mask = (1u << lane) - 1u;
 
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
@@ -224,7 +185,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         fence_mbar_init();
     }
     __syncthreads();
-    if (C > 1) cluster.sync();                         // every block's merged histograms are zero before any push
+    // Split cluster barrier: arrive now, wait only before the first access to a peer's shared memory
+    // (after the streaming phase), so its latency hides behind the loads.
+    if (C > 1) cluster_arrive();
 
     phase_stamp(1);
     const int n_tiles = (ncand + kTileRows - 1) / kTileRows;
@@ -260,7 +223,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             });
             uint32_t key = order_key(sc);
             keys[slot] = key;
-            atomicAdd(&hist[key >> 21], 1);
+            smem_add(&hist[key >> 21], 1);
         }
         __syncthreads();                               // all reads of this stage are done
         if (tid == 0 && i + kStages < my_tiles) {
@@ -273,13 +236,160 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
     phase_stamp(2);
 
-    // ---- radix select: three digits (11, 11, 10 bits), histograms merged over the cluster --------
     uint32_t prefix = 0;          // digits fixed so far (value of key >> low_bits)
     int low_bits = 32;            // bits of the key not yet fixed
     int krem = k;
     bool exact = false;           // the class {key >> low_bits == prefix} is taken whole
+    int start_pass = 0;
+    bool have_bases = false;      // fast path: taken / class counts of the lower ranks are already known
+    int gt_base = 0, eq_base = 0;
+
+    // ---- fast path over a cluster ----------------------------------------------------------------
+    if (C > 1) {
+        // my non-empty first-digit bins -> lists[rank] (own copy), then the same entries to every peer
+        int b[8];
+        load_bins<8>(hist, tid, b);
+        int nz = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) nz += b[i] != 0;
+        int total;
+        int off = block_excl_scan(nz, sm->warp_b, total);
+        if (total <= kListCap) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (b[i]) sm->lists[rank][off++] = ((uint32_t)(tid * 8 + i) << 16) | (uint32_t)b[i];
+        }
+        if (tid == 0) sm->list_len[rank] = total;
+        __syncthreads();
+        cluster_wait();                                // all peers run and have zeroed their histograms
+        if (total <= kListCap) {
+            for (int r = 1; r < C; ++r) {              // one remote store per thread and peer
+                const int peer = (rank + r) % C;
+                if (tid < total) *cluster.map_shared_rank(&sm->lists[rank][tid], peer) = sm->lists[rank][tid];
+            }
+        }
+        if (tid < C && tid != rank) *cluster.map_shared_rank(&sm->list_len[rank], tid) = total;
+        phase_stamp(8);
+        cluster.sync();                                // barrier 1
+        phase_stamp(9);
+        bool fast = true;
+        for (int r = 0; r < C; ++r) fast = fast && sm->list_len[r] <= kListCap;
+        if (fast) {
+            // warp w merges rank w's list into merged[0] (still zero)
+            if (warp < C)
+                for (int i = lane; i < sm->list_len[warp]; i += 32) {
+                    const uint32_t e = sm->lists[warp][i];
+                    smem_add(&merged[e >> 16], (int)(e & 0xFFFFu));
+                }
+            __syncthreads();
+            int bin, kr, bc;
+            find_digit<8>(merged, k, sm, bin, kr, bc);
+            prefix = (uint32_t)bin, low_bits = 21, krem = kr, start_pass = 1;
+            if (warp < C) {                            // warp w sums rank w's list around the threshold bin
+                int ab = 0, ib = 0;
+                for (int i = lane; i < sm->list_len[warp]; i += 32) {
+                    const uint32_t e = sm->lists[warp][i];
+                    const int eb = (int)(e >> 16), ec = (int)(e & 0xFFFFu);
+                    ab += eb > bin ? ec : 0;
+                    ib += eb == bin ? ec : 0;
+                }
+                ab = warp_sum_int(ab), ib = warp_sum_int(ib);
+                if (lane == 0) sm->above[warp] = ab, sm->inbin[warp] = ib;
+            }
+            for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
+            __syncthreads();
+            phase_stamp(10);
+            if (bc == kr) {                            // the whole threshold bin is taken: nothing to refine
+                exact = true, have_bases = true, start_pass = 3;
+                for (int r = 0; r < rank; ++r) gt_base += sm->above[r], eq_base += sm->inbin[r];
+            } else if (bc <= kCandCap) {
+                // my keys of the threshold bin -> rank 0 (any order inside my region)
+                const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
+                const int n_vec = (n_local + 3) / 4;
+                int mine = 0;
+                for (int v = tid; v < n_vec; v += kSelThreads) {
+                    const uint4 x = keys4[v];
+                    const int base = v * 4;
+                    mine += (base < n_local && (x.x >> 21) == (uint32_t)bin) + (base + 1 < n_local && (x.y >> 21) == (uint32_t)bin) +
+                            (base + 2 < n_local && (x.z >> 21) == (uint32_t)bin) + (base + 3 < n_local && (x.w >> 21) == (uint32_t)bin);
+                }
+                int tot_mine;
+                int pos = block_excl_scan(mine, sm->warp_b, tot_mine);
+                for (int r = 0; r < rank; ++r) pos += sm->inbin[r];
+                uint32_t* cand_local = reinterpret_cast<uint32_t*>(merged + kBins);
+                uint32_t* cand0 = cluster.map_shared_rank(cand_local, 0);
+                if (mine) {
+                    for (int v = tid; v < n_vec; v += kSelThreads) {
+                        const uint4 x = keys4[v];
+                        const int base = v * 4;
+                        if (base < n_local && (x.x >> 21) == (uint32_t)bin) cand0[pos++] = x.x;
+                        if (base + 1 < n_local && (x.y >> 21) == (uint32_t)bin) cand0[pos++] = x.y;
+                        if (base + 2 < n_local && (x.z >> 21) == (uint32_t)bin) cand0[pos++] = x.z;
+                        if (base + 3 < n_local && (x.w >> 21) == (uint32_t)bin) cand0[pos++] = x.w;
+                    }
+                }
+                phase_stamp(11);
+                cluster.sync();                        // barrier 2
+                phase_stamp(12);
+                if (rank == 0) {
+                    uint32_t pf = (uint32_t)bin;
+                    int lb = 21, kk = kr;
+                    bool ex = false;
 #pragma unroll 1
-    for (int pass = 0; pass < 3; ++pass) {
+                    for (int pass = 1; pass < 3 && !ex; ++pass) {
+                        const int bits = pass == 2 ? 10 : 11, nb = 1 << bits, shift = lb - bits;
+#pragma unroll 4
+                        for (int i = tid; i < bc; i += kSelThreads) {
+                            const uint32_t key = cand_local[i];
+                            if ((key >> lb) == pf) smem_add(&hist[(key >> shift) & (nb - 1)], 1);
+                        }
+                        __syncthreads();
+                        int d, kr2, c2;
+                        if (pass == 1) find_digit<8>(hist, kk, sm, d, kr2, c2);
+                        else find_digit<4>(hist, kk, sm, d, kr2, c2);
+                        pf = (pf << bits) | (uint32_t)d, lb = shift, kk = kr2;
+                        ex = c2 == kr2;
+                        if (!ex) {
+                            for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
+                            __syncthreads();
+                        }
+                    }
+                    if (warp < C) {                    // warp w counts rank w's candidates against the threshold
+                        int base_w = 0;
+                        for (int r = 0; r < warp; ++r) base_w += sm->inbin[r];
+                        const int n_w = sm->inbin[warp];
+                        int gt = 0, eq = 0;
+#pragma unroll 4
+                        for (int i = lane; i < n_w; i += 32) {
+                            const uint32_t kk2 = cand_local[base_w + i] >> lb;
+                            gt += kk2 > pf, eq += kk2 == pf;
+                        }
+                        gt = warp_sum_int(gt), eq = warp_sum_int(eq);
+                        if (lane == 0) sm->warp_a[warp] = gt, sm->warp_b[warp] = eq;
+                    }
+                    __syncthreads();
+                    if (tid < C) {
+                        int gb = 0, eb = 0;
+                        for (int r = 0; r < tid; ++r) gb += sm->above[r] + sm->warp_a[r], eb += sm->warp_b[r];
+                        int4* dst = reinterpret_cast<int4*>(cluster.map_shared_rank(&sm->res[0], tid));
+                        dst[0] = make_int4((int)pf, lb, kk, gb);
+                        dst[1] = make_int4(eb, 0, 0, 0);
+                    }
+                }
+                phase_stamp(13);
+                cluster.sync();                        // barrier 3
+                phase_stamp(14);
+                prefix = (uint32_t)sm->res[0], low_bits = sm->res[1], krem = sm->res[2];
+                gt_base = sm->res[3], eq_base = sm->res[4];
+                exact = true, have_bases = true, start_pass = 3;   // nothing left for the general passes
+            }
+        }
+    }
+    phase_stamp(3);
+
+    // ---- general path: digits not yet fixed are found with cluster-merged histograms ----------------
+#pragma unroll 1
+    for (int pass = start_pass; pass < 3; ++pass) {
         const int bits = pass == 2 ? 10 : 11;
         const int nbins = 1 << bits;
         const int shift = low_bits - bits;
@@ -287,7 +397,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             if (!exact) {
                 for (int i = tid; i < n_local; i += kSelThreads) {
                     uint32_t key = keys[i];
-                    if ((key >> low_bits) == prefix) atomicAdd(&hist[(key >> shift) & (nbins - 1)], 1);
+                    if ((key >> low_bits) == prefix) smem_add(&hist[(key >> shift) & (nbins - 1)], 1);
                 }
             }
             __syncthreads();
@@ -306,7 +416,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         }
         if (!exact) {
             int bin, kr, bc;
-            find_digit(src, nbins, krem, sm, bin, kr, bc);
+            if (pass == 2) find_digit<4>(src, krem, sm, bin, kr, bc);
+            else find_digit<8>(src, krem, sm, bin, kr, bc);
             prefix = (prefix << bits) | (uint32_t)bin;
             low_bits = shift;
             krem = kr;
@@ -314,17 +425,17 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
         }
         __syncthreads();
-        phase_stamp(3 + pass);
     }
 
     // ---- ordered compaction ------------------------------------------------------------------------
     // A slot is taken if its key is above the class, or inside the class and among the class's first
-    // `krem` members in position order (the lower-position tie rule).
+    // `krem` members in position order (the lower-position tie rule).  Warp w owns a contiguous range.
     const int seg = ((n_local + kSelThreads - 1) / kSelThreads) * 32;   // slots per warp, multiple of 32
     const int seg_begin = min(n_local, warp * seg), seg_end = min(n_local, (warp + 1) * seg);
     int n_gt = 0, n_eq = 0;
+#pragma unroll 4
     for (int i = seg_begin + lane; i < seg_end; i += 32) {
-        uint32_t kk = keys[i] >> low_bits;
+        const uint32_t kk = keys[i] >> low_bits;
         n_gt += kk > prefix;
         n_eq += kk == prefix;
     }
@@ -333,11 +444,15 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     if (lane == 0) sm->warp_a[warp] = n_gt, sm->warp_b[warp] = n_eq;
     __syncthreads();
     int gt_before = 0, eq_before = 0, gt_cta = 0, eq_cta = 0;
-    for (int w = 0; w < kSelThreads / 32; ++w) {
-        if (w < warp) gt_before += sm->warp_a[w], eq_before += sm->warp_b[w];
-        gt_cta += sm->warp_a[w], eq_cta += sm->warp_b[w];
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+        const int x = sm->warp_a[w], y = sm->warp_b[w];
+        gt_before += w < warp ? x : 0, eq_before += w < warp ? y : 0;
+        gt_cta += x, eq_cta += y;
     }
-    if (C > 1) {
+    if (have_bases) {
+        gt_before += gt_base, eq_before += eq_base;
+    } else if (C > 1) {
         if (tid < C) {
             int* dst = cluster.map_shared_rank(&sm->tot[rank][0], tid);
             dst[0] = gt_cta, dst[1] = eq_cta;
@@ -347,19 +462,25 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     }
     phase_stamp(6);
     int out_pos = gt_before + min(eq_before, krem);
-    const unsigned lt_mask = (1u << lane) - 1u;
-    for (int i0 = seg_begin; i0 < seg_end; i0 += 32) {
-        const int i = i0 + lane;
-        uint32_t kk = 0;
-        bool in = i < seg_end;
-        if (in) kk = keys[i] >> low_bits;
-        const bool is_gt = in && kk > prefix, is_eq = in && kk == prefix;
-        const unsigned eq_ballot = __ballot_sync(0xffffffffu, is_eq);
-        const bool take = is_gt || (is_eq && eq_before + __popc(eq_ballot & lt_mask) < krem);
-        const unsigned take_ballot = __ballot_sync(0xffffffffu, take);
-        if (take) idx_dst[out_pos + __popc(take_ballot & lt_mask)] = tok0 + i;
-        out_pos += __popc(take_ballot);
-        eq_before += __popc(eq_ballot);
+    for (int i0 = seg_begin; i0 < seg_end; i0 += 128) {
+        uint32_t kk[4];
+        bool in[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {                  // four independent loads before the ballots
+            const int i = i0 + u * 32 + lane;
+            in[u] = i < seg_end;
+            kk[u] = in[u] ? keys[i] >> low_bits : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const bool is_gt = in[u] && kk[u] > prefix, is_eq = in[u] && kk[u] == prefix;
+            const unsigned eq_ballot = __ballot_sync(0xffffffffu, is_eq);
+            const bool take = is_gt || (is_eq && eq_before + __popc(eq_ballot & lt_mask) < krem);
+            const unsigned take_ballot = __ballot_sync(0xffffffffu, take);
+            if (take) idx_dst[out_pos + __popc(take_ballot & lt_mask)] = tok0 + i0 + u * 32 + lane;
+            out_pos += __popc(take_ballot);
+            eq_before += __popc(eq_ballot);
+        }
     }
     if (rank == 0 && tid == 0) *cnt_dst = k;
     phase_stamp(7);
@@ -380,7 +501,7 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     }
     const int n_tiles = (max_cand + kTileRows - 1) / kTileRows;
     // Cluster size: enough blocks to cover the GPU about twice, at least 4 tiles per block, and a
-    // key array per block of at most 64 KB.
+    // key array per block of at most 32 KB where the cluster limit allows (64 KB otherwise).
     int C = 1;
     while (C < kMaxCluster && (n_units * C < 2 * c->sm_count && n_tiles / (2 * C) >= 4)) C *= 2;
     while (C < kMaxCluster && (n_tiles + C - 1) / C * kTileRows > 8192) C *= 2;
@@ -420,116 +541,6 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
         if (gm.dp == 32) TB_SEL(float, 32); else TB_SEL(float, 16);
     }
 #undef TB_SEL
-}
-
-// ---- neighbour fetching ---------------------------------------------------------------------------
-
-constexpr int kNbThreads = 256;
-
-__global__ void __launch_bounds__(kNbThreads) neighbor_kernel(Geom gm, UnitTable ut, NeighborArgs a, int32_t* __restrict__ state_idx,
-                                                              int32_t* __restrict__ state_cnt) {
-    extern __shared__ uint32_t mask[];               // one bit per candidate position
-    __shared__ int warp_tot[kNbThreads / 32];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int ll, s, h;
-    decode_unit(gm, ut, blockIdx.x, ll, s, h);
-    const int L = ut.len[ll * ut.n_seq + s];
-    const int lo = min(a.sinks, L), hi = max(lo, L - a.recent);
-    const int span = hi - lo;
-    const int n_words = (span + 31) / 32;
-    const int32_t* src = a.idx_src + (size_t)blockIdx.x * a.src_stride;
-    const int cnt = a.cnt_src[blockIdx.x];
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
-    int32_t* dst = state_idx + cu * gm.idx_cap;
-
-    for (int i = tid; i < n_words; i += kNbThreads) mask[i] = 0;
-    __syncthreads();
-    auto mark = [&](int p) {
-        if (p >= lo && p < hi) atomicOr(&mask[(p - lo) >> 5], 1u << ((p - lo) & 31));
-    };
-    const int r = a.radius;
-    for (int i = tid; i < cnt; i += kNbThreads) {
-        const int p = src[i];
-        if (a.nmode == TB_NEIGHBOR_DILATE) {
-            for (int d = -r; d <= r; ++d) mark(p + d);
-        } else {
-            mark(p);
-            if (i == 0 || src[i - 1] != p - 1) {       // first token of a run of consecutive positions
-                int j = i;
-                while (j + 1 < cnt && src[j + 1] == src[j] + 1) ++j;
-                const int b = src[j], n = r * (b - p + 1);
-                const int right = (n + 1) / 2, left = n / 2;
-                for (int x = b + 1; x <= b + right; ++x) mark(x);
-                for (int x = p - left; x <= p - 1; ++x) mark(x);
-            }
-        }
-    }
-    __syncthreads();
-
-    // ordered compaction of the bitmask: each warp owns a contiguous range of words
-    const int wseg = ((n_words + kNbThreads - 1) / kNbThreads) * 32;
-    const int wb = min(n_words, warp * wseg), we = min(n_words, (warp + 1) * wseg);
-    int tot = 0;
-    for (int i = wb + lane; i < we; i += 32) tot += __popc(mask[i]);
-    tot = warp_sum_int(tot);
-    if (lane == 0) warp_tot[warp] = tot;
-    __syncthreads();
-    int pos = 0, all = 0;
-    for (int w = 0; w < kNbThreads / 32; ++w) {
-        if (w < warp) pos += warp_tot[w];
-        all += warp_tot[w];
-    }
-    for (int i0 = wb; i0 < we; i0 += 32) {
-        const int i = i0 + lane;
-        uint32_t m = i < we ? mask[i] : 0u;
-        const int c = __popc(m);
-        const int incl = warp_incl_scan(c, lane);
-        int o = pos + incl - c;
-        while (m) {
-            int bit = __ffs(m) - 1;
-            m &= m - 1;
-            dst[o++] = lo + i * 32 + bit;
-        }
-        pos += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (tid == 0) state_cnt[cu] = all;
-}
-
-cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s) {
-    const Geom& gm = c->geom;
-    int max_span = 0;
-    for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) {
-        int L = ut.len[i], lo = a.sinks < L ? a.sinks : L, hi = L - a.recent > lo ? L - a.recent : lo;
-        if (hi - lo > max_span) max_span = hi - lo;
-    }
-    size_t smem = (size_t)((max_span + 31) / 32) * 4 + 16;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(neighbor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
-    neighbor_kernel<<<ut.layer_count * ut.n_seq * gm.Hkv, kNbThreads, smem, s>>>(gm, ut, a, c->st.idx, c->st.cnt);
-    return cudaGetLastError();
-}
-
-// ---- copy stored lists out --------------------------------------------------------------------------
-
-__global__ void copy_lists_kernel(Geom gm, UnitTable ut, const int32_t* __restrict__ state_idx, const int32_t* __restrict__ state_cnt,
-                                  int32_t* __restrict__ idx_out, int32_t* __restrict__ cnt_out) {
-    int ll, s, h;
-    decode_unit(gm, ut, blockIdx.x, ll, s, h);
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
-    const int n = state_cnt[cu];
-    if (idx_out)
-        for (int i = threadIdx.x; i < n; i += blockDim.x) idx_out[(size_t)blockIdx.x * gm.idx_cap + i] = state_idx[cu * gm.idx_cap + i];
-    if (cnt_out && threadIdx.x == 0) cnt_out[blockIdx.x] = n;
-}
-
-cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s) {
-    copy_lists_kernel<<<ut.layer_count * ut.n_seq * c->geom.Hkv, 256, 0, s>>>(c->geom, ut, c->st.idx, c->st.cnt, idx_out, cnt_out);
-    return cudaGetLastError();
 }
 
 }  // namespace tb

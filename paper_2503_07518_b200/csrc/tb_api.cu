@@ -169,7 +169,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     g.D = cfg->head_dim, g.dp = cfg->imp_dim, g.max_batch = cfg->max_batch, g.max_seq_len = cfg->max_seq_len;
     g.idx_cap = l.idx_cap, g.dtype = cfg->kv_dtype;
     const size_t n = (size_t)cfg->n_layers * cfg->max_batch;
-    c->len.assign(n, 0), c->len_proj.assign(n, 0), c->has_sel.assign(n, 0);
+    c->len.assign(n, 0), c->len_proj.assign(n, 0), c->has_sel.assign(n, 0), c->sel_cnt.assign(n, -1);
     c->last_bytes = 0, c->launches = 0;
     c->tile_rows = 256;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete c; return TB_ERR_CUDA; }
@@ -206,7 +206,7 @@ tb_status tb_reset_sequence(tb_ctx* c, int32_t seq) {
     if (!c || seq < 0 || seq >= c->cfg.max_batch) return TB_ERR_INVALID_ARG;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const size_t i = (size_t)l * c->cfg.max_batch + seq;
-        c->len[i] = c->len_proj[i] = c->has_sel[i] = 0;
+        c->len[i] = c->len_proj[i] = c->has_sel[i] = 0, c->sel_cnt[i] = -1;
     }
     return TB_OK;
 }
@@ -318,7 +318,7 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                 if (c->len[u] <= 0) return TB_ERR_INVALID_ARG;
                 int lo, hi;
                 cand_range(c->len[u], p->sinks, p->recent, &lo, &hi);
-                if (hi - lo > 8 * 16384) return TB_ERR_UNSUPPORTED;          // 8 blocks x 16384 on-chip scores
+                if (hi - lo > 8 * 32768) return TB_ERR_UNSUPPORTED;          // 8 blocks x 32768 on-chip scores
                 if (c->len_proj[u] < hi) return TB_ERR_UNPROJECTED;
                 bytes += (uint64_t)(hi - lo) * c->cfg.n_kv_heads * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);
             }
@@ -361,7 +361,14 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
     }
     if (refresh) {
         for (int l = lb; l < lb + lc; ++l)
-            for (int i = 0; i < n_seq; ++i) c->has_sel[(size_t)l * mb + seqs[i]] = 1;
+            for (int i = 0; i < n_seq; ++i) {
+                const size_t u = (size_t)l * mb + seqs[i];
+                c->has_sel[u] = 1;
+                int lo, hi;
+                cand_range(c->len[u], p->sinks, p->recent, &lo, &hi);
+                // without neighbour expansion the stored count is known here: min(budget, candidates)
+                c->sel_cnt[u] = p->radius == 0 ? (p->budget < hi - lo ? p->budget : hi - lo) : -1;
+            }
         c->last_bytes = bytes;
     }
     return TB_OK;
@@ -413,6 +420,9 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
         a.lse = lse ? lse + hq_off : nullptr;
         a.dense = dense, a.sinks = dense ? 0 : p->sinks, a.recent = dense ? 0 : p->recent;
         a.list_bound = bound;
+        for (int l = 0; l < n; ++l)
+            for (int i = 0; i < n_seq; ++i)
+                a.known_cnt[l * n_seq + i] = (dense || idx) ? -1 : c->sel_cnt[(size_t)(l0 + l) * mb + seqs[i]];
         a.nsplit = 0;
         a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)c->cfg.head_dim);
         if (launch_attention(c, ut, a, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;

@@ -5,14 +5,19 @@
 // memory) is loaded once and shared by the g query heads of its KV head.  Each split keeps an online
 // softmax (m, l, o) per query head; the last block to arrive for a (sequence, KV head) merges the
 // splits in split order, so the result is bit-reproducible.
+#include <cooperative_groups.h>
+
 #include "tb_common.cuh"
 #include "tb_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace tb {
 
 constexpr int kAttnThreads = 128;
 constexpr int kAttnWarps = kAttnThreads / 32;
 constexpr int kRowsPerIter = 4;
+constexpr int kAttnMaxCluster = 16;      // splits that can be merged inside a thread-block cluster (16 is non-portable)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -141,7 +146,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
     rm.w_begin = a.dense ? 0 : max(rm.n_sink, L - a.recent);
     int n_list = 0;
     if (!a.dense) {
-        n_list = a.idx ? a.cnt[lu] : state_cnt[cu];
+        const int known = a.known_cnt[ll * ut.n_seq + s];
+        n_list = a.idx ? a.cnt[lu] : (known >= 0 ? known : state_cnt[cu]);
         n_list = max(0, min(n_list, gm.idx_cap));
     }
     rm.n_list = n_list;
@@ -256,22 +262,25 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
 }
 
 // ---------------------------------------------------------------------------------------------------
-// bf16 path: tensor-core tiles of (query heads padded to 16) x (16 gathered tokens).
+// bf16 path: tensor-core tiles of (16 gathered tokens) x (query heads padded to 8).
 //
 // Each warp owns a ring of shared-memory stages; a stage holds 16 gathered K|V row pairs (512 B each,
-// fetched by one bulk copy per row through the TMA engine, completion counted on the stage's
-// mbarrier) at a 528-byte pitch so that ldmatrix reads are bank-conflict free.  S = Q K^T and
-// O += P V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate); P is split into a bf16 high and low
-// part so that the probabilities keep ~16 bits.  The GQA group's heads are the M rows of the tiles,
-// which is where batch x group makes the contraction a real dense tile.
+// copied by the whole warp with 16-byte cp.async) at a 528-byte pitch so that ldmatrix reads are
+// bank-conflict free.  S = K Q^T (tokens x heads) and O^T += V^T P^T (channels x heads) run on
+// mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the GQA group's heads as the N = 8 columns --
+// the one place where batch x group makes the contraction a real dense tile; P is split into a bf16
+// high and low part (two MMAs) so that the probabilities keep ~16 bits, and reaches the B operand
+// through movmatrix transposes.  24 MMAs per 16 tokens.
 
 #ifdef TB_PHASE_TIMING
 __device__ unsigned long long g_attn_phase_ns[2][16];
+__device__ unsigned long long g_attn_blk_ns[7][1024];   // per block of the last launch: every stamp
 __device__ __forceinline__ void attn_stamp(int i) {
-    if (threadIdx.x == 0 && (i == 0 || i == 6)) {    // slots 8/9 of row 0: earliest start / latest end over all blocks
+    if (threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        if (i == 0) atomicMin(&g_attn_phase_ns[0][8], t); else atomicMax(&g_attn_phase_ns[0][9], t);
+        const int b = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        if (b < 1024 && i < 7) g_attn_blk_ns[i][b] = t;
     }
     if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
         unsigned long long t;
@@ -282,11 +291,13 @@ __device__ __forceinline__ void attn_stamp(int i) {
 extern "C" int tb_debug_attn_phase_ns(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, g_attn_phase_ns, sizeof(g_attn_phase_ns));
 }
+extern "C" int tb_debug_attn_blocks_ns(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_attn_blk_ns, sizeof(g_attn_blk_ns));
+}
 #else
 __device__ __forceinline__ void attn_stamp(int) {}
 #endif
 
-constexpr int kMmaStages = 3;
 constexpr int kTileTok = 16;
 constexpr int kRowPitch = 528;                        // 512 B of K|V + 16 B pad
 constexpr int kStageBytes = kTileTok * kRowPitch;     // 8448
@@ -302,20 +313,32 @@ __device__ __forceinline__ void mma_bf16(float* d, uint32_t a0, uint32_t a1, uin
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// Transposes an 8x8 matrix of 16-bit elements held one 32-bit pair per lane.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTable ut, AttnArgs a, const __nv_bfloat16* __restrict__ kv,
-                                                                const int32_t* __restrict__ state_idx,
-                                                                const int32_t* __restrict__ state_cnt, float* __restrict__ part_o,
-                                                                float* __restrict__ part_ml, uint32_t* __restrict__ counters,
-                                                                int32_t* __restrict__ status) {
+// NW warps per block.  With a.cluster_merge the blocks of one (sequence, KV head) form a thread-block
+// cluster (one block per split): every block writes its (m, l, o) into rank 0's shared memory through
+// distributed shared memory, one cluster barrier, and rank 0 merges in rank order -- no partials in
+// global memory, no last-block round trips.  Without it (more splits than a cluster holds) the splits
+// go through the global workspace and the last block to arrive merges them (NW must be 4 then).
+template <int NW, int kMmaStages>
+__global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut, AttnArgs a, const __nv_bfloat16* __restrict__ kv,
+                                                           const int32_t* __restrict__ state_idx,
+                                                           const int32_t* __restrict__ state_cnt, float* __restrict__ part_o,
+                                                           float* __restrict__ part_ml, uint32_t* __restrict__ counters,
+                                                           int32_t* __restrict__ status) {
     constexpr int D = 128;
+    constexpr int kMergePitch = 132;                  // floats per (rank, head) slot: 128 channels, m, l, pad
     extern __shared__ __align__(128) unsigned char smem_dyn[];
-    __shared__ uint64_t full[kAttnWarps][kMmaStages];
-    __shared__ float sh_m[kAttnWarps][kMaxGroup], sh_l[kAttnWarps][kMaxGroup];
+    __shared__ float sh_m[NW][kMaxGroup], sh_l[NW][kMaxGroup];
     __shared__ int sh_last;
 
     attn_stamp(0);
@@ -334,7 +357,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
     rm.w_begin = a.dense ? 0 : max(rm.n_sink, L - a.recent);
     int n_list = 0;
     if (!a.dense) {
-        n_list = a.idx ? a.cnt[lu] : state_cnt[cu];
+        const int known = a.known_cnt[ll * ut.n_seq + s];
+        n_list = a.idx ? a.cnt[lu] : (known >= 0 ? known : state_cnt[cu]);
         n_list = max(0, min(n_list, gm.idx_cap));
     }
     rm.n_list = n_list;
@@ -345,7 +369,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
     const int r_begin = (int)((long long)n_rows * split / a.nsplit);
     const int r_end = (int)((long long)n_rows * (split + 1) / a.nsplit);
     const int tiles_all = (r_end - r_begin + kTileTok - 1) / kTileTok;
-    const int tiles_per_warp = (tiles_all + kAttnWarps - 1) / kAttnWarps;
+    const int tiles_per_warp = (tiles_all + NW - 1) / NW;
     const int wb = min(r_end, r_begin + warp * tiles_per_warp * kTileTok);
     const int we = min(r_end, wb + tiles_per_warp * kTileTok);
     const int n_tiles = (we - wb + kTileTok - 1) / kTileTok;
@@ -353,57 +377,72 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
     unsigned char* my_stage = smem_dyn + (size_t)warp * kMmaStages * kStageBytes;
     const unsigned char* kv_unit = reinterpret_cast<const unsigned char*>(kv) + cu * gm.max_seq_len * 2 * D * 2;
 
-    if (lane == 0) {
-        for (int i = 0; i < kMmaStages; ++i) mbar_init(&full[warp][i], 1);
-        fence_mbar_init();
-    }
-    __syncwarp();
-
     bool any_bad = false;
-    // One bulk copy per row; rows past the end of the warp's range repeat its last row (their
-    // probabilities are masked to zero), so a stage always holds finite numbers.
-    auto issue = [&](int tile) {
-        const int st = tile % kMmaStages;
-        const int r0 = wb + tile * kTileTok;
-        if (lane == 0) mbar_arrive_expect_tx(&full[warp][st], kTileTok * 512);
-        __syncwarp();
-        if (lane < kTileTok) {
-            bool bad;
-            const int t = rm.token(min(r0 + lane, we - 1), bad);
-            bulk_copy_g2s(my_stage + st * kStageBytes + lane * kRowPitch, kv_unit + (size_t)t * 512, 512, &full[warp][st]);
+    // Gather of one tile: the whole warp copies each 512-byte K|V row with one 16-byte cp.async per
+    // lane (one warp instruction per row; the per-row TMA bulk copies this replaces queued up at the
+    // SM's single TMA port and took ~2 us to issue).  Rows past the end of the warp's range repeat
+    // its last row (their probabilities are masked to zero), so a stage always holds finite numbers.
+    // Every tile slot commits exactly one group, empty or not, so "all but the newest
+    // kMmaStages-1 groups are complete" always means "the tile about to be used has landed".
+    const uint32_t stage_u32 = smem_u32(my_stage);
+    auto issue_token = [&](int tile, int t) {     // t: lane i < 16 holds the token of row i
+        const uint32_t dst = stage_u32 + (tile % kMmaStages) * kStageBytes + lane * 16;
+        const unsigned char* src = kv_unit + lane * 16;
+#pragma unroll
+        for (int i = 0; i < kTileTok; ++i) {
+            const int ti = __shfl_sync(0xffffffffu, t, i);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * kRowPitch), "l"(src + (size_t)ti * 512) : "memory");
         }
     };
+    auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
+    auto issue = [&](int tile) {
+        bool bad;
+        const int t = lane < kTileTok ? rm.token(min(wb + tile * kTileTok + lane, we - 1), bad) : 0;
+        issue_token(tile, t);
+    };
     attn_stamp(1);
-    for (int t = 0; t < kMmaStages && t < n_tiles; ++t) issue(t);
+    {   // the first tiles' list entries are fetched together (one memory round trip), then their rows
+        int tok[kMmaStages];
+#pragma unroll
+        for (int t = 0; t < kMmaStages; ++t) {
+            bool bad;
+            tok[t] = (t < n_tiles && lane < kTileTok) ? rm.token(min(wb + t * kTileTok + lane, we - 1), bad) : 0;
+        }
+#pragma unroll
+        for (int t = 0; t < kMmaStages; ++t) {
+            if (t < n_tiles) issue_token(t, tok[t]);
+            commit();
+        }
+    }
     attn_stamp(2);
 
-    // Q as the A operand: rows = query heads (gid; rows 8..15 are padding), k = channels
-    uint32_t qa[8][2];
+    // Q^T as the B operand of S = K Q^T: k = channels, n = query heads (gid; heads >= g are zero padding)
+    uint32_t qb[8][2];
     {
         const __nv_bfloat16* qbase = reinterpret_cast<const __nv_bfloat16*>(a.q) + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * g) * D;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            qa[ks][0] = qa[ks][1] = 0u;
+            qb[ks][0] = qb[ks][1] = 0u;
             if (gid < g) {
-                qa[ks][0] = __ldg(reinterpret_cast<const uint32_t*>(qbase + gid * D + ks * 16 + tig * 2));
-                qa[ks][1] = __ldg(reinterpret_cast<const uint32_t*>(qbase + gid * D + ks * 16 + 8 + tig * 2));
+                qb[ks][0] = __ldg(reinterpret_cast<const uint32_t*>(qbase + gid * D + ks * 16 + tig * 2));
+                qb[ks][1] = __ldg(reinterpret_cast<const uint32_t*>(qbase + gid * D + ks * 16 + 8 + tig * 2));
             }
         }
     }
     const float qscale = a.sm_scale * kLog2e;
 
-    float o[16][4];
+    // O^T accumulators: 8 tiles of (16 channels x 8 heads); this thread: channels mt*16 + gid (+8),
+    // heads 2*tig and 2*tig+1 -- the same two heads as its columns of S.
+    float o[8][4];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;             // of head gid, over this thread's token columns
+    for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // heads 2*tig, 2*tig+1; l over this thread's tokens
 
-    const uint32_t stage_u32 = smem_u32(my_stage);
     // per-lane ldmatrix row addresses inside a stage
     const int mi = lane >> 3, r8 = lane & 7;
-    const uint32_t k_lane_off = ((mi >> 1) * 8 + r8) * kRowPitch + (mi & 1) * 16;          // + ks * 32
-    const uint32_t v_lane_off = ((mi & 1) * 8 + r8) * kRowPitch + 256 + (mi >> 1) * 16;    // + np * 32
+    const uint32_t k_lane_off = ((mi & 1) * 8 + r8) * kRowPitch + (mi >> 1) * 16;          // + ks * 32   (A of S = K Q^T)
+    const uint32_t v_lane_off = ((mi >> 1) * 8 + r8) * kRowPitch + 256 + (mi & 1) * 16;    // + mt * 32   (A of O^T = V^T P^T)
 
-    bool timed_out = false;
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int st = tile % kMmaStages;
         const int r0 = wb + tile * kTileTok;
@@ -416,99 +455,165 @@ __global__ void __launch_bounds__(kAttnThreads) attn_mma_kernel(Geom gm, UnitTab
             any_bad |= bad;
         }
         const unsigned vmask = __ballot_sync(0xffffffffu, ok);
-        if (!mbar_wait(&full[warp][st], (tile / kMmaStages) & 1)) timed_out = true;
+        asm volatile("cp.async.wait_group %0;" ::"n"(kMmaStages - 1) : "memory");
+        __syncwarp();                                  // every lane's copies of this tile are visible to the warp
         if (tile == 0) attn_stamp(3);
         const uint32_t sb = stage_u32 + st * kStageBytes;
 
-        float sc[2][4];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+        // S[token][head]: this thread holds tokens gid (c0,c1) and gid+8 (c2,c3), heads 2*tig, 2*tig+1
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4(sb + k_lane_off + ks * 32, b0, b1, b2, b3);
-            mma_bf16(sc[0], qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
-            mma_bf16(sc[1], qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(sb + k_lane_off + ks * 32, a0, a1, a2, a3);
+            mma_bf16(sc, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
         }
-        // this thread: head gid, tokens j*8 + tig*2 + {0,1}
+        const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
         float x[4];
-        float tmax = -INFINITY;
+        x[0] = v0 ? sc[0] * qscale : -INFINITY, x[1] = v0 ? sc[1] * qscale : -INFINITY;
+        x[2] = v1 ? sc[2] * qscale : -INFINITY, x[3] = v1 ? sc[3] * qscale : -INFINITY;
+        float tmax[2] = {fmaxf(x[0], x[2]), fmaxf(x[1], x[3])};
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int col = j * 8 + tig * 2 + e;
-                x[j * 2 + e] = (vmask >> col) & 1u ? sc[j][e] * qscale : -INFINITY;
-                tmax = fmaxf(tmax, x[j * 2 + e]);
-            }
-        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-        tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-        const float m_new = fmaxf(m_run, tmax);
-        const float ms = m_new == -INFINITY ? 0.f : m_new;
-        const float corr = exp2f(m_run - ms);
-        m_run = m_new;
-        float p[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) p[i] = exp2f(x[i] - ms);
-        l_run = l_run * corr + (p[0] + p[1] + p[2] + p[3]);
-        const bool rescale = __any_sync(0xffffffffu, corr != 1.f);
-        if (rescale) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) o[i][0] *= corr, o[i][1] *= corr;
+        for (int off = 4; off < 32; off <<= 1) {       // over the 8 token rows held by lanes with the same tig
+            tmax[0] = fmaxf(tmax[0], __shfl_xor_sync(0xffffffffu, tmax[0], off));
+            tmax[1] = fmaxf(tmax[1], __shfl_xor_sync(0xffffffffu, tmax[1], off));
         }
-        // P = P_hi + P_lo in bf16
+        float corr[2], ms[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const float m_new = fmaxf(m_run[e], tmax[e]);
+            ms[e] = m_new == -INFINITY ? 0.f : m_new;
+            corr[e] = exp2f(m_run[e] - ms[e]);
+            m_run[e] = m_new;
+        }
+        float p[4];
+        p[0] = exp2f(x[0] - ms[0]), p[1] = exp2f(x[1] - ms[1]), p[2] = exp2f(x[2] - ms[0]), p[3] = exp2f(x[3] - ms[1]);
+        l_run[0] = l_run[0] * corr[0] + p[0] + p[2];
+        l_run[1] = l_run[1] * corr[1] + p[1] + p[3];
+        if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i][0] *= corr[0], o[i][1] *= corr[1], o[i][2] *= corr[0], o[i][3] *= corr[1];
+        }
+        // P = P_hi + P_lo in bf16, transposed into the B operand (k = tokens, n = heads)
         float ph[4], pl[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             ph[i] = __bfloat162float(__float2bfloat16_rn(p[i]));
             pl[i] = p[i] - ph[i];
         }
-        const uint32_t pa_hi0 = pack_bf16(ph[0], ph[1]), pa_hi2 = pack_bf16(ph[2], ph[3]);
-        const uint32_t pa_lo0 = pack_bf16(pl[0], pl[1]), pa_lo2 = pack_bf16(pl[2], pl[3]);
+        const uint32_t bh0 = movmatrix_trans(pack_bf16(ph[0], ph[1])), bh1 = movmatrix_trans(pack_bf16(ph[2], ph[3]));
+        const uint32_t bl0 = movmatrix_trans(pack_bf16(pl[0], pl[1])), bl1 = movmatrix_trans(pack_bf16(pl[2], pl[3]));
 #pragma unroll
-        for (int np = 0; np < 8; ++np) {
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(sb + v_lane_off + np * 32, b0, b1, b2, b3);
-            mma_bf16(o[2 * np], pa_hi0, 0u, pa_hi2, 0u, b0, b1);
-            mma_bf16(o[2 * np], pa_lo0, 0u, pa_lo2, 0u, b0, b1);
-            mma_bf16(o[2 * np + 1], pa_hi0, 0u, pa_hi2, 0u, b2, b3);
-            mma_bf16(o[2 * np + 1], pa_lo0, 0u, pa_lo2, 0u, b2, b3);
+        for (int mt = 0; mt < 8; ++mt) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4_trans(sb + v_lane_off + mt * 32, a0, a1, a2, a3);
+            mma_bf16(o[mt], a0, a1, a2, a3, bh0, bh1);
+            mma_bf16(o[mt], a0, a1, a2, a3, bl0, bl1);
         }
-        __syncwarp();
-        if (tile + kMmaStages < n_tiles) {
-            fence_proxy_async();
-            issue(tile + kMmaStages);
-        }
+        __syncwarp();                                  // the warp is done reading this stage
+        if (tile + kMmaStages < n_tiles) issue(tile + kMmaStages);
+        commit();
     }
-    if ((any_bad || timed_out) && lane < kTileTok) atomicExch(status, timed_out ? kStatusTimeout : kStatusBadIndex);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (any_bad && lane < kTileTok) atomicExch(status, kStatusBadIndex);
 
     // ---- warp result -> shared (reusing the warp's own stages), block combine, publish ------------------
     attn_stamp(4);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
+    }
     __syncwarp();
     float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][128 channels]
 #pragma unroll
-    for (int nt = 0; nt < 16; ++nt) *reinterpret_cast<float2*>(&wo[gid * D + nt * 8 + tig * 2]) = make_float2(o[nt][0], o[nt][1]);
-    if (tig == 0) sh_m[warp][gid] = m_run, sh_l[warp][gid] = l_run;
+    for (int mt = 0; mt < 8; ++mt) {
+        wo[(2 * tig) * D + mt * 16 + gid] = o[mt][0];
+        wo[(2 * tig + 1) * D + mt * 16 + gid] = o[mt][1];
+        wo[(2 * tig) * D + mt * 16 + gid + 8] = o[mt][2];
+        wo[(2 * tig + 1) * D + mt * 16 + gid + 8] = o[mt][3];
+    }
+    if (gid == 0) {
+        sh_m[warp][2 * tig] = m_run[0], sh_l[warp][2 * tig] = l_run[0];
+        sh_m[warp][2 * tig + 1] = m_run[1], sh_l[warp][2 * tig + 1] = l_run[1];
+    }
     __syncthreads();
-    SplitSink sink{part_o, part_ml, counters, a.out, a.lse, (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g, lu, split, a.nsplit};
-    for (int u = 0; u < g; ++u) {
+    const size_t hq0 = (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g;
+    // weights 2^(m_w - M) of every (warp, head), computed once by NW*8 threads
+    __shared__ float sh_w[NW][kMaxGroup], sh_M[kMaxGroup];
+    if (tid < NW * kMaxGroup) {
+        const int w = tid / kMaxGroup, u = tid % kMaxGroup;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, sh_m[w][u]);
-        const float Ms = M == -INFINITY ? 0.f : M;
-        float lsum = 0.f, acc = 0.f;
+        for (int x = 0; x < NW; ++x) M = fmaxf(M, sh_m[x][u]);
+        sh_w[w][u] = exp2f(sh_m[w][u] - (M == -INFINITY ? 0.f : M));
+        if (w == 0) sh_M[u] = M;
+    }
+    __syncthreads();
+    float cM[kMaxGroup], cL[kMaxGroup], cO[kMaxGroup];        // block result per head; cO: channel tid (tid < 128)
 #pragma unroll
-        for (int w = 0; w < kAttnWarps; ++w) {
-            const float e = exp2f(sh_m[w][u] - Ms);
-            lsum += sh_l[w][u] * e;
-            acc += reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * D + tid] * e;
+    for (int u = 0; u < kMaxGroup; ++u) {
+        cM[u] = -INFINITY, cL[u] = 0.f, cO[u] = 0.f;
+        if (u < g && tid < D) {
+            float lsum = 0.f, acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const float e = sh_w[w][u];
+                lsum += sh_l[w][u] * e;
+                acc = fmaf(reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * D + tid], e, acc);
+            }
+            cM[u] = sh_M[u], cL[u] = lsum, cO[u] = acc;
         }
-        sink.publish(u, M, lsum, acc);
     }
     attn_stamp(5);
-    sink.merge_if_last(g, &sh_last);
+    if (a.cluster_merge) {
+        cg::cluster_group cluster = cg::this_cluster();
+        const int rank = (int)cluster.block_rank(), C = (int)cluster.num_blocks();
+        float* area = reinterpret_cast<float*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [C][g][kMergePitch]
+        float* area0 = cluster.map_shared_rank(area, 0);
+        if (tid < D) {
+#pragma unroll
+            for (int u = 0; u < kMaxGroup; ++u)
+                if (u < g) {
+                    float* slot = area0 + (size_t)(rank * g + u) * kMergePitch;
+                    slot[tid] = cO[u];
+                    if (tid == 0) slot[D] = cM[u], slot[D + 1] = cL[u];
+                }
+        }
+        cluster.sync();
+        if (rank == 0) {
+            __shared__ float cw[kAttnMaxCluster][kMaxGroup], cMx[kMaxGroup];
+            if (tid < C * kMaxGroup) {
+                const int r = tid / kMaxGroup, u = tid % kMaxGroup;
+                if (u < g) {
+                    float M = -INFINITY;
+                    for (int x = 0; x < C; ++x) M = fmaxf(M, area[(size_t)(x * g + u) * kMergePitch + D]);
+                    cw[r][u] = exp2f(area[(size_t)(r * g + u) * kMergePitch + D] - (M == -INFINITY ? 0.f : M));
+                    if (r == 0) cMx[u] = M;
+                }
+            }
+            __syncthreads();
+            if (tid < D) {
+                for (int u = 0; u < g; ++u) {
+                    float lsum = 0.f, acc = 0.f;
+                    for (int r = 0; r < C; ++r) {
+                        const float* slot = area + (size_t)(r * g + u) * kMergePitch;
+                        const float e = cw[r][u];
+                        lsum += slot[D + 1] * e;
+                        acc = fmaf(slot[tid], e, acc);
+                    }
+                    a.out[(hq0 + u) * D + tid] = acc / lsum;
+                    if (a.lse && tid == 0) a.lse[hq0 + u] = (cMx[u] + log2f(lsum)) * kLn2;
+                }
+            }
+        }
+    } else if constexpr (NW == kAttnWarps) {
+        SplitSink sink{part_o, part_ml, counters, a.out, a.lse, hq0, lu, split, a.nsplit};
+#pragma unroll
+        for (int u = 0; u < kMaxGroup; ++u)
+            if (u < g) sink.publish(u, cM[u], cL[u], cO[u]);
+        sink.merge_if_last(g, &sh_last);
+    }
     attn_stamp(6);
 }
 
@@ -532,7 +637,61 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         if (rows > L) rows = L;
         if (rows > max_rows) max_rows = rows;
     }
-    if (a.nsplit <= 0) a.nsplit = pick_nsplit(c, ut.layer_count * ut.n_seq * gm.Hkv, max_rows);
+    const int units = ut.layer_count * ut.n_seq * gm.Hkv;
+    a.cluster_merge = 0;
+    int nw = kAttnWarps;
+    if (gm.dtype == TB_BF16) {
+        static bool configured = false;
+        static int max_active[17];                    // co-resident clusters of the 8-warp kernel per cluster size (0 = not asked yet)
+        if (!configured) {
+            cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+            if (e != cudaSuccess) return e;
+            (void)cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            (void)cudaGetLastError();
+            configured = true;
+        }
+        auto clusters_that_fit = [&](int csize) {     // how many clusters of `csize` 8-warp blocks run at once
+            if (max_active[csize] == 0) {
+                cudaLaunchConfig_t q = {};
+                q.gridDim = dim3(csize, 1, 1), q.blockDim = dim3(256, 1, 1);
+                q.dynamicSmemBytes = 8 * 2 * kStageBytes + (size_t)csize * gm.g * 132 * sizeof(float);
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = csize, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
+                q.attrs = at, q.numAttrs = 1;
+                int n_clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&n_clusters, attn_mma_kernel<8, 2>, &q) != cudaSuccess) n_clusters = 0;
+                (void)cudaGetLastError();
+                max_active[csize] = n_clusters > 0 ? n_clusters : -1;
+            }
+            return max_active[csize];
+        };
+        // Few problems (one layer of a small batch): blocks of 8 warps, one per SM, and the largest
+        // cluster (up to 16 blocks, sizes above 8 are non-portable) that the device can keep resident
+        // for every problem at once; the splits merge inside the cluster.  Many problems: 4-warp
+        // blocks, two per SM, clusters of up to 8; splits beyond that go through the global workspace.
+        int n = 0;
+        const int by_rows = max_rows / (8 * kTileTok) < 1 ? 1 : max_rows / (8 * kTileTok);
+#ifdef TB_FORCE_ATTN_CLUSTER
+        n = TB_FORCE_ATTN_CLUSTER;
+#else
+        for (int cand = 16; cand >= 1 && !n; cand = cand > 8 ? cand - 2 : cand - 1)
+            if (cand <= by_rows && units * cand <= c->sm_count && (cand <= 8 || clusters_that_fit(cand) >= units)) n = cand;
+#endif
+        if (n && max_rows / n <= 1024) {
+            a.nsplit = n, nw = 8, a.cluster_merge = 1;
+        } else {
+            a.nsplit = pick_nsplit(c, units, max_rows);
+            if (a.nsplit <= 8 + 2) {
+                if (a.nsplit > 8) a.nsplit = 8;
+                a.cluster_merge = 1;
+            }
+        }
+    } else {
+        a.nsplit = pick_nsplit(c, units, max_rows);
+    }
     dim3 grid(a.nsplit, gm.Hkv, ut.layer_count * ut.n_seq);
 #define TB_ATTN(T, G)                                                                                                   \
     attn_kernel<T, G><<<grid, kAttnThreads, 0, s>>>(gm, ut, a, (const T*)c->kv, c->st.idx, c->st.cnt, c->wk.part_o,     \
@@ -545,15 +704,31 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         else TB_ATTN(T, 8);                           \
     } while (0)
     if (gm.dtype == TB_BF16) {
-        static bool configured = false;
-        const size_t smem = (size_t)kAttnWarps * kMmaStages * kStageBytes;
-        if (!configured) {
-            cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return e;
-            configured = true;
-        }
-        attn_mma_kernel<<<grid, kAttnThreads, smem, s>>>(gm, ut, a, (const __nv_bfloat16*)c->kv, c->st.idx, c->st.cnt,
-                                                         c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
+        const size_t merge_bytes = a.cluster_merge ? (size_t)a.nsplit * gm.g * 132 * sizeof(float) : 0;
+        // three stages per warp when the 8-warp block still fits the SM with them
+        const int nst = (nw == 8 && 8 * 3 * kStageBytes + merge_bytes <= 220 * 1024 && a.nsplit <= 8) ? 3 : 2;
+        const size_t smem = (size_t)nw * nst * kStageBytes + merge_bytes;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(nw * 32, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = a.cluster_merge ? a.nsplit : 1;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const __nv_bfloat16* kvp = (const __nv_bfloat16*)c->kv;
+        if (nw == 8 && nst == 3)
+            return cudaLaunchKernelEx(&cfg, attn_mma_kernel<8, 3>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
+                                      c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
+        if (nw == 8)
+            return cudaLaunchKernelEx(&cfg, attn_mma_kernel<8, 2>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
+                                      c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
+        return cudaLaunchKernelEx(&cfg, attn_mma_kernel<4, 2>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
+                                  c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
     } else {
         TB_ATTN_G(float);
     }
@@ -599,8 +774,7 @@ tb_status static_scratch_for_current_device(unsigned char** out, int* sm_count) 
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return TB_ERR_CUDA;
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TB_ERR_CUDA;
-        if (cudaFuncSetAttribute(tb::attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 tb::kAttnWarps * tb::kMmaStages * tb::kStageBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(tb::attn_mma_kernel<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) != cudaSuccess)
             return TB_ERR_CUDA;
         g_sm_count[dev] = sms;
         g_scratch_addr[dev] = static_cast<unsigned char*>(p);
@@ -660,6 +834,8 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     a.q = q_dev, a.idx = idx_dev, a.cnt = cnt_dev, a.out = out_dev, a.lse = lse_dev;
     a.dense = idx_dev ? 0 : 1, a.sinks = idx_dev ? sinks : 0, a.recent = idx_dev ? recent : 0;
     a.list_bound = idx_dev ? idx_stride : 0;
+    a.cluster_merge = 0;
+    for (int i = 0; i < n_seq; ++i) a.known_cnt[i] = -1;
     a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim);
     {   // same split rule as the context path
         int units = n_seq * n_kv_heads, target = 4 * sm_count;
@@ -675,7 +851,7 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     dim3 grid(a.nsplit, n_kv_heads, n_seq);
     // the stored-list arguments of the kernels are never read here (caller lists or dense)
     if (kv_dtype == TB_BF16) {
-        attn_mma_kernel<<<grid, kAttnThreads, kAttnWarps * kMmaStages * kStageBytes, s>>>(
+        attn_mma_kernel<4, 2><<<grid, kAttnThreads, kAttnWarps * 2 * kStageBytes, s>>>(
             gm, ut, a, (const __nv_bfloat16*)kv_dev, nullptr, nullptr, part_o, part_ml, counters, status);
     } else {
 #define TB_ATTN_S(G) attn_kernel<float, G><<<grid, kAttnThreads, 0, s>>>(gm, ut, a, (const float*)kv_dev, nullptr, nullptr, part_o, part_ml, counters, status)

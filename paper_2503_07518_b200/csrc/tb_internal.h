@@ -54,8 +54,13 @@ struct AttnArgs {
     float* out;             // [layer_count][n_seq][Hq][D]
     float* lse;             // optional
     int dense, sinks, recent, nsplit;
+    int cluster_merge;      // 1: the splits of a (sequence, KV head) are one cluster and merge through DSMEM
     int list_bound;         // host-known upper bound of the list length (sizes the split count)
     float sm_scale;
+    // Length of the stored list per (layer-local, sequence) when the host knows it exactly (selection
+    // without neighbour expansion: min(budget, candidates), equal for all KV heads), else -1: saves
+    // the kernels a dependent global load before they can split the rows.
+    int known_cnt[kMaxLaunchUnits];
 };
 
 struct DevState {
@@ -86,6 +91,7 @@ struct tb_ctx {
     size_t state_bytes, work_bytes;
     std::vector<int> len, len_proj;       // [n_layers * max_batch]
     std::vector<int> has_sel;             // [n_layers * max_batch]
+    std::vector<int> sel_cnt;             // [n_layers * max_batch] stored list length when the host knows it, else -1
     CUtensorMap kimp_map;                 // 2-D view of kimp: rows = all token slots, cols = d'
     int tile_rows;                        // rows per TMA box of the score pass
     int sm_count;
@@ -105,7 +111,6 @@ cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_im
 cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s);
 cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s);
-size_t select_smem_bytes(const tb_ctx* c, int chunk_tokens);
 
 // tb_attention.cu
 cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArgs& a, cudaStream_t s);

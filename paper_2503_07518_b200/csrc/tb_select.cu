@@ -26,9 +26,10 @@ namespace tb {
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kTileRows = 256;      // rows per TMA box = one row per thread
-constexpr int kStages = 3;
+constexpr int kMaxStages = 12;      // depth of the TMA ring is chosen per launch (bytes in flight vs. blocks per SM)
 constexpr int kBins = 2048;         // 11-bit digits (the last digit has 10 bits)
 constexpr int kMaxCluster = 8;
+constexpr int kMaxKeysPerBlock = 32768;   // 128 KB of on-chip keys per block at most
 constexpr int kListCap = 256;       // non-empty first-digit bins a block may publish on the fast path
 constexpr int kCandCap = 4096;      // keys of the threshold bin gathered at rank 0 (aliases merged[1..2])
 
@@ -52,7 +53,7 @@ __device__ __forceinline__ void phase_stamp(int) {}
 
 struct __align__(16) SelSmem {
     int res[8];                         // rank 0's verdict: prefix, low_bits, krem, gt_base, eq_base (16-byte stores)
-    uint64_t full[kStages];
+    uint64_t full[kMaxStages];
     int warp_a[kSelWarps];
     int warp_b[kSelWarps];
     int tot[kMaxCluster][2];
@@ -132,19 +133,24 @@ __device__ __forceinline__ void find_digit(const int* hist, int k, SelSmem* sm, 
 
 template <typename T, int DP>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_constant__ CUtensorMap tmap, Geom gm, UnitTable ut,
-                                                             SelectArgs a, int tiles_per_cta, int32_t* __restrict__ state_idx,
-                                                             int32_t* __restrict__ state_cnt, int32_t* __restrict__ status) {
+                                                             SelectArgs a, int tiles_per_cta, int n_stages,
+                                                             int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt,
+                                                             int32_t* __restrict__ status) {
     constexpr int RB = DP * Elem<T>::kBytes;          // bytes per projected-key row: 32, 64 or 128
     constexpr int NCH = RB / 16;
     constexpr uint32_t kTileBytes = kTileRows * RB;
 
     extern __shared__ unsigned char smem_raw[];
     // swizzled TMA boxes need their shared-memory base on the swizzle period (up to 1024 bytes)
-    unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // kStages * kTileBytes
-    int* hist = reinterpret_cast<int*>(stage_base + kStages * kTileBytes);        // local histogram
-    int* merged = hist + kBins;                                                   // 3 cluster-merged histograms
-    SelSmem* sm = reinterpret_cast<SelSmem*>(merged + 3 * kBins);
+    unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // n_stages * kTileBytes
+    int* hist = reinterpret_cast<int*>(stage_base + n_stages * kTileBytes);       // local histogram
+    int* merged = hist + kBins;                                                   // cluster-merged first-digit histogram
+    SelSmem* sm = reinterpret_cast<SelSmem*>(merged + kBins);
     uint32_t* keys = reinterpret_cast<uint32_t*>(sm + 1);                         // tiles_per_cta * kTileRows
+    // The ring is idle once the block has streamed its rows; its first 16 KB then serve as the merged
+    // histograms of digits 2 and 3 (general path) or as rank 0's candidate buffer (fast path).  Peers
+    // write there only after a cluster barrier that every block reaches after its streaming loop.
+    int* merged_late = reinterpret_cast<int*>(stage_base);                        // 2 * kBins ints
 
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
@@ -178,10 +184,10 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
 
     // ---- set-up -------------------------------------------------------------------------------
     phase_stamp(0);
-    for (int i = tid; i < 4 * kBins; i += kSelThreads) hist[i] = 0;               // local + 3 merged
+    for (int i = tid; i < 2 * kBins; i += kSelThreads) hist[i] = 0;               // local + merged first digit
     if (tid == 0) {
         prefetch_tmap(&tmap);
-        for (int i = 0; i < kStages; ++i) mbar_init(&sm->full[i], 1);
+        for (int i = 0; i < n_stages; ++i) mbar_init(&sm->full[i], 1);
         fence_mbar_init();
     }
     __syncthreads();
@@ -201,7 +207,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     load_group_query<DP>(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
 
     if (tid == 0) {
-        for (int i = 0; i < kStages && i < my_tiles; ++i) {
+        for (int i = 0; i < n_stages && i < my_tiles; ++i) {
             mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
             tma_load_2d(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kTileRows), &sm->full[i]);
         }
@@ -209,9 +215,10 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
 
     // ---- stream + score + first digit histogram -------------------------------------------------
     bool timed_out = false;
+    int st = 0;
+    uint32_t phase = 0;
     for (int i = 0; i < my_tiles; ++i) {
-        const int st = i % kStages;
-        if (!mbar_wait(&sm->full[st], (i / kStages) & 1)) timed_out = true;   // keep going: control flow stays uniform
+        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;   // keep going: control flow stays uniform
         const unsigned char* tile = stage_base + st * kTileBytes;
         const int slot = i * kTileRows + tid;
         if (slot < n_local) {
@@ -226,14 +233,18 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             smem_add(&hist[key >> 21], 1);
         }
         __syncthreads();                               // all reads of this stage are done
-        if (tid == 0 && i + kStages < my_tiles) {
+        if (tid == 0 && i + n_stages < my_tiles) {
             fence_proxy_async();
             mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
-            tma_load_2d(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + kStages) * kTileRows),
+            tma_load_2d(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kTileRows),
                         &sm->full[st]);
         }
+        if (++st == n_stages) st = 0, phase ^= 1u;
     }
     if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    // the ring is idle now: clear the part that later serves as merged histograms (see merged_late)
+    for (int i = tid; i < 2 * kBins; i += kSelThreads) merged_late[i] = 0;
+    __syncthreads();
     phase_stamp(2);
 
     uint32_t prefix = 0;          // digits fixed so far (value of key >> low_bits)
@@ -316,7 +327,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
                 int tot_mine;
                 int pos = block_excl_scan(mine, sm->warp_b, tot_mine);
                 for (int r = 0; r < rank; ++r) pos += sm->inbin[r];
-                uint32_t* cand_local = reinterpret_cast<uint32_t*>(merged + kBins);
+                uint32_t* cand_local = reinterpret_cast<uint32_t*>(merged_late);
                 uint32_t* cand0 = cluster.map_shared_rank(cand_local, 0);
                 if (mine) {
                     for (int v = tid; v < n_vec; v += kSelThreads) {
@@ -404,15 +415,16 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         }
         const int* src = hist;
         if (C > 1) {
+            int* mrg = pass == 0 ? merged : merged_late + (pass - 1) * kBins;
             if (!exact) {
                 for (int b = tid; b < nbins; b += kSelThreads) {
                     int v = hist[b];
                     if (v)
-                        for (int r = 0; r < C; ++r) atomicAdd(cluster.map_shared_rank(&merged[pass * kBins + b], r), v);
+                        for (int r = 0; r < C; ++r) atomicAdd(cluster.map_shared_rank(&mrg[b], r), v);
                 }
             }
             cluster.sync();
-            src = merged + pass * kBins;
+            src = mrg;
         }
         if (!exact) {
             int bin, kr, bc;
@@ -430,14 +442,30 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     // ---- ordered compaction ------------------------------------------------------------------------
     // A slot is taken if its key is above the class, or inside the class and among the class's first
     // `krem` members in position order (the lower-position tie rule).  Warp w owns a contiguous range.
-    const int seg = ((n_local + kSelThreads - 1) / kSelThreads) * 32;   // slots per warp, multiple of 32
+    // Within a group of 128 slots lane l holds slots 4l..4l+3 (one 16-byte load), so lane order is
+    // position order.
+    const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
+    const int seg = ((n_local + kSelWarps * 128 - 1) / (kSelWarps * 128)) * 128;   // slots per warp, multiple of 128
     const int seg_begin = min(n_local, warp * seg), seg_end = min(n_local, (warp + 1) * seg);
+    auto classify = [&](int base, int& gt_bits, int& eq_bits) {   // bit e set: slot base+e is above / in the class
+        gt_bits = eq_bits = 0;
+        if (base < seg_end) {
+            const uint4 x = keys4[base >> 2];
+            const uint32_t v[4] = {x.x >> low_bits, x.y >> low_bits, x.z >> low_bits, x.w >> low_bits};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool in = base + e < seg_end;
+                gt_bits |= (in && v[e] > prefix) << e;
+                eq_bits |= (in && v[e] == prefix) << e;
+            }
+        }
+    };
     int n_gt = 0, n_eq = 0;
-#pragma unroll 4
-    for (int i = seg_begin + lane; i < seg_end; i += 32) {
-        const uint32_t kk = keys[i] >> low_bits;
-        n_gt += kk > prefix;
-        n_eq += kk == prefix;
+#pragma unroll 2
+    for (int i0 = seg_begin; i0 < seg_end; i0 += 128) {
+        int gb, eb;
+        classify(i0 + 4 * lane, gb, eb);
+        n_gt += __popc(gb), n_eq += __popc(eb);
     }
     n_gt = warp_sum_int(n_gt);
     n_eq = warp_sum_int(n_eq);
@@ -462,33 +490,55 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     }
     phase_stamp(6);
     int out_pos = gt_before + min(eq_before, krem);
+#pragma unroll 2
     for (int i0 = seg_begin; i0 < seg_end; i0 += 128) {
-        uint32_t kk[4];
-        bool in[4];
+        const int base = i0 + 4 * lane;
+        int gb, eb;
+        classify(base, gb, eb);
+        int take = gb;
+        if (__any_sync(0xffffffffu, eb != 0)) {        // class members here: hand out what is left of the quota in order
+            const int ne = __popc(eb);
+            int before = eq_before + warp_incl_scan(ne, lane) - ne;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {                  // four independent loads before the ballots
-            const int i = i0 + u * 32 + lane;
-            in[u] = i < seg_end;
-            kk[u] = in[u] ? keys[i] >> low_bits : 0u;
+            for (int e = 0; e < 4; ++e)
+                if ((eb >> e) & 1) {
+                    if (before < krem) take |= 1 << e;
+                    ++before;
+                }
+            eq_before += warp_sum_int(ne);
         }
+        const int nt = __popc(take);
+        if (__any_sync(0xffffffffu, nt != 0)) {
+            const int incl = warp_incl_scan(nt, lane);
+            int o = out_pos + incl - nt;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const bool is_gt = in[u] && kk[u] > prefix, is_eq = in[u] && kk[u] == prefix;
-            const unsigned eq_ballot = __ballot_sync(0xffffffffu, is_eq);
-            const bool take = is_gt || (is_eq && eq_before + __popc(eq_ballot & lt_mask) < krem);
-            const unsigned take_ballot = __ballot_sync(0xffffffffu, take);
-            if (take) idx_dst[out_pos + __popc(take_ballot & lt_mask)] = tok0 + i0 + u * 32 + lane;
-            out_pos += __popc(take_ballot);
-            eq_before += __popc(eq_ballot);
+            for (int e = 0; e < 4; ++e)
+                if ((take >> e) & 1) idx_dst[o++] = tok0 + base + e;
+            out_pos += __shfl_sync(0xffffffffu, incl, 31);
         }
     }
     if (rank == 0 && tid == 0) *cnt_dst = k;
     phase_stamp(7);
 }
 
-size_t select_smem_bytes(const tb_ctx* c, int tiles_per_cta) {
-    int rb = c->geom.dp * (c->geom.dtype == TB_BF16 ? 2 : 4);
-    return 1024 + (size_t)kStages * kTileRows * rb + 4 * kBins * sizeof(int) + sizeof(SelSmem) + (size_t)tiles_per_cta * kTileRows * 4;
+// Shared memory of one block without its TMA ring: alignment slack, two histograms, control block, keys.
+static size_t select_fixed_smem(int tiles_per_cta) {
+    return 1024 + 2 * kBins * sizeof(int) + sizeof(SelSmem) + (size_t)tiles_per_cta * kTileRows * 4;
+}
+
+// Ring depth: the score pass is bound by bytes in flight (bandwidth x loaded latency is about 90 KB
+// per SM), so take as many stages as fit while keeping two blocks per SM when the keys leave room
+// for that, one block per SM otherwise.  At least 16 KB of ring (reused after streaming).
+static int select_stage_count(int tiles_per_cta, int tile_bytes) {
+    const size_t fixed = select_fixed_smem(tiles_per_cta);
+    const size_t two_per_sm = 113 * 1024, one_per_sm = 226 * 1024;
+    const int min_stages = tile_bytes >= 16384 ? 2 : 16384 / tile_bytes + 1;
+    int n = fixed + (size_t)3 * tile_bytes <= two_per_sm ? (int)((two_per_sm - fixed) / tile_bytes)
+                                                          : (int)((one_per_sm - fixed) / tile_bytes);
+    if (n > kMaxStages) n = kMaxStages;
+    if (n > tiles_per_cta && tiles_per_cta >= min_stages) n = tiles_per_cta;
+    if (n < min_stages) n = min_stages;
+    return n;
 }
 
 cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
@@ -503,12 +553,31 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     // Cluster size: enough blocks to cover the GPU about twice, at least 4 tiles per block, and a
     // key array per block of at most 32 KB where the cluster limit allows (64 KB otherwise).
     int C = 1;
-    while (C < kMaxCluster && (n_units * C < 2 * c->sm_count && n_tiles / (2 * C) >= 4)) C *= 2;
-    while (C < kMaxCluster && (n_tiles + C - 1) / C * kTileRows > 8192) C *= 2;
+    if (2 * n_units > c->sm_count) {
+        // several waves of blocks: keep the key array small enough for two blocks per SM, so one
+        // block's selection phase overlaps the other's streaming
+        while (C < kMaxCluster && (n_tiles + C - 1) / C * kTileRows > 8192) C *= 2;
+    } else {
+        // few problems: one wave.  Two blocks per SM when their key arrays leave room for two rings
+        // (more bytes in flight), otherwise one block per SM.
+        const int tile_b = kTileRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
+        C = 2 * c->sm_count / n_units;
+        if (C > kMaxCluster) C = kMaxCluster;
+        while (C > 1 && n_tiles / C < 4) --C;
+        const int tpc = (n_tiles + C - 1) / C;
+        if (1024 + 2 * kBins * 4 + sizeof(SelSmem) + (size_t)tpc * kTileRows * 4 + 3 * (size_t)tile_b > 113 * 1024) {
+            C = c->sm_count / n_units;
+            if (C > kMaxCluster) C = kMaxCluster;
+            while (C > 1 && n_tiles / C < 4) --C;
+        }
+    }
+    while (C < kMaxCluster && (n_tiles + C - 1) / C * kTileRows > kMaxKeysPerBlock) ++C;
     int tiles_per_cta = (n_tiles + C - 1) / C;
     if (tiles_per_cta < 1) tiles_per_cta = 1;
-    if (tiles_per_cta * kTileRows > 16384) return cudaErrorInvalidConfiguration;
-    size_t smem = select_smem_bytes(c, tiles_per_cta);
+    if (tiles_per_cta * kTileRows > kMaxKeysPerBlock) return cudaErrorInvalidConfiguration;
+    const int tile_bytes = kTileRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
+    const int n_stages = select_stage_count(tiles_per_cta, tile_bytes);
+    size_t smem = select_fixed_smem(tiles_per_cta) + (size_t)n_stages * tile_bytes;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(C, n_units, 1);
@@ -528,11 +597,11 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
         static bool configured = false;                                                                            \
         if (!configured) {                                                                                         \
             cudaError_t e = cudaFuncSetAttribute(select_kernel<T, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                                 200 * 1024);                                                      \
+                                                 227 * 1024);                                                      \
             if (e != cudaSuccess) return e;                                                                        \
             configured = true;                                                                                     \
         }                                                                                                          \
-        return cudaLaunchKernelEx(&cfg, select_kernel<T, DP>, c->kimp_map, gm, ut, a, tiles_per_cta, c->st.idx,    \
+        return cudaLaunchKernelEx(&cfg, select_kernel<T, DP>, c->kimp_map, gm, ut, a, tiles_per_cta, n_stages, c->st.idx, \
                                   c->st.cnt, c->st.status);                                                        \
     } while (0)
     if (gm.dtype == TB_BF16) {

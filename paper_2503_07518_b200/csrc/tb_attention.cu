@@ -649,6 +649,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
             if (e != cudaSuccess) return e;
             (void)cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            (void)cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             (void)cudaGetLastError();
             configured = true;
         }
@@ -656,13 +657,17 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             if (max_active[csize] == 0) {
                 cudaLaunchConfig_t q = {};
                 q.gridDim = dim3(csize, 1, 1), q.blockDim = dim3(256, 1, 1);
-                q.dynamicSmemBytes = 8 * 2 * kStageBytes + (size_t)csize * gm.g * 132 * sizeof(float);
+                const size_t mb = (size_t)csize * gm.g * 132 * sizeof(float);
+                const bool three = csize <= 8 && 8 * 3 * kStageBytes + mb <= 220 * 1024;
+                q.dynamicSmemBytes = 8 * (three ? 3 : 2) * kStageBytes + mb;
                 cudaLaunchAttribute at[1];
                 at[0].id = cudaLaunchAttributeClusterDimension;
                 at[0].val.clusterDim.x = csize, at[0].val.clusterDim.y = 1, at[0].val.clusterDim.z = 1;
                 q.attrs = at, q.numAttrs = 1;
                 int n_clusters = 0;
-                if (cudaOccupancyMaxActiveClusters(&n_clusters, attn_mma_kernel<8, 2>, &q) != cudaSuccess) n_clusters = 0;
+                cudaError_t qe = three ? cudaOccupancyMaxActiveClusters(&n_clusters, attn_mma_kernel<8, 3>, &q)
+                                       : cudaOccupancyMaxActiveClusters(&n_clusters, attn_mma_kernel<8, 2>, &q);
+                if (qe != cudaSuccess) n_clusters = 0;
                 (void)cudaGetLastError();
                 max_active[csize] = n_clusters > 0 ? n_clusters : -1;
             }

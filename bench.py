@@ -318,6 +318,161 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_trajectory(args, w):
+    """Workloads that decode: every step appends one token per sequence and layer, keys are projected
+    in deferred batches of `recent` tokens, the selection (with neighbour expansion) is refreshed every
+    `interval` steps and reused in between, attention runs every step.  Lengths change each step, so
+    the launches are issued directly (kernel parameters carry the lengths); a step's GPU time is
+    milliseconds, far above the launch cost."""
+    import torch
+    import torch.distributed as dist
+    from paper_2503_07518_b200 import binding as tbh
+    from paper_2503_07518_b200 import build
+    build.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    P, Wn = w.interval, w.recent
+    steps = max(P, args.steps // P * P)                      # whole refresh periods
+    warm = max(P, (args.warmup + P - 1) // P * P)
+    total = warm + 2 * steps                                  # device-timed pass + end-to-end pass
+    ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + total + Wn,
+                      w.budget, w.radius, device=local)
+    fill_caches(ctx, w, torch, tbh)
+    dt = tbh.torch_dtype(w.dtype)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(wl.seed_for(w.cfg_id, 0, 0, wl.TAG_Q))
+    shape_q = (w.n_layers, w.batch, w.n_q_heads)
+    q = torch.randn(*shape_q, w.head_dim, generator=gen, device="cuda").to(dt)
+    qi = torch.randn(*shape_q, w.imp_dim, generator=gen, device="cuda")
+    k_new = torch.randn(w.n_layers, w.batch, w.n_kv_heads, w.head_dim, generator=gen, device="cuda").to(dt)
+    v_new = torch.randn(w.n_layers, w.batch, w.n_kv_heads, w.head_dim, generator=gen, device="cuda").to(dt)
+    out = torch.empty(*shape_q, w.head_dim, device="cuda")
+    host = [t.cpu().pin_memory() for t in (q, qi, k_new, v_new)]
+    out_host = torch.empty_like(out, device="cpu").pin_memory()
+    groups = [(l, min(GROUP_LAYERS, w.n_layers - l)) for l in range(0, w.n_layers, GROUP_LAYERS)]
+    proj = list(w.lengths)                                    # projected length per sequence (same in every layer)
+    ones = [1] * w.batch
+    bytes_sel, bytes_att = [0.0], [0.0]
+
+    def step(t):
+        p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode, P, t)
+        refresh = t % P == 0
+        for (l0, n) in groups:
+            for l in range(l0, l0 + n):
+                ctx.append_kv(l, 1, None, ones, k_new[l], v_new[l])
+                if refresh and t > 0:                         # the window wrapped: project its tokens in one batch
+                    ctx.project_keys(l, 1, None, proj, [x + Wn for x in proj])
+            ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p)   # launches only on refresh steps
+            if refresh:
+                bytes_sel[0] += ctx.last_step_bytes()
+            for l in range(l0, l0 + n):
+                ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l])
+                bytes_att[0] += ctx.last_step_bytes()
+        if refresh and t > 0:
+            for b in range(w.batch):
+                proj[b] += Wn
+
+    stream = torch.cuda.Stream()
+    sampler = ClockSampler(local)
+    with torch.cuda.stream(stream):
+        t = 0
+        for _ in range(warm):
+            step(t)
+            t += 1
+        torch.cuda.synchronize()
+        assert ctx.get_status(stream) == 0, "device status set during warm-up"
+        if world > 1:
+            dist.barrier()
+        bytes_sel[0] = bytes_att[0] = 0.0
+        n0 = ctx.launch_count()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        sampler.start()
+        ev[0].record(stream)
+        for i in range(steps):
+            step(t)
+            t += 1
+            ev[i + 1].record(stream)
+        while not ev[-1].query():
+            time.sleep(0.002)
+        torch.cuda.synchronize()
+        sampler.sample()
+        sampler.stop_flag = True
+        launches = ctx.launch_count() - n0
+        per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        ms_step = ev[0].elapsed_time(ev[-1]) / steps
+        if world > 1:
+            tt = torch.tensor([ms_step], device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms_step = float(tt.item())
+        refresh_ms = float(np.mean(per_step[0::P]))
+        reuse_ms = float(np.mean([x for i, x in enumerate(per_step) if i % P]))
+        step_bytes = (bytes_sel[0] + bytes_att[0]) / steps
+        att_bytes = bytes_att[0] / steps / w.n_layers
+        sel_bytes = bytes_sel[0] / max(1, steps // P) / len(groups)
+        # end to end: the step's new K/V rows and queries come from pinned host memory, outputs go back
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            for dst, src in zip((q, qi, k_new, v_new), host):
+                dst.copy_(src, non_blocking=True)
+            step(t)
+            t += 1
+            out_host.copy_(out, non_blocking=True)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms_e2e = e0.elapsed_time(e1) / steps
+        # the two main kernels alone (same state, no appends): attention of every layer, refresh of every group
+        pr = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode, P, 0)
+
+        def alone(fn, reps):
+            fn()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(reps):
+                fn()
+            a1.record(stream)
+            torch.cuda.synchronize()
+            return a0.elapsed_time(a1) / reps
+
+        att_ms = alone(lambda: [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], pr, out[l]) for l in range(w.n_layers)], 5) / w.n_layers
+        sel_ms = alone(lambda: [ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], pr) for (l0, n) in groups], 3) / len(groups)
+        assert ctx.get_status(stream) == 0, "device status set during the timed region"
+
+    peak, peak_kind = measured_peaks()
+    tokens = w.batch * world
+    line = {
+        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+        "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "context": w.lengths[0], "budget": w.budget,
+                   "recent": w.recent, "radius": w.radius, "neighbor_mode": "dilate" if w.nmode == 0 else "cluster",
+                   "interval": P, "schedule": "per layer: append, (deferred projection), attention; select+expand per 4 layers on "
+                   "refresh steps; direct launches", "l2": "inputs larger than L2: %.0f MB touched per step" % (step_bytes / 1e6)},
+        "refresh_step_us": refresh_ms * 1e3, "reuse_step_us": reuse_ms * 1e3,
+        "step_hbm_gbs": step_bytes / (ms_step * 1e-3) / 1e9, "step_bytes": step_bytes,
+        "step_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak, "gpu_launches": int(launches),
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
+                "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host), "d2h_bytes_per_step": out_host.numel() * 4},
+        "kernels": {"select_kernel+neighbor_kernel": {"us_per_launch": sel_ms * 1e3, "bytes_per_launch": sel_bytes,
+                                                      "gbs": sel_bytes / (sel_ms * 1e-3) / 1e9, "launches_per_refresh": len(groups)},
+                    "attn_kernel": {"us_per_launch": att_ms * 1e3, "bytes_per_launch": att_bytes,
+                                    "gbs": att_bytes / (att_ms * 1e-3) / 1e9, "launches_per_step": w.n_layers}},
+        "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": att_bytes / (att_ms * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": att_bytes / (att_ms * 1e-3) / 1e9 / peak, "peak_kind": "of " + peak_kind,
+                     "traffic": None, "bytes_per_launch": att_bytes, "us_per_launch": att_ms * 1e3},
+        "clocks": sampler.summary(),
+    }
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -338,7 +493,12 @@ def main():
     else:
         if args.warmup < 3:
             args.warmup = 3
-        run_ours(args, w)
+        if w.decode_steps > 1:
+            if args.steps > w.decode_steps:
+                args.steps = w.decode_steps
+            run_trajectory(args, w)
+        else:
+            run_ours(args, w)
 
 
 if __name__ == "__main__":

@@ -104,6 +104,27 @@ def run_reference(args, w):
 
 
 # --------------------------------------------------------------------------------------------------
+# multi-GPU: the path shards by (sequence, layer, KV head) with no exchange step, so N GPUs run N
+# replicas of the workload (weak scaling); the only communication is the barrier and the max-over-ranks
+# of the device-measured time.
+
+def max_over_ranks(ms: float, device="cpu") -> float:
+    """The slowest rank's time (every rank gets it).  No-op without an initialised process group."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(batch_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Tokens all ranks decode per second: every rank advances `batch_per_rank` sequences per step."""
+    return batch_per_rank * world / (ms_per_step * 1e-3)
+
+
+# --------------------------------------------------------------------------------------------------
 # device leg
 
 class ClockSampler(threading.Thread):
@@ -258,12 +279,7 @@ def run_ours(args, w):
                 sampler.stop_flag = True
             if world > 1:
                 dist.barrier()
-            ms = e0.elapsed_time(e1)
-            if world > 1:
-                t = torch.tensor([ms], device="cuda")
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ms = float(t.item())
-            return ms / steps
+            return max_over_ranks(e0.elapsed_time(e1), "cuda") / steps
 
         sampler = ClockSampler(local)
         ms_step = timed(g_step.replay, args.steps, args.warmup, sampler)
@@ -286,7 +302,7 @@ def run_ours(args, w):
     dom = ("select_kernel", sel_b, ms_sel) if ms_sel * len(groups) >= ms_att * w.n_layers else ("attn_kernel", att_b, ms_att)
     achieved = dom[1] / (dom[2] * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "q_heads": w.n_q_heads,
@@ -407,11 +423,7 @@ def run_trajectory(args, w):
         sampler.stop_flag = True
         launches = ctx.launch_count() - n0
         per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
-        ms_step = ev[0].elapsed_time(ev[-1]) / steps
-        if world > 1:
-            tt = torch.tensor([ms_step], device="cuda")
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms_step = float(tt.item())
+        ms_step = max_over_ranks(ev[0].elapsed_time(ev[-1]), "cuda") / steps
         refresh_ms = float(np.mean(per_step[0::P]))
         reuse_ms = float(np.mean([x for i, x in enumerate(per_step) if i % P]))
         step_bytes = (bytes_sel[0] + bytes_att[0]) / steps
@@ -449,7 +461,7 @@ def run_trajectory(args, w):
     peak, peak_kind = measured_peaks()
     tokens = w.batch * world
     line = {
-        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
+        "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
         "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "context": w.lengths[0], "budget": w.budget,

@@ -171,6 +171,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     const size_t n = (size_t)cfg->n_layers * cfg->max_batch;
     c->len.assign(n, 0), c->len_proj.assign(n, 0), c->has_sel.assign(n, 0), c->sel_cnt.assign(n, -1);
     c->last_bytes = 0, c->launches = 0;
+    c->last_cache_write = c->last_list_write = -4;
     c->tile_rows = 256;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete c; return TB_ERR_CUDA; }
     // only the small control parts need defined contents; the index lists and partials are always
@@ -199,6 +200,7 @@ tb_status tb_set_projection(tb_ctx* c, int32_t layer, const void* W_dev, void* s
     const size_t bytes = (size_t)c->cfg.n_kv_heads * c->cfg.head_dim * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);
     if (cudaMemcpyAsync((char*)c->st.W + layer * bytes, W_dev, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream) != cudaSuccess)
         return TB_ERR_CUDA;
+    c->last_cache_write = (long long)c->launches;   // treat as written by the next launch's predecessor
     return TB_OK;
 }
 
@@ -245,6 +247,7 @@ tb_status tb_append_kv(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_ids
         if (launch_append(c, ut, n_new, tok_off, total, (const char*)k + (size_t)(l0 - lb) * layer_stride,
                           (const char*)v + (size_t)(l0 - lb) * layer_stride, (cudaStream_t)stream) != cudaSuccess)
             return TB_ERR_CUDA;
+        c->last_cache_write = (long long)c->launches;
         c->launches++;
     }
     for (int l = lb; l < lb + lc; ++l)
@@ -272,6 +275,7 @@ tb_status tb_project_keys(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_
         UnitTable ut;
         fill_table(c, &ut, l0, n, seqs, n_seq);
         if (launch_project(c, ut, pos_begin, pos_end, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+        c->last_cache_write = (long long)c->launches;
         c->launches++;
     }
     for (int l = lb; l < lb + lc; ++l)
@@ -343,12 +347,14 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                 a.idx_dst = c->wk.sel_idx, a.cnt_dst = c->wk.sel_cnt, a.dst_is_state = 0, a.idx_stride = c->wk.sel_stride;
             }
             if (launch_select(c, ut, a, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+            c->last_list_write = (long long)c->launches;
             c->launches++;
             if (p->radius > 0) {
                 NeighborArgs na;
                 na.idx_src = c->wk.sel_idx, na.cnt_src = c->wk.sel_cnt, na.src_stride = c->wk.sel_stride;
                 na.radius = p->radius, na.nmode = p->nmode, na.sinks = p->sinks, na.recent = p->recent;
                 if (launch_neighbors(c, ut, na, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+                c->last_list_write = (long long)c->launches;
                 c->launches++;
             }
         }
@@ -425,6 +431,7 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
                 a.known_cnt[l * n_seq + i] = (dense || idx) ? -1 : c->sel_cnt[(size_t)(l0 + l) * mb + seqs[i]];
         a.nsplit = 0;
         a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)c->cfg.head_dim);
+        a.early_ok = !idx && (long long)c->launches - c->last_cache_write >= 2 && (long long)c->launches - c->last_list_write >= 2;
         if (launch_attention(c, ut, a, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
         c->launches++;
     }

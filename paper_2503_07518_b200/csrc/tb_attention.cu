@@ -342,6 +342,10 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     __shared__ int sh_last;
 
     attn_stamp(0);
+    // Dependency wait (see pdl_wait): up front when the lists or cache rows may come from the
+    // predecessor; otherwise only before the queries are read, so that the row map, the list fetch
+    // and the first gathers overlap the predecessor's tail.
+    if (!a.early_ok) pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gid = lane >> 2, tig = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y;
@@ -416,6 +420,8 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     }
     attn_stamp(2);
 
+    if (a.early_ok) pdl_wait();                        // the queries are this call's input
+    pdl_launch_dependents();
     // Q^T as the B operand of S = K Q^T: k = channels, n = query heads (gid; heads >= g are zero padding)
     uint32_t qb[8][2];
     {
@@ -718,13 +724,15 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         cfg.blockDim = dim3(nw * 32, 1, 1);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = s;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = a.cluster_merge ? a.nsplit : 1;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see pdl_wait()
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         const __nv_bfloat16* kvp = (const __nv_bfloat16*)c->kv;
         if (nw == 8 && nst == 3)
             return cudaLaunchKernelEx(&cfg, attn_mma_kernel<8, 3>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
@@ -840,6 +848,7 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     a.dense = idx_dev ? 0 : 1, a.sinks = idx_dev ? sinks : 0, a.recent = idx_dev ? recent : 0;
     a.list_bound = idx_dev ? idx_stride : 0;
     a.cluster_merge = 0;
+    a.early_ok = 0;
     for (int i = 0; i < n_seq; ++i) a.known_cnt[i] = -1;
     a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim);
     {   // same split rule as the context path

@@ -74,6 +74,15 @@ __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may start while its predecessor in the stream still runs.  pdl_wait() blocks until the
+// predecessor has completed and its writes are visible (a no-op for ordinary launches);
+// pdl_launch_dependents() lets the successor begin.  Every kernel here waits before it touches
+// anything its predecessor may have produced and before its own global writes, and only then
+// releases its successor, so completion stays transitive along the stream.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- storage types ---------------------------------------------------------------------------
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -54,6 +54,7 @@ struct AttnArgs {
     float* out;             // [layer_count][n_seq][Hq][D]
     float* lse;             // optional
     int dense, sinks, recent, nsplit;
+    int early_ok;           // 1: lists and cache rows were written at least two launches ago
     int cluster_merge;      // 1: the splits of a (sequence, KV head) are one cluster and merge through DSMEM
     int list_bound;         // host-known upper bound of the list length (sizes the split count)
     float sm_scale;
@@ -96,6 +97,9 @@ struct tb_ctx {
     int tile_rows;                        // rows per TMA box of the score pass
     int sm_count;
     uint64_t last_bytes, launches;
+    // index (value of `launches` at launch time) of the last kernel that wrote the caches / the stored
+    // lists; a kernel may read them before its dependency wait only if that writer is not its predecessor
+    long long last_cache_write, last_list_write;
 };
 
 namespace tb {

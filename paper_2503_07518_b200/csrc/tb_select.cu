@@ -203,15 +203,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     const int n_local = max(0, min(my_tiles * kTileRows, hi - tok0));
     const long long row_base = (long long)cu * gm.max_seq_len + tok0;   // row of the 2-D view of the cache
 
-    float qr[DP];
-    load_group_query<DP>(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
-
     if (tid == 0) {
         for (int i = 0; i < n_stages && i < my_tiles; ++i) {
             mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
             tma_load_2d(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kTileRows), &sm->full[i]);
         }
     }
+    float qr[DP];
+    load_group_query<DP>(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
 
     // ---- stream + score + first digit histogram -------------------------------------------------
     bool timed_out = false;
@@ -584,6 +583,8 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     cfg.blockDim = dim3(kSelThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
+    // No programmatic dependent launch here: a selection that starts while the previous kernel still
+    // holds SMs gets its clusters placed in two batches (measured: +13 us per launch).
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = C;

@@ -695,10 +695,9 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             a.nsplit = n, nw = 8, a.cluster_merge = 1;
         } else {
             a.nsplit = pick_nsplit(c, units, max_rows);
-            if (a.nsplit <= 8 + 2) {
-                if (a.nsplit > 8) a.nsplit = 8;
-                a.cluster_merge = 1;
-            }
+            // clusters only when the whole launch is resident at once: in multi-wave launches the
+            // co-scheduling constraint costs more than the global merge (measured on the batch-8 workload)
+            if (a.nsplit <= 8 && units * a.nsplit <= 2 * c->sm_count) a.cluster_merge = 1;
         }
     } else {
         a.nsplit = pick_nsplit(c, units, max_rows);

@@ -656,6 +656,8 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             if (e != cudaSuccess) return e;
             (void)cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             (void)cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (cudaFuncSetAttribute(attn_mma_kernel<12, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) == cudaSuccess)
+                (void)cudaFuncSetAttribute(attn_mma_kernel<12, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             (void)cudaGetLastError();
             configured = true;
         }
@@ -693,6 +695,10 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
 #endif
         if (n && max_rows / n <= 1024) {
             a.nsplit = n, nw = 8, a.cluster_merge = 1;
+            // more than two tiles per warp would leave the third waiting for a free stage: 12 warps
+            // per block when their rings and the merge area still fit the SM
+            const int rows_per_block = (max_rows + n - 1) / n;
+            if (rows_per_block > 8 * 2 * kTileTok && 12 * 2 * kStageBytes + (size_t)n * gm.g * 132 * sizeof(float) <= 224 * 1024) nw = 12;
         } else {
             a.nsplit = pick_nsplit(c, units, max_rows);
             // clusters only when the whole launch is resident at once: in multi-wave launches the
@@ -733,6 +739,9 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         cfg.attrs = attr;
         cfg.numAttrs = 2;
         const __nv_bfloat16* kvp = (const __nv_bfloat16*)c->kv;
+        if (nw == 12)
+            return cudaLaunchKernelEx(&cfg, attn_mma_kernel<12, 2>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
+                                      c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
         if (nw == 8 && nst == 3)
             return cudaLaunchKernelEx(&cfg, attn_mma_kernel<8, 3>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
                                       c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);

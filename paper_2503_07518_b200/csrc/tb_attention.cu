@@ -531,13 +531,13 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
         l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
     }
     __syncwarp();
-    float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][128 channels]
+    float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][kMergePitch]
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) {
-        wo[(2 * tig) * D + mt * 16 + gid] = o[mt][0];
-        wo[(2 * tig + 1) * D + mt * 16 + gid] = o[mt][1];
-        wo[(2 * tig) * D + mt * 16 + gid + 8] = o[mt][2];
-        wo[(2 * tig + 1) * D + mt * 16 + gid + 8] = o[mt][3];
+        wo[(2 * tig) * kMergePitch + mt * 16 + gid] = o[mt][0];          // pitch 132: the 32 lanes hit 32 banks
+        wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid] = o[mt][1];
+        wo[(2 * tig) * kMergePitch + mt * 16 + gid + 8] = o[mt][2];
+        wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid + 8] = o[mt][3];
     }
     if (gid == 0) {
         sh_m[warp][2 * tig] = m_run[0], sh_l[warp][2 * tig] = l_run[0];
@@ -566,7 +566,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
             for (int w = 0; w < NW; ++w) {
                 const float e = sh_w[w][u];
                 lsum += sh_l[w][u] * e;
-                acc = fmaf(reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * D + tid], e, acc);
+                acc = fmaf(reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * kMergePitch + tid], e, acc);
             }
             cM[u] = sh_M[u], cL[u] = lsum, cO[u] = acc;
         }

@@ -173,6 +173,7 @@ def fill_caches(ctx, w, torch, tbh):
     dt = tbh.torch_dtype(w.dtype)
     gen = torch.Generator(device="cuda")
     total = sum(w.lengths)
+    ev = []
     for l in range(w.n_layers):
         gen.manual_seed(wl.seed_for(w.cfg_id, l, 0, wl.TAG_K))
         Wl = (torch.randn(w.n_kv_heads, w.head_dim, w.imp_dim, generator=gen, device="cuda") / np.sqrt(w.head_dim)).to(dt)
@@ -184,9 +185,17 @@ def fill_caches(ctx, w, torch, tbh):
                 k[:, h, torch.from_numpy(ch[h]).cuda()] *= 8.0
         v = torch.randn(total, w.n_kv_heads, w.head_dim, generator=gen, device="cuda")
         ctx.append_kv(l, 1, None, w.lengths, k.to(dt), v.to(dt))
-        ctx.project_keys(l, 1, None, [0] * w.batch, w.lengths)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.project_keys(l, 1, None, [0] * w.batch, w.lengths)          # the batched (post-prefill) projection
+        e1.record()
+        ev.append((e0, e1))
         del k, v
     torch.cuda.synchronize()
+    ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+    es = 2 if w.dtype == wl.BF16 else 4
+    nbytes = total * w.n_kv_heads * (w.head_dim + w.imp_dim) * es       # K rows read + projected rows written
+    return {"us_per_layer": ms * 1e3, "bytes_per_layer": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9}
 
 
 def run_ours(args, w):
@@ -206,7 +215,7 @@ def run_ours(args, w):
     p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode)
     ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + 8,
                       w.budget, w.radius, device=local)
-    fill_caches(ctx, w, torch, tbh)
+    proj_info = fill_caches(ctx, w, torch, tbh)
     dt = tbh.torch_dtype(w.dtype)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(wl.seed_for(w.cfg_id, 0, 0, wl.TAG_Q))
@@ -324,6 +333,7 @@ def run_ours(args, w):
                                       "gbs": sel_b / (ms_sel * 1e-3) / 1e9, "launches_per_step": len(groups)},
                     "attn_kernel": {"us_per_launch": ms_att * 1e3, "bytes_per_launch": att_b,
                                     "gbs": att_b / (ms_att * 1e-3) / 1e9, "launches_per_step": w.n_layers}},
+        "prefill_projection": proj_info,
         "clocks": sampler.summary(),
     }
     if rank == 0:

@@ -118,8 +118,10 @@ tb_status tb_append_kv(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, co
                        const int32_t* n_new, int32_t n_seq, const void* k_dev, const void* v_dev, void* stream);
 
 /* Sec. 3.1 "Key-cache projection" K_imp = K W_K for token positions [pos_begin[i], pos_end[i]) of
- * each listed sequence (fp32 accumulation over channels in ascending order, one rounding to
- * kv_dtype).  Eager (one token) or deferred batches (Sec. 3.3) are both just ranges.  Ranges must
+ * each listed sequence (fp32 accumulation -- tensor-core tiles for bf16 storage, an FMA chain in
+ * channel order for fp32 storage -- and one round-to-nearest-even to kv_dtype; a row's result does
+ * not depend on which call or batch projected it).  Eager (one token) or deferred batches
+ * (Sec. 3.3) are both just ranges.  Ranges must
  * lie inside the cached tokens and start at or before the sequence's projected length (no holes). */
 tb_status tb_project_keys(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, const int32_t* seq_ids,
                           const int32_t* pos_begin, const int32_t* pos_end, int32_t n_seq, void* stream);

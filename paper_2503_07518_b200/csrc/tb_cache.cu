@@ -107,6 +107,99 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTabl
     for (int j = 0; j < JPT; ++j) dst[j] = Elem<T>::from_f32(acc[j]);
 }
 
+// bf16 storage: the projection is the one dense contraction of the path ([tokens x 128] . [128 x d']
+// per KV head), so it runs on the tensor cores: 128 tokens per block, K rows and the W_K slice staged
+// in shared memory with 16-byte cp.async at conflict-free pitches, mma.sync m16n8k16 with fp32
+// accumulation, one round-to-nearest-even to bf16.  HBM-bound: 256 B read + 2 d' B written per token.
+constexpr int kPmTokens = 128;
+constexpr int kPmThreads = 128;
+constexpr int kPmKPitch = 272;            // 256 B of K + 16 B pad
+
+template <int DP>
+__global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTable ut, ProjectTable pt,
+                                                                 const __nv_bfloat16* __restrict__ kv,
+                                                                 const __nv_bfloat16* __restrict__ Wall,
+                                                                 __nv_bfloat16* __restrict__ kimp) {
+    constexpr int D = 128;
+    constexpr int kWPitch = DP * 2 + 16;  // bytes per W row (one channel, d' outputs) + pad
+    constexpr int NT = DP / 8;            // 8-wide output tiles
+    extern __shared__ __align__(16) unsigned char smem[];
+    unsigned char* Ks = smem;                                  // [128 tokens][kPmKPitch]
+    unsigned char* Ws = smem + kPmTokens * kPmKPitch;          // [128 channels][kWPitch]
+
+    const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq, h = blockIdx.y;
+    const int layer = ut.layer_begin + ll;
+    const int t0 = pt.pos_begin[s] + blockIdx.x * kPmTokens;
+    const int t_end = pt.pos_end[s];
+    if (t0 >= t_end) return;
+    const int nt_valid = min(kPmTokens, t_end - t0);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+
+    const size_t row0 = (((size_t)layer * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h) * gm.max_seq_len + t0;
+    const unsigned char* kbase = reinterpret_cast<const unsigned char*>(kv) + row0 * 2 * D * 2;
+    const unsigned char* wbase = reinterpret_cast<const unsigned char*>(Wall + ((size_t)layer * gm.Hkv + h) * D * DP);
+    const uint32_t ks_u32 = smem_u32(Ks), ws_u32 = smem_u32(Ws);
+    for (int i = tid; i < kPmTokens * 16; i += kPmThreads) {          // 16 chunks of 16 B per K row
+        const int t = i >> 4, ch = i & 15;
+        const int tc = min(t, nt_valid - 1);                           // rows past the range repeat the last one
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ks_u32 + t * kPmKPitch + ch * 16),
+                     "l"(kbase + (size_t)tc * 512 + ch * 16) : "memory");
+    }
+    for (int i = tid; i < D * (DP / 8); i += kPmThreads) {             // DP/8 chunks per W row
+        const int r = i / (DP / 8), ch = i % (DP / 8);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ws_u32 + r * kWPitch + ch * 16),
+                     "l"(wbase + (size_t)r * DP * 2 + ch * 16) : "memory");
+    }
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+    const int mi = lane >> 3, r8 = lane & 7;
+    // B fragments (W: k = channel, n = output) for every k-step and output tile, loaded once per warp
+    uint32_t bw[8][NT][2];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+        for (int np = 0; np < NT / 2; ++np) {
+            // matrices: (ch lo, outs np*16+0..7), (ch hi, same), (ch lo, outs +8), (ch hi, outs +8)
+            const uint32_t addr = ws_u32 + (ks * 16 + (mi & 1) * 8 + r8) * kWPitch + (np * 16 + (mi >> 1) * 8) * 2;
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(bw[ks][2 * np][0]), "=r"(bw[ks][2 * np][1]), "=r"(bw[ks][2 * np + 1][0]), "=r"(bw[ks][2 * np + 1][1])
+                         : "r"(addr));
+        }
+    __nv_bfloat16* out = kimp + row0 * DP;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+        const int tok = warp * 32 + mt * 16;                           // first token of this 16-token tile
+        float acc[NT][4];
+#pragma unroll
+        for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a0, a1, a2, a3;
+            const uint32_t addr = ks_u32 + (tok + (mi & 1) * 8 + r8) * kPmKPitch + ks * 32 + (mi >> 1) * 16;
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+#pragma unroll
+            for (int n = 0; n < NT; ++n)
+                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                             : "+f"(acc[n][0]), "+f"(acc[n][1]), "+f"(acc[n][2]), "+f"(acc[n][3])
+                             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bw[ks][n][0]), "r"(bw[ks][n][1]));
+        }
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+            const int j = n * 8 + tig * 2;
+            if (tok + gid < nt_valid) {
+                __nv_bfloat162 v = __floats2bfloat162_rn(acc[n][0], acc[n][1]);
+                *reinterpret_cast<__nv_bfloat162*>(out + (size_t)(tok + gid) * DP + j) = v;
+            }
+            if (tok + gid + 8 < nt_valid) {
+                __nv_bfloat162 v = __floats2bfloat162_rn(acc[n][2], acc[n][3]);
+                *reinterpret_cast<__nv_bfloat162*>(out + (size_t)(tok + gid + 8) * DP + j) = v;
+            }
+        }
+    }
+}
+
 cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, cudaStream_t s) {
     ProjectTable pt;
     int max_range = 0;
@@ -117,14 +210,35 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
     }
     if (max_range <= 0) return cudaSuccess;
     const Geom& gm = c->geom;
+    if (gm.dtype == TB_BF16) {
+        dim3 grid_mma((max_range + kPmTokens - 1) / kPmTokens, gm.Hkv, ut.layer_count * ut.n_seq);
+        const __nv_bfloat16* kvp = (const __nv_bfloat16*)c->kv;
+        const __nv_bfloat16* wp = (const __nv_bfloat16*)c->st.W;
+        if (gm.dp == 32) {
+            const size_t smem = kPmTokens * kPmKPitch + 128 * (32 * 2 + 16);
+            static bool configured = false;
+            if (!configured) {
+                cudaError_t e = cudaFuncSetAttribute(project_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                if (e != cudaSuccess) return e;
+                configured = true;
+            }
+            project_mma_kernel<32><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp);
+        } else {
+            const size_t smem = kPmTokens * kPmKPitch + 128 * (16 * 2 + 16);
+            static bool configured = false;
+            if (!configured) {
+                cudaError_t e = cudaFuncSetAttribute(project_mma_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                if (e != cudaSuccess) return e;
+                configured = true;
+            }
+            project_mma_kernel<16><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp);
+        }
+        return cudaGetLastError();
+    }
     dim3 grid((max_range + kProjTokens - 1) / kProjTokens, gm.Hkv, ut.layer_count * ut.n_seq);
 #define TB_PROJ(T, DP) \
     project_kernel<T, DP><<<grid, kProjThreads, 0, s>>>(gm, ut, pt, (const T*)c->kv, (const T*)c->st.W, (T*)c->kimp)
-    if (gm.dtype == TB_BF16) {
-        if (gm.dp == 32) TB_PROJ(__nv_bfloat16, 32); else TB_PROJ(__nv_bfloat16, 16);
-    } else {
-        if (gm.dp == 32) TB_PROJ(float, 32); else TB_PROJ(float, 16);
-    }
+    if (gm.dp == 32) TB_PROJ(float, 32); else TB_PROJ(float, 16);
 #undef TB_PROJ
     return cudaGetLastError();
 }

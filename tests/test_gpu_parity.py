@@ -302,3 +302,49 @@ def test_bit_reproducible(H):
     ob, lb = H.gpu_attention(case, q, p)
     assert all(np.array_equal(x, y) for l in range(2) for s in range(2) for x, y in zip(a[l][s], b[l][s]))
     assert np.array_equal(oa, ob) and np.array_equal(la, lb)
+
+
+def _crafted_scores_case(H, scores_per_head, budget, sinks=0, recent=0):
+    """A cluster-sized problem (one sequence, L = len(scores)) whose importance scores are exactly the
+    given values: K_imp rows are score * e_0 and the importance query is e_0."""
+    L = scores_per_head.shape[1]
+    n_heads = scores_per_head.shape[0]
+    w = wl.workload(2, n_layers=1, n_q_heads=n_heads, n_kv_heads=n_heads, lengths=[L], budget=budget, sinks=sinks, recent=recent)
+    case = H.Case(w, project="oracle-only")
+    for h in range(n_heads):
+        kimp = np.zeros((L, w.imp_dim), np.float32)
+        kimp[:, 0] = scores_per_head[h]
+        bits = wl.to_storage(kimp, w.dtype)
+        assert np.array_equal(wl.storage_to_f32(bits, w.dtype)[:, 0], scores_per_head[h]), "scores must be bf16-exact"
+        case.Kimp[0][0][h, :L] = bits
+        case.ctx.kimp[0, 0, h, :L] = H.to_dev(bits, w.dtype)
+    qi = np.zeros((1, 1, n_heads, w.imp_dim), np.float32)
+    qi[..., 0] = 1.0
+    p = tb().select_params(budget, sinks, recent)
+    lists = H.gpu_select(case, qi, p)
+    assert case.ctx.get_status() == 0
+    for h in range(n_heads):
+        _, full, _ = case.oracle_select(0, 0, h, qi[0, 0], p)
+        assert np.array_equal(lists[0][0][h], full), "head %d" % h     # exact scores: no tolerance
+    return lists
+
+
+def test_cluster_selection_unusual_distributions(H):
+    """Paths of the cluster radix select that ordinary data never takes (20011 tokens, 2 heads: a cluster of 8)."""
+    r = np.random.Generator(np.random.PCG64(77))
+    L = 20011
+    # every score equal: the threshold bin holds everything, the lowest positions win
+    _crafted_scores_case(H, np.zeros((2, L), np.float32), budget=777, sinks=5, recent=9)
+    _crafted_scores_case(H, np.full((2, L), -3.5, np.float32), budget=1)
+    # scores over ~400 binades and both signs: more non-empty first-digit bins than a block may publish
+    expo = r.integers(-100, 101, size=(2, L))
+    sign = r.choice([-1.0, 1.0], size=(2, L))
+    _crafted_scores_case(H, (sign * np.exp2(expo)).astype(np.float32), budget=2500)
+    # a few distinct values: thousands of exact ties at the threshold, spread over all blocks
+    vals = r.integers(0, 12, size=(2, L)).astype(np.float32)
+    _crafted_scores_case(H, vals, budget=3000)                          # ~1670 per value: the quota ends inside a class
+    _crafted_scores_case(H, r.integers(0, 3, size=(2, L)).astype(np.float32), budget=9000)   # class of ~6670 keys
+    # the budget ends exactly at a class boundary (whole threshold bin taken)
+    v = np.zeros((2, L), np.float32)
+    v[:, ::7] = 4.0
+    _crafted_scores_case(H, v, budget=int((v[0] == 4.0).sum()))

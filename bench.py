@@ -509,10 +509,14 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=2, help="layers in the CPU oracle's sample")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--profile", action="store_true", help="only warm-up + steps of plain launches (for ncu)")
+    ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
+                    help="neighbour rule of the interval workload (default: its own, +-r dilation)")
     args = ap.parse_args()
     w = wl.workload(args.config)
     if args.layers:
         w = w.scaled(n_layers=args.layers)
+    if args.neighbors:
+        w = w.scaled(nmode=0 if args.neighbors == "dilate" else 1)
     if args.impl == "reference":
         run_reference(args, w)
     else:

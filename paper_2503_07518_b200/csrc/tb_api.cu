@@ -173,6 +173,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->last_bytes = 0, c->launches = 0;
     c->last_cache_write = c->last_list_write = -4;
     c->tile_rows = 256;
+    for (int i = 0; i < 17; ++i) c->attn_max_active[i] = 0;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete c; return TB_ERR_CUDA; }
     // only the small control parts need defined contents; the index lists and partials are always
     // written before they are read
@@ -394,7 +395,8 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
     uint64_t bytes = 0;
     int bound = c->geom.idx_cap;
     if (!dense && !idx) {
-        long long b = (long long)(2 * p->radius + 1) * p->budget;
+        // DILATE grows a selection to at most (2r+1)B positions, CLUSTER to (1+r)B
+        long long b = (long long)(p->nmode == TB_NEIGHBOR_CLUSTER ? 1 + p->radius : 2 * p->radius + 1) * p->budget;
         if (b < bound) bound = (int)b;
     }
     for (int l = lb; l < lb + lc; ++l)

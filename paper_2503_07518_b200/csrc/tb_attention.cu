@@ -69,7 +69,7 @@ struct SplitSink {
         __threadfence();
         // all (head, split) statistics in one round trip, then weights, then 16-byte wide sums
         __shared__ float mm[kMaxGroup][kMaxSplits], lw[kMaxGroup][kMaxSplits], w[kMaxGroup][kMaxSplits];
-        __shared__ float Lsum[kMaxGroup], Mmax[kMaxGroup];
+        __shared__ float Lsum[kMaxGroup];
         for (int i = tid; i < g * nsplit; i += kAttnThreads) {
             const int u = i / nsplit, j = i % nsplit;
             const size_t pq = (hq0 + u) * kMaxSplits + j;
@@ -87,7 +87,7 @@ struct SplitSink {
                 w[tid][j] = e;
                 lsum += lw[tid][j] * e;
             }
-            Lsum[tid] = lsum, Mmax[tid] = M;
+            Lsum[tid] = lsum;
             if (lse) lse[hq0 + tid] = (M + log2f(lsum)) * kLn2;
         }
         __syncthreads();
@@ -647,9 +647,9 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
     a.cluster_merge = 0;
     int nw = kAttnWarps;
     if (gm.dtype == TB_BF16) {
-        static bool configured = false;
-        static int max_active[17];                    // co-resident clusters of the 8-warp kernel per cluster size (0 = not asked yet)
-        if (!configured) {
+        static unsigned char seen[64];
+        int* max_active = const_cast<tb_ctx*>(c)->attn_max_active;
+        if (first_use_on_this_device(seen)) {
             cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
             if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
@@ -659,7 +659,6 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             if (cudaFuncSetAttribute(attn_mma_kernel<12, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) == cudaSuccess)
                 (void)cudaFuncSetAttribute(attn_mma_kernel<12, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             (void)cudaGetLastError();
-            configured = true;
         }
         auto clusters_that_fit = [&](int csize) {     // how many clusters of `csize` 8-warp blocks run at once
             if (max_active[csize] == 0) {

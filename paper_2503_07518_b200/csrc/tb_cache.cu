@@ -216,20 +216,18 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
         const __nv_bfloat16* wp = (const __nv_bfloat16*)c->st.W;
         if (gm.dp == 32) {
             const size_t smem = kPmTokens * kPmKPitch + 128 * (32 * 2 + 16);
-            static bool configured = false;
-            if (!configured) {
+            static unsigned char seen[64];
+            if (first_use_on_this_device(seen)) {
                 cudaError_t e = cudaFuncSetAttribute(project_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 if (e != cudaSuccess) return e;
-                configured = true;
             }
             project_mma_kernel<32><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp);
         } else {
             const size_t smem = kPmTokens * kPmKPitch + 128 * (16 * 2 + 16);
-            static bool configured = false;
-            if (!configured) {
+            static unsigned char seen[64];
+            if (first_use_on_this_device(seen)) {
                 cudaError_t e = cudaFuncSetAttribute(project_mma_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 if (e != cudaSuccess) return e;
-                configured = true;
             }
             project_mma_kernel<16><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp);
         }

@@ -96,6 +96,7 @@ struct tb_ctx {
     CUtensorMap kimp_map;                 // 2-D view of kimp: rows = all token slots, cols = d'
     int tile_rows;                        // rows per TMA box of the score pass
     int sm_count;
+    int attn_max_active[17];              // co-resident attention clusters per cluster size (0 = not asked yet)
     uint64_t last_bytes, launches;
     // index (value of `launches` at launch time) of the last kernel that wrote the caches / the stored
     // lists; a kernel may read them before its dependency wait only if that writer is not its predecessor
@@ -103,6 +104,16 @@ struct tb_ctx {
 };
 
 namespace tb {
+
+// Kernel attributes (dynamic shared-memory limit, non-portable cluster sizes) belong to a device's
+// context, so each launcher configures its kernels on first use per device.
+inline bool first_use_on_this_device(unsigned char (&seen)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+    if (seen[dev]) return false;
+    seen[dev] = 1;
+    return true;
+}
 
 // tb_cache.cu
 cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new, const int* tok_off, int total_new,

@@ -156,7 +156,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     const int C = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const unsigned lt_mask = (1u << lane) - 1u;
 
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
@@ -595,12 +594,11 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
 
 #define TB_SEL(T, DP)                                                                                              \
     do {                                                                                                           \
-        static bool configured = false;                                                                            \
-        if (!configured) {                                                                                         \
+        static unsigned char seen[64];                                                                            \
+        if (first_use_on_this_device(seen)) {                                                                                         \
             cudaError_t e = cudaFuncSetAttribute(select_kernel<T, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                                  227 * 1024);                                                      \
             if (e != cudaSuccess) return e;                                                                        \
-            configured = true;                                                                                     \
         }                                                                                                          \
         return cudaLaunchKernelEx(&cfg, select_kernel<T, DP>, c->kimp_map, gm, ut, a, tiles_per_cta, n_stages, c->st.idx, \
                                   c->st.cnt, c->st.status);                                                        \

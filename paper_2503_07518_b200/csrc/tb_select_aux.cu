@@ -122,11 +122,10 @@ cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const Neighbo
         if (hi - lo > max_span) max_span = hi - lo;
     }
     size_t smem = (size_t)((max_span + 31) / 32) * 4 + 16;
-    static bool configured = false;
-    if (!configured) {
+    static unsigned char seen[64];
+    if (first_use_on_this_device(seen)) {
         cudaError_t e = cudaFuncSetAttribute(neighbor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
     neighbor_kernel<<<ut.layer_count * ut.n_seq * gm.Hkv, kNbThreads, smem, s>>>(gm, ut, a, c->st.idx, c->st.cnt);

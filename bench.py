@@ -50,9 +50,10 @@ def measured_peaks():
 # --------------------------------------------------------------------------------------------------
 # CPU oracle leg (cpu_baseline and --impl reference)
 
-def oracle_sample(w: wl.Workload, n_layers: int, passes: int, threads: int):
-    """Times the oracle, as it stands, on all (sequence, KV head) units of `n_layers` layers of the
-    workload, host-generated inputs.  Returns (seconds per pass list, units in the sample)."""
+def oracle_sample(w: wl.Workload, n_layers: int, passes: int, threads: int, max_units: int = 0):
+    """Times the oracle, as it stands, on the (sequence, KV head) units of `n_layers` layers of the
+    workload (at most `max_units` of them if given), host-generated inputs.  Returns (seconds per pass
+    list, units in the sample)."""
     from oracle import tb_oracle as orc
     orc.build()
     units, qis, qs, Ls = [], [], [], []
@@ -60,9 +61,13 @@ def oracle_sample(w: wl.Workload, n_layers: int, passes: int, threads: int):
     for l in range(n_layers):
         W = wl.gen_W(w, l)
         for b in range(w.batch):
+            if max_units and len(units) >= max_units:
+                break
             K, V = wl.gen_KV(w, l, b)
             q, qi = wl.gen_queries(w, l, b)
             for h in range(w.n_kv_heads):
+                if max_units and len(units) >= max_units:
+                    break
                 Kh, Vh = np.ascontiguousarray(K[h]), np.ascontiguousarray(V[h])
                 units.append(orc.Unit(Kh, Vh, orc.project_keys(Kh, np.ascontiguousarray(W[h]), w.dtype), cap))
                 qis.append(qi[h * w.group:(h + 1) * w.group])
@@ -77,21 +82,25 @@ def oracle_sample(w: wl.Workload, n_layers: int, passes: int, threads: int):
     return times, len(units)
 
 
-def cpu_leg(w: wl.Workload, sample_layers: int, passes: int):
+def cpu_leg(w: wl.Workload, sample_layers: int, passes: int, max_units: int = 0):
     threads = len(os.sched_getaffinity(0))
-    times, n_units = oracle_sample(w, sample_layers, passes, threads)
+    times, n_units = oracle_sample(w, sample_layers, passes, threads, max_units)
     total_units = w.n_layers * w.batch * w.n_kv_heads
     step_s = [t * total_units / n_units for t in times]          # units are independent: linear scaling
-    return {"times": step_s, "threads": threads,
-            "sample": "%d of %d layers (%d of %d (sequence, KV head) units) of %s, one refresh step each pass, "
-                      "scaled linearly to the whole step" % (sample_layers, w.n_layers, n_units, total_units, w.name)}
+    return {"times": step_s, "threads": min(threads, n_units),
+            "sample": "%d of %d (layer, sequence, KV head) units of %s (layer 0 first), one refresh step each pass, "
+                      "scaled linearly to the whole step" % (n_units, total_units, w.name)}
 
 
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    leg = cpu_leg(w, 1, args.steps + args.warmup)       # one layer per step keeps K steps within minutes
+    # bounded sample per step so that K steps end within minutes: a layer's 8 heads for short runs,
+    # down to a single (layer, sequence, KV head) unit for long ones
+    passes = args.steps + args.warmup
+    max_units = 8 if passes <= 25 else (2 if passes <= 250 else 1)
+    leg = cpu_leg(w, 1, passes, max_units)
     t = leg["times"][args.warmup:]
     ms = 1e3 * float(np.mean(t))
     val = w.batch / (ms * 1e-3)

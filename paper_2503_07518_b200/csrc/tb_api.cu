@@ -17,7 +17,7 @@ int elem_size(int dtype) { return dtype == TB_BF16 ? 2 : 4; }
 struct Layout {
     size_t kv_bytes, kimp_bytes;
     size_t off_W, off_idx, off_cnt, off_status, off_counter, state_bytes;
-    size_t off_part_o, off_part_ml, off_sel_idx, off_sel_cnt, work_bytes;
+    size_t off_part_o, off_part_ml, off_sel_idx, off_sel_cnt, off_sel_keys, work_bytes;
     int idx_cap, sel_stride;
 };
 
@@ -59,6 +59,7 @@ void compute_layout(const tb_config* c, Layout* l) {
     l->off_part_ml = o, o = align_up(o + units_q * kMaxSplits * 2 * 4, 256);
     l->off_sel_idx = o, o = align_up(o + units * l->sel_stride * 4, 256);
     l->off_sel_cnt = o, o = align_up(o + units * 4, 256);
+    l->off_sel_keys = o, o = align_up(o + units * align_up((size_t)c->max_seq_len, 4) * 4, 256);   // one 32-bit key per token
     l->work_bytes = o;
 }
 
@@ -164,6 +165,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->wk.sel_idx = (int32_t*)(wp + l.off_sel_idx);
     c->wk.sel_cnt = (int32_t*)(wp + l.off_sel_cnt);
     c->wk.sel_stride = l.sel_stride;
+    c->wk.sel_keys = (uint32_t*)(wp + l.off_sel_keys);
     Geom& g = c->geom;
     g.n_layers = cfg->n_layers, g.Hq = cfg->n_q_heads, g.Hkv = cfg->n_kv_heads, g.g = cfg->n_q_heads / cfg->n_kv_heads;
     g.D = cfg->head_dim, g.dp = cfg->imp_dim, g.max_batch = cfg->max_batch, g.max_seq_len = cfg->max_seq_len;
@@ -323,7 +325,6 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                 if (c->len[u] <= 0) return TB_ERR_INVALID_ARG;
                 int lo, hi;
                 cand_range(c->len[u], p->sinks, p->recent, &lo, &hi);
-                if (hi - lo > 8 * 32768) return TB_ERR_UNSUPPORTED;          // 8 blocks x 32768 on-chip scores
                 if (c->len_proj[u] < hi) return TB_ERR_UNPROJECTED;
                 bytes += (uint64_t)(hi - lo) * c->cfg.n_kv_heads * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);
             }

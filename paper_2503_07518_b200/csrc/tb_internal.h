@@ -78,6 +78,7 @@ struct DevWork {
     int32_t* sel_idx;     // [n_layers*max_batch*Hkv][max_budget rounded]  pre-expansion selection
     int32_t* sel_cnt;
     int sel_stride;
+    uint32_t* sel_keys;   // [n_layers*max_batch*Hkv][max_seq_len rounded up to 4]  score keys of a many-problem selection launch
 };
 
 }  // namespace tb
@@ -124,6 +125,8 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
 cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, float scale, float* scores,
                          cudaStream_t s);
 cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
+// one block per problem; launch_select hands over to it when a launch holds at least two problems per SM
+cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s);
 cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s);
 

@@ -547,6 +547,10 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
         int L = ut.len[i], lo = a.sinks < L ? a.sinks : L, hi = L - a.recent > lo ? L - a.recent : lo;
         if (hi - lo > max_cand) max_cand = hi - lo;
     }
+    // Many problems (one and a half per SM or more; measured crossover between 32 and 256 on 148 SMs)
+    // fill the GPU by themselves: one block each, no clusters.  So do problems too long for a cluster's
+    // on-chip key arrays.
+    if (2 * n_units >= 3 * c->sm_count || max_cand > kMaxCluster * kMaxKeysPerBlock) return launch_select_wave(c, ut, a, s);
     const int n_tiles = (max_cand + kTileRows - 1) / kTileRows;
     // Cluster size: enough blocks to cover the GPU about twice, at least 4 tiles per block, and a
     // key array per block of at most 32 KB where the cluster limit allows (64 KB otherwise).

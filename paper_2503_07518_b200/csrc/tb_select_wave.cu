@@ -1,0 +1,627 @@
+// Fused importance scoring + exact top-B selection for launches with many problems (paper Sec. 3.4
+// "score computation against all projected keys ... top-B selection", Sec. 4 "Token Selection
+// Policy"): batched serving, where one launch holds several hundred (layer, sequence, KV head)
+// problems and the GPU is filled by problems, not by splitting one.
+//
+// One block per problem, four blocks per SM, longest problems first.
+//   sample   the block scores 64 rows spread over its problem and brackets, generously, where the
+//            B-th largest score will fall.  That only places the bins of the first radix digit: 2046
+//            equal slices across the bracket, one open bin below, one above.  The digit is monotone in
+//            the key whatever the sample says, so the result never depends on it; only how few keys
+//            share the threshold's bin does (a handful, against a tenth of the problem for the key's
+//            top bits).
+//   stream   candidate rows of the projected-key cache through a ring of 2-D TMA tiles (evict-first in
+//            L2); every row is scored, its order-preserving 32-bit key parked in a workspace row
+//            (4 bytes per token against the 64 just read, evict-last so it is still in L2 later) and
+//            its first digit counted in shared memory.
+//   finish   threshold bin from the histogram; one pass over the parked keys turns "above the bin"
+//            into a bitmask (one word per eight lanes) and sets the few keys inside the bin aside;
+//            those are ranked among themselves (equal keys by position), the winners' bits set, and a
+//            prefix over the mask's popcounts places the ascending list.
+//   general  a threshold in the open bin below the bracket, or a bin too crowded to set aside
+//            (massive ties), falls back to a plain three-digit radix select over all parked keys with
+//            an ordered compaction.  Slower, never wrong.
+// No block waits for another.  The cluster kernel in tb_select.cu serves launches with few, large
+// problems, where one problem must be split over many SMs; in this regime it would spend its time in
+// cluster barriers.
+#include <algorithm>
+#include <cstddef>
+
+#include "tb_select.cuh"
+
+namespace tb {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kRows = 256;          // rows per TMA box = one row per thread
+constexpr int kStagesMax = 8;
+constexpr int kRingBytes = 32 * 1024;
+constexpr int kDigitBins = 2048;    // 11-bit digits (the last digit has 10 bits)
+constexpr int kSampleRows = 64;     // rows scored up front to place the first digit's bins
+constexpr int kMinSampled = 2048;   // smaller problems use the key's top bits as first digit
+constexpr int kBatch = 8;           // 16-byte key loads a thread keeps in flight
+
+// Launch order of the (layer, sequence) pairs: longest first, so that the blocks still running when
+// the grid drains are the short ones.
+struct WaveOrder {
+    uint16_t pair[kMaxLaunchUnits];
+};
+
+#ifdef TB_PHASE_TIMING
+__device__ unsigned long long g_fin_ns[8];
+__device__ unsigned long long g_wave_ns[4][1024];       // per block: start, first tile landed, rows streamed, end
+__device__ __forceinline__ unsigned long long wave_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void wave_stamp(int i) {
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_wave_ns[i][blockIdx.x] = t;
+    }
+}
+#else
+__device__ __forceinline__ void wave_stamp(int) {}
+#endif
+
+struct __align__(16) WaveSmem {
+    uint32_t sample[kSampleRows];   // first: read with 16-byte loads
+    uint64_t full[kStagesMax];
+    int warp_a[kWarps];
+    int warp_b[kWarps];
+    int bc_bin, bc_krem, bc_count, n_list;
+    uint32_t s_lo, s_hi;            // sample keys bracketing the expected threshold
+};
+static_assert(offsetof(WaveSmem, sample) % 16 == 0, "sample is read as uint4");
+
+// First digit of the radix select: 2048 bins, monotone in the key.  Bin 0 = below `base`, bins
+// 1..2046 = equal slices of 2^shift keys from `base` up, bin 2047 = everything above.  With base = 0
+// and shift = 21 it is the key's top 11 bits; with base and shift taken from a sample of the problem's
+// scores the slices around the expected threshold hold a handful of keys each.
+struct Digit {
+    uint32_t base;
+    int shift;
+    __device__ __forceinline__ int bin(uint32_t key) const {
+        return key < base ? 0 : (int)min((key - base) >> shift, 2046u) + 1;
+    }
+};
+
+__device__ __forceinline__ void hist_add(int* p) {
+    asm volatile("red.shared.add.s32 [%0], 1;" ::"r"(smem_u32(p)) : "memory");
+}
+
+// Exclusive prefix of `v` over the block in thread order, and the block total.  One barrier; uses
+// `slots` (kWarps ints), which must not be reused before the next barrier.
+__device__ __forceinline__ int wave_excl_scan(int v, int* slots, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int incl = warp_incl_scan(v, lane);
+    if (lane == 31) slots[warp] = incl;
+    __syncthreads();
+    int before = 0;
+    total = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        const int x = slots[w];
+        total += x;
+        before += w < warp ? x : 0;
+    }
+    return before + incl - v;
+}
+
+// Finds, over PER*256 counters ordered by digit value, the digit b with
+//   count(digits > b) < k <= count(digits >= b)
+// and returns it with k' = k - count(digits > b) and the population of b.  All threads call it and
+// all receive the same answer.  Preconditions: 1 <= k <= total count.
+template <int PER>
+__device__ __forceinline__ void wave_find_digit(const int* hist, int k, WaveSmem* sm, int& bin, int& krem, int& bcount) {
+    const int tid = threadIdx.x;
+    int b[PER];
+    const int4* p = reinterpret_cast<const int4*>(hist + tid * PER);
+#pragma unroll
+    for (int v = 0; v < PER / 4; ++v) {
+        const int4 x = p[v];
+        b[4 * v] = x.x, b[4 * v + 1] = x.y, b[4 * v + 2] = x.z, b[4 * v + 3] = x.w;
+    }
+    int mine = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) mine += b[i];
+    int total;
+    const int excl = wave_excl_scan(mine, sm->warp_a, total);
+    const int above = total - excl - mine;           // keys in digits above this thread's digits
+    if (above < k && k <= above + mine) {            // exactly one thread
+        int run = above;
+        bool done = false;
+#pragma unroll
+        for (int i = PER - 1; i >= 0; --i) {
+            if (!done && run + b[i] >= k) {
+                sm->bc_bin = tid * PER + i, sm->bc_krem = k - run, sm->bc_count = b[i];
+                done = true;
+            }
+            run += b[i];
+        }
+    }
+    __syncthreads();
+    bin = sm->bc_bin, krem = sm->bc_krem, bcount = sm->bc_count;
+    __syncthreads();                                  // bc_* and warp_a may be reused right away
+}
+
+}  // namespace
+
+// Finish of one problem from its complete first-digit histogram, with ONE pass over the keys.
+// The first digit already decides almost every key: above the threshold bin = selected, below = not.
+// The pass turns that into a bitmask (one ballot per 32 positions) and sets aside the few keys of the
+// threshold bin as (low 21 bits, position) pairs; two more digits are then resolved on that short
+// list, equal keys by position, the winners' bits are set, and a prefix over the mask's popcounts
+// places the ascending list.  `scratch` (the idle ring) holds mask and list.  Returns false, having
+// written nothing, when they do not fit (a crowded threshold bin): the caller then takes the general
+// path.  All threads call it and all get the same answer.
+__device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const Digit dg, const uint32_t* __restrict__ keys,
+                                                 unsigned char* scratch, int scratch_bytes, int ncand, int k, int lo,
+                                                 int32_t* __restrict__ idx_dst, int32_t* __restrict__ cnt_dst) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
+#ifdef TB_PHASE_TIMING
+    unsigned long long tf0 = wave_now();
+#define FIN_MARK(i) do { if (tid == 0) { unsigned long long tn = wave_now(); atomicAdd(&g_fin_ns[i], tn - tf0); tf0 = tn; } } while (0)
+#else
+#define FIN_MARK(i) do {} while (0)
+#endif
+    int bin, krem, bc;
+    wave_find_digit<8>(hist, k, sm, bin, krem, bc);
+    FIN_MARK(0);
+    const bool exact = bc == krem;                     // the whole threshold bin is selected
+    const int n_grp = (ncand + kRows - 1) / kRows;     // groups of 256 positions = 8 mask words
+    const int n_words = n_grp * kWarps;
+    const int mask_bytes = (n_words * 4 + 15) & ~15;
+    uint32_t* mask = reinterpret_cast<uint32_t*>(scratch);
+    uint2* list = reinterpret_cast<uint2*>(scratch + mask_bytes);
+    // bin 0 (everything below the sampled range) is too crowded to list
+    if (mask_bytes > scratch_bytes || (!exact && (bc > (scratch_bytes - mask_bytes) / 8 || bin == 0))) return false;
+    const uint32_t bin_base = dg.base + ((uint32_t)(bin - 1) << dg.shift);       // lowest key of the threshold bin
+    const int bin_bits = bin == 2047 ? 32 : dg.shift;  // bits of (key - bin_base) inside the bin; the top bin is open-ended
+    if (tid == 0) sm->n_list = 0;
+    __syncthreads();
+#ifdef TB_PHASE_TIMING
+    if (tid == 0) atomicAdd(&g_fin_ns[7], 1ull), atomicAdd(&g_fin_ns[6], (unsigned long long)(exact ? 0 : bc));
+#endif
+
+    // Lane l of a warp holds positions 128 g + 4 l .. + 3 (one 16-byte load): its four verdicts are a
+    // nibble, eight lanes' nibbles make a mask word.
+    const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
+    const int n_vec = (ncand + 3) / 4;
+    const uint32_t oct = 0xffu << (lane & 24);         // the eight lanes that share a mask word
+    for (int v0 = tid; v0 < n_grp * (kRows / 4); v0 += kThreads * kBatch) {   // kBatch loads in flight, then their verdicts
+        uint4 x[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int v = v0 + u * kThreads;
+            x[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (v < n_vec) x[u] = __ldcg(keys4 + v);
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int v = v0 + u * kThreads;
+            if (v - lane >= n_grp * (kRows / 4)) break;    // warp-uniform: whole warps leave together
+            const uint32_t kk[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+            uint32_t take = 0, eqm = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int c = dg.bin(kk[e]);
+                const bool valid = v * 4 + e < ncand;
+                take |= (uint32_t)(valid && (c > bin || (c == bin && exact))) << e;
+                eqm |= (uint32_t)(valid && c == bin) << e;
+            }
+            const uint32_t word = __reduce_or_sync(oct, take << (4 * (lane & 7)));
+            if ((lane & 7) == 0) mask[v >> 3] = word;  // positions 32 (v / 8) .. + 31
+            if (!exact && __any_sync(0xffffffffu, eqm != 0)) {
+                const int ne = __popc(eqm);
+                const int incl = warp_incl_scan(ne, lane);
+                int base = 0;
+                if (lane == 31) base = atomicAdd(&sm->n_list, incl);
+                base = __shfl_sync(0xffffffffu, base, 31) + incl - ne;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if ((eqm >> e) & 1) list[base++] = make_uint2(kk[e] - bin_base, (uint32_t)(v * 4 + e));
+            }
+        }
+    }
+    __syncthreads();
+    FIN_MARK(1);
+
+    if (!exact) {
+        const int n_in = sm->n_list;                   // == bc
+        uint32_t prefix = 0;
+        int low_bits = bin_bits;
+        bool ex = false;
+        if (n_in <= kThreads) {
+            // a short list: every entry counts the entries ranked before it (larger key, or equal key at
+            // a lower position) and knows at once whether it is among the `krem` winners
+            if (tid < n_in) {
+                const uint2 it = list[tid];
+                int before = 0;
+                for (int j = 0; j < n_in; ++j) {
+                    const uint2 o = list[j];
+                    before += (o.x > it.x) | ((o.x == it.x) & (o.y < it.y));
+                }
+                if (before < krem) atomicOr(&mask[it.y >> 5], 1u << (it.y & 31));
+            }
+            __syncthreads();
+            low_bits = -1;                             // done
+        }
+        // otherwise the remaining bits of the keys in the list, 11 at a time
+#pragma unroll 1
+        while (!ex && low_bits > 0) {
+            const int bits = low_bits < 11 ? low_bits : 11, shift = low_bits - bits;
+            const uint32_t dmask = (1u << bits) - 1u;
+            for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
+            __syncthreads();
+            for (int i = tid; i < n_in; i += kThreads) {
+                const uint32_t v = list[i].x;
+                if ((uint32_t)((uint64_t)v >> low_bits) == prefix) hist_add(&hist[(v >> shift) & dmask]);
+            }
+            __syncthreads();
+            int d, kr, c;
+            wave_find_digit<8>(hist, krem, sm, d, kr, c);
+            prefix = (prefix << bits) | (uint32_t)d, low_bits = shift, krem = kr, ex = c == kr;
+        }
+        // winners: above the class; the whole class when `ex`; else (equal keys, more than places
+        // left) the `krem` lowest positions among them
+        for (int i = tid; i < n_in && low_bits >= 0; i += kThreads) {
+            const uint2 it = list[i];
+            const uint32_t c = it.x >> low_bits;
+            bool take = c > prefix;
+            if (c == prefix) {
+                take = ex;
+                if (!ex) {
+                    int before = 0;                    // equal keys at lower positions
+                    for (int j = 0; j < n_in; ++j) {
+                        const uint2 o = list[j];
+                        before += (o.x == it.x) & (o.y < it.y);
+                    }
+                    take = before < krem;
+                }
+            }
+            if (take) atomicOr(&mask[it.y >> 5], 1u << (it.y & 31));
+        }
+        __syncthreads();
+    }
+
+    FIN_MARK(2);
+    // ascending list from the mask: each thread owns a run of words
+    const int per = (n_words + kThreads - 1) / kThreads;
+    const int w0 = min(n_words, tid * per), w1 = min(n_words, w0 + per);
+    int cnt = 0;
+    for (int w = w0; w < w1; ++w) cnt += __popc(mask[w]);
+    int total;
+    int o = wave_excl_scan(cnt, sm->warp_a, total);
+    for (int w = w0; w < w1; ++w) {
+        uint32_t bits = mask[w];
+        while (bits) {
+            const int b = __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (o < k) idx_dst[o] = lo + w * 32 + b;
+            ++o;
+        }
+    }
+    if (tid == 0) *cnt_dst = k;
+    FIN_MARK(3);
+    return true;
+}
+
+template <typename T, int DP>
+__global__ void __launch_bounds__(kThreads, 4)
+    select_wave_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut,
+                       WaveOrder order, SelectArgs a, int n_stages,
+                       int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt, int32_t* __restrict__ status,
+                       uint32_t* __restrict__ keys_g) {
+    constexpr int RB = DP * Elem<T>::kBytes;          // bytes per projected-key row: 32, 64 or 128
+    constexpr int NCH = RB / 16;
+    constexpr uint32_t kTileBytes = kRows * RB;
+
+    extern __shared__ unsigned char smem_raw[];
+    // swizzled TMA boxes need their shared-memory base on the swizzle period (up to 1024 bytes)
+    unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    int* hist = reinterpret_cast<int*>(stage_base + n_stages * kTileBytes);       // one digit at a time
+    WaveSmem* sm = reinterpret_cast<WaveSmem*>(hist + kDigitBins);
+    // The ring is idle once the rows are streamed; it then caches the problem's keys (as many as fit).
+    uint4* key_cache = reinterpret_cast<uint4*>(stage_base);
+    const int cache_vecs = n_stages * (int)kTileBytes / 16;                      // 16-byte vectors of 4 keys
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pair = order.pair[blockIdx.x / gm.Hkv], h = blockIdx.x % gm.Hkv;
+    const int ll = pair / ut.n_seq, s = pair % ut.n_seq;
+    const int L = ut.len[pair];
+    const int lo = min(a.sinks, L);
+    const int hi = max(lo, L - a.recent);
+    const int ncand = hi - lo;
+    const int k = min(a.budget, ncand);
+    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t dst_row = a.dst_is_state ? cu : (size_t)pair * gm.Hkv + h;
+    int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
+    int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
+
+    if (k <= 0) {
+        if (tid == 0) *cnt_dst = 0;
+        return;
+    }
+    if (k == ncand) {                                  // budget covers every candidate: no ranking needed
+        for (int i = tid; i < ncand; i += kThreads) idx_dst[i] = lo + i;
+        if (tid == 0) *cnt_dst = k;
+        return;
+    }
+
+    // ---- set-up -------------------------------------------------------------------------------
+    wave_stamp(0);
+    for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
+    if (tid == 0) {
+        prefetch_tmap(&tmap);
+        for (int i = 0; i < n_stages; ++i) mbar_init(&sm->full[i], 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    const int n_tiles = (ncand + kRows - 1) / kRows;
+    const long long row_base = (long long)cu * gm.max_seq_len + lo;              // row of candidate 0 in the 2-D view
+    uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 3) & ~3);     // by candidate index, 16-byte aligned
+    // The projected keys stream through L2 once; the score keys parked there must still be there when
+    // the block comes back for them.
+    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
+    // The sample row and the query are requested before the ring's first tiles: behind the whole
+    // grid's opening burst of bulk copies they would wait for microseconds.
+    const bool sampled = ncand >= kMinSampled;
+    uint4 srow[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) srow[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (sampled && tid < kSampleRows) {
+        const int slot = (int)(((long long)tid * ncand) / kSampleRows);
+        const uint4* rowp = reinterpret_cast<const uint4*>(kimp + (size_t)(row_base + slot) * RB);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
+    }
+    float qr[DP];
+    load_group_query<DP>(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
+    if (tid == 0)
+        for (int i = 0; i < n_stages && i < n_tiles; ++i) {
+            mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
+            tma_load_2d_hint(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kRows), &sm->full[i], stream_policy);
+        }
+
+    // ---- where to put the first digit's bins: a look at 256 rows spread over the problem ----------------
+    // Only the bins' resolution depends on the sample, never the result: the digit is monotone in the
+    // key whatever base and shift are, and a threshold that falls outside the sampled range lands in an
+    // open-ended bin, which sends the problem down the general path.
+    Digit dg = {0u, 21};
+    if (sampled) {
+        if (tid < kSampleRows) sm->sample[tid] = order_key(row_score<T, DP>(qr, [&](int c) { return srow[c]; }));
+        __syncthreads();
+        if (tid < kSampleRows) {   // descending rank of this thread's sample key (equal keys by index)
+            const uint32_t mine = sm->sample[tid];
+            const uint4* s4 = reinterpret_cast<const uint4*>(sm->sample);
+            int r = 0;
+#pragma unroll 8
+            for (int j4 = 0; j4 < kSampleRows / 4; ++j4) {
+                const uint4 x = s4[j4];
+                const int j = j4 * 4;
+                r += (x.x > mine) | ((x.x == mine) & (j < tid));
+                r += (x.y > mine) | ((x.y == mine) & (j + 1 < tid));
+                r += (x.z > mine) | ((x.z == mine) & (j + 2 < tid));
+                r += (x.w > mine) | ((x.w == mine) & (j + 3 < tid));
+            }
+            // about p * kSampleRows sample keys lie above the threshold (p = k / candidates); bracket it widely
+            const float p = (float)k / (float)ncand, mean = p * kSampleRows, sd = sqrtf(mean * (1.f - p));
+            const int r_hi = max(0, (int)floorf(mean - 6.f * sd) - 3), r_lo = min(kSampleRows - 1, (int)ceilf(mean + 6.f * sd) + 3);
+            if (r == r_hi) sm->s_hi = mine;
+            if (r == r_lo) sm->s_lo = mine;
+        }
+        __syncthreads();
+        const uint32_t s_lo = sm->s_lo, s_hi = sm->s_hi;
+        uint32_t range = s_hi - s_lo;
+        range += range >> 1;                           // room above the highest bracketing sample
+        if (range < s_hi - s_lo) range = 0xffffffffu;
+        dg.base = s_lo, dg.shift = 0;
+        while ((range >> dg.shift) >= 2046u) ++dg.shift;
+    }
+
+    // ---- stream + score + first digit histogram -------------------------------------------------
+    bool timed_out = false;
+    int st = 0;
+    uint32_t phase = 0;
+    for (int i = 0; i < n_tiles; ++i) {
+        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;   // keep going: control flow stays uniform
+        const unsigned char* tile = stage_base + st * kTileBytes;
+        const int slot = i * kRows + tid;
+        if (i == 0) wave_stamp(1);
+        if (slot < ncand) {
+            const uint32_t off = tid * RB;
+            const float sc = row_score<T, DP>(qr, [&](int c) {
+                uint32_t o = off + c * 16;
+                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
+                return *reinterpret_cast<const uint4*>(tile + o);
+            });
+            const uint32_t key = order_key(sc);
+            st_global_hint(keys_unit + slot, key, keep_policy);
+            hist_add(&hist[dg.bin(key)]);
+        }
+        __syncthreads();                               // all reads of this stage are done
+        if (tid == 0 && i + n_stages < n_tiles) {
+            fence_proxy_async();
+            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+            tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kRows), &sm->full[st],
+                             stream_policy);
+        }
+        if (++st == n_stages) st = 0, phase ^= 1u;
+    }
+    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    __syncthreads();                                   // histogram complete, own keys visible to the block
+    wave_stamp(2);
+
+    // ---- finish -----------------------------------------------------------------------------------
+    if (wave_finish_mask(hist, sm, dg, keys_unit, stage_base, n_stages * (int)kTileBytes, ncand, k, lo, idx_dst, cnt_dst)) {
+        wave_stamp(3);
+        return;
+    }
+    // general path: exact radix select over all of the problem's keys
+    const uint4* keys4 = reinterpret_cast<const uint4*>(keys_unit);
+    const int n_vec = (ncand + 3) / 4;
+    bool cached = false;                               // key_cache holds vectors [0, min(n_vec, cache_vecs))
+    // One pass over all key vectors, kBatch loads in flight per thread; the first pass leaves the keys
+    // in the ring.  f(v, x): vector index and its four keys (slots 4v .. 4v+3; slots >= ncand are stale).
+    auto scan = [&](auto&& f) {
+        for (int v0 = tid; v0 < n_vec; v0 += kThreads * kBatch) {
+            uint4 x[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int v = v0 + u * kThreads;
+                x[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (v < n_vec) x[u] = (cached && v < cache_vecs) ? key_cache[v] : __ldcg(keys4 + v);
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int v = v0 + u * kThreads;
+                if (v < n_vec) {
+                    if (!cached && v < cache_vecs) key_cache[v] = x[u];
+                    f(v, x[u]);
+                }
+            }
+        }
+        __syncthreads();
+        cached = true;
+    };
+
+    uint32_t prefix = 0;                               // digits fixed so far (value of key >> low_bits)
+    int low_bits = 32, krem = k;
+    bool exact = false;                                // the class {key >> low_bits == prefix} is taken whole
+#pragma unroll 1
+    for (int pass = 0; pass < 3 && !exact; ++pass) {   // 11 + 11 + 10 bits of the key itself
+        const int bits = pass == 2 ? 10 : 11, shift = low_bits - bits;
+        const uint32_t dmask = (1u << bits) - 1u;
+        for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
+        __syncthreads();
+        scan([&](int v, const uint4& x) {
+            const uint32_t kk[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (v * 4 + e < ncand && (pass == 0 || (kk[e] >> low_bits) == prefix)) hist_add(&hist[(kk[e] >> shift) & dmask]);
+        });
+        int d, kr, c;
+        if (pass < 2) wave_find_digit<8>(hist, krem, sm, d, kr, c);
+        else wave_find_digit<4>(hist, krem, sm, d, kr, c);
+        prefix = (prefix << bits) | (uint32_t)d, low_bits = shift, krem = kr, exact = c == kr;
+    }
+
+    // ---- ordered compaction ------------------------------------------------------------------------
+    // A slot is taken if its key is above the class, or inside the class and among the class's first
+    // `krem` members in position order (the lower-position tie rule).  Warp w owns a contiguous range;
+    // within a group of 128 slots lane l holds slots 4l..4l+3 (one 16-byte load), so lane order is
+    // position order.
+    const int seg = ((ncand + kWarps * 128 - 1) / (kWarps * 128)) * 128;          // slots per warp, multiple of 128
+    const int seg_begin = min(ncand, warp * seg), seg_end = min(ncand, (warp + 1) * seg);
+    auto classify = [&](int base, int& gt_bits, int& eq_bits) {   // bit e: slot base+e above / in the class
+        gt_bits = eq_bits = 0;
+        if (base < seg_end) {
+            const int v = base >> 2;
+            const uint4 x = v < cache_vecs ? key_cache[v] : __ldcg(keys4 + v);
+            const uint32_t c[4] = {x.x >> low_bits, x.y >> low_bits, x.z >> low_bits, x.w >> low_bits};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool in = base + e < seg_end;
+                gt_bits |= (in && c[e] > prefix) << e;
+                eq_bits |= (in && c[e] == prefix) << e;
+            }
+        }
+    };
+    int n_gt = 0, n_eq = 0;
+#pragma unroll 2
+    for (int i0 = seg_begin; i0 < seg_end; i0 += 128) {
+        int gb, eb;
+        classify(i0 + 4 * lane, gb, eb);
+        n_gt += __popc(gb), n_eq += __popc(eb);
+    }
+    n_gt = warp_sum_int(n_gt);
+    n_eq = warp_sum_int(n_eq);
+    if (lane == 0) sm->warp_a[warp] = n_gt, sm->warp_b[warp] = n_eq;
+    __syncthreads();
+    int gt_before = 0, eq_before = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        const int x = sm->warp_a[w], y = sm->warp_b[w];
+        gt_before += w < warp ? x : 0, eq_before += w < warp ? y : 0;
+    }
+    int out_pos = gt_before + min(eq_before, krem);
+#pragma unroll 2
+    for (int i0 = seg_begin; i0 < seg_end; i0 += 128) {
+        const int base = i0 + 4 * lane;
+        int gb, eb;
+        classify(base, gb, eb);
+        int take = gb;
+        if (__any_sync(0xffffffffu, eb != 0)) {        // class members here: hand out what is left of the quota in order
+            const int ne = __popc(eb);
+            int before = eq_before + warp_incl_scan(ne, lane) - ne;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if ((eb >> e) & 1) {
+                    if (before < krem) take |= 1 << e;
+                    ++before;
+                }
+            eq_before += warp_sum_int(ne);
+        }
+        const int nt = __popc(take);
+        if (__any_sync(0xffffffffu, nt != 0)) {
+            const int incl = warp_incl_scan(nt, lane);
+            int o = out_pos + incl - nt;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if ((take >> e) & 1) idx_dst[o++] = lo + base + e;
+            out_pos += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+    if (tid == 0) *cnt_dst = k;
+    wave_stamp(3);
+}
+
+#ifdef TB_PHASE_TIMING
+extern "C" int tb_debug_fin_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_fin_ns, sizeof(g_fin_ns)); }
+extern "C" int tb_debug_wave_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_wave_ns, sizeof(g_wave_ns)); }
+#endif
+
+cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
+    const Geom& gm = c->geom;
+    const int n_pairs = ut.layer_count * ut.n_seq, n_units = n_pairs * gm.Hkv;
+    WaveOrder order;
+    int cand[kMaxLaunchUnits];
+    for (int i = 0; i < n_pairs; ++i) {
+        const int L = ut.len[i], lo = a.sinks < L ? a.sinks : L, hi = L - a.recent > lo ? L - a.recent : lo;
+        cand[i] = hi - lo, order.pair[i] = (uint16_t)i;
+    }
+    std::stable_sort(order.pair, order.pair + n_pairs, [&](uint16_t x, uint16_t y) { return cand[x] > cand[y]; });
+    const int tile_bytes = kRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
+    int n_stages = kRingBytes / tile_bytes;            // 32 KB of ring: four blocks per SM keep 128 KB in flight
+    if (n_stages > kStagesMax) n_stages = kStagesMax;
+    if (n_stages < 2) n_stages = 2;
+    const size_t smem = 1024 + (size_t)n_stages * tile_bytes + kDigitBins * sizeof(int) + sizeof(WaveSmem);
+
+#define TB_SEL(T, DP)                                                                                                   \
+    do {                                                                                                                \
+        static unsigned char seen[64];                                                                                  \
+        if (first_use_on_this_device(seen)) {                                                                           \
+            cudaError_t e = cudaFuncSetAttribute(select_wave_kernel<T, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                 80 * 1024);                                                            \
+            if (e != cudaSuccess) return e;                                                                             \
+        }                                                                                                               \
+        select_wave_kernel<T, DP><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, c->st.idx, c->st.cnt, \
+                                                                  c->st.status, c->wk.sel_keys);                        \
+        return cudaGetLastError();                                                                                      \
+    } while (0)
+    if (gm.dtype == TB_BF16) {
+        if (gm.dp == 32) TB_SEL(__nv_bfloat16, 32); else TB_SEL(__nv_bfloat16, 16);
+    } else {
+        if (gm.dp == 32) TB_SEL(float, 32); else TB_SEL(float, 16);
+    }
+#undef TB_SEL
+}
+
+}  // namespace tb

@@ -348,3 +348,73 @@ def test_cluster_selection_unusual_distributions(H):
     v = np.zeros((2, L), np.float32)
     v[:, ::7] = 4.0
     _crafted_scores_case(H, v, budget=int((v[0] == 4.0).sum()))
+
+
+def _crafted_batch_case(H, scores, budget, sinks=0, recent=0):
+    """Many problems in one launch (scores[seq, head, position], equal lengths): K_imp rows are
+    score * e_0 and the importance query is e_0, so the importance scores are exactly `scores`."""
+    n_seq, n_heads, L = scores.shape
+    w = wl.workload(2, n_layers=1, n_q_heads=n_heads, n_kv_heads=n_heads, batch=n_seq, lengths=[L] * n_seq, budget=budget,
+                    sinks=sinks, recent=recent)
+    case = H.Case(w, project="oracle-only")
+    for b in range(n_seq):
+        for h in range(n_heads):
+            kimp = np.zeros((L, w.imp_dim), np.float32)
+            kimp[:, 0] = scores[b, h]
+            bits = wl.to_storage(kimp, w.dtype)
+            assert np.array_equal(wl.storage_to_f32(bits, w.dtype)[:, 0], scores[b, h]), "scores must be bf16-exact"
+            case.Kimp[0][b][h, :L] = bits
+            case.ctx.kimp[0, b, h, :L] = H.to_dev(bits, w.dtype)
+    qi = np.zeros((1, n_seq, n_heads, w.imp_dim), np.float32)
+    qi[..., 0] = 1.0
+    p = tb().select_params(budget, sinks, recent)
+    lists = H.gpu_select(case, qi, p)
+    assert case.ctx.get_status() == 0
+    for b in range(n_seq):
+        for h in range(n_heads):
+            _, full, _ = case.oracle_select(0, b, h, qi[0, b], p)
+            assert np.array_equal(lists[0][b][h], full), "seq %d head %d" % (b, h)   # exact scores: no tolerance
+    return lists
+
+
+def _bf16_exact(x):
+    return wl.storage_to_f32(wl.to_storage(x.astype(np.float32), wl.BF16), wl.BF16)
+
+
+def test_many_problem_selection_kernel(H):
+    """Launches with hundreds of problems take the one-block-per-problem kernel (40 sequences x 8 heads
+    here).  Its first digit is placed from a sample of each problem's scores; these cases put the
+    threshold in every kind of bin that digit has, and on the general path behind it."""
+    r = np.random.Generator(np.random.PCG64(78))
+    n_seq, n_heads = 40, 8
+    # ordinary data, long enough to be sampled, ending mid-tile; and too short to be sampled
+    _crafted_batch_case(H, _bf16_exact(r.standard_normal((n_seq, n_heads, 5003))), budget=400, sinks=2, recent=31)
+    _crafted_batch_case(H, _bf16_exact(r.standard_normal((n_seq, n_heads, 1501))), budget=100)
+    # every score equal, and a few distinct values: the threshold bin is one crowded class of ties
+    _crafted_batch_case(H, np.full((n_seq, n_heads, 3001), 1.5, np.float32), budget=200, sinks=1, recent=3)
+    _crafted_batch_case(H, r.integers(0, 5, size=(n_seq, n_heads, 4099)).astype(np.float32), budget=1000)
+    # a handful of huge scores at positions the sample does not see, budget below their number: the
+    # threshold lies in the open-ended top bin
+    L = 4096
+    s = _bf16_exact(r.standard_normal((n_seq, n_heads, L)))
+    s[:, :, 7::509] = _bf16_exact(1000.0 + 8.0 * r.integers(0, 64, size=s[:, :, 7::509].shape))
+    _crafted_batch_case(H, s, budget=5)
+    # the sampled positions (every 64th of the candidates) hold large scores, everything else small
+    # ones, and the budget reaches deep into the small ones: the threshold lies below the sampled range
+    s = _bf16_exact(0.01 * r.standard_normal((n_seq, n_heads, L)))
+    s[:, :, ::64] = _bf16_exact(50.0 + r.standard_normal((n_seq, n_heads, L // 64)))
+    _crafted_batch_case(H, s, budget=2000)
+    # scores over ~400 binades and both signs
+    expo = r.integers(-100, 101, size=(n_seq, n_heads, 3000))
+    sign = r.choice([-1.0, 1.0], size=expo.shape)
+    _crafted_batch_case(H, (sign * np.exp2(expo)).astype(np.float32), budget=700)
+    # budget covers every candidate; no candidates at all
+    _crafted_batch_case(H, _bf16_exact(r.standard_normal((n_seq, n_heads, 600))), budget=600)
+    _crafted_batch_case(H, _bf16_exact(r.standard_normal((n_seq, n_heads, 300))), budget=10, sinks=100, recent=200)
+
+
+def test_selection_beyond_cluster_capacity(H):
+    """A single problem with more candidates than a cluster keeps on chip (8 x 32768) goes to the
+    one-block-per-problem kernel, whose bitmask does not fit its scratch either: the general path."""
+    r = np.random.Generator(np.random.PCG64(79))
+    _crafted_scores_case(H, _bf16_exact(r.standard_normal((1, 270001))), budget=5000, sinks=4, recent=64)

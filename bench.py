@@ -311,6 +311,11 @@ def run_ours(args, w):
         ms_e2e = timed(e2e_step, args.steps, args.warmup)
         ms_sel = timed(g_sel.replay, max(20, args.steps // 4), 3) / len(groups)
         ms_att = timed(g_att.replay, max(20, args.steps // 4), 3) / w.n_layers
+        # Upper bound, not the method's schedule: the importance queries of all layers at once, so the
+        # selection runs as one call over every layer (many problems per launch) before the attentions.
+        g_all = capture(lambda: (ctx.select_topk(0, w.n_layers, None, w.batch, qi, p),
+                                 [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)]))
+        ms_all = timed(g_all.replay, max(20, args.steps // 4), 3)
         assert ctx.get_status(stream) == 0, "device status set during the timed region"
 
     peak, peak_kind = measured_peaks()
@@ -342,6 +347,10 @@ def run_ours(args, w):
                                       "gbs": sel_b / (ms_sel * 1e-3) / 1e9, "launches_per_step": len(groups)},
                     "attn_kernel": {"us_per_launch": ms_att * 1e3, "bytes_per_launch": att_b,
                                     "gbs": att_b / (ms_att * 1e-3) / 1e9, "launches_per_step": w.n_layers}},
+        "upper_bound_all_layers_one_select_call": {"us_per_step": ms_all * 1e3,
+                                                    "step_frac_of_peak": step_bytes / (ms_all * 1e-3) / 1e9 / peak,
+                                                    "note": "selection for all layers in one call; needs every layer's importance "
+                                                            "query up front, which the per-producer schedule does not have"},
         "prefill_projection": proj_info,
         "clocks": sampler.summary(),
     }

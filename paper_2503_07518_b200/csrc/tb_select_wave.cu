@@ -37,7 +37,6 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kRows = 256;          // rows per TMA box = one row per thread
 constexpr int kStagesMax = 8;
-constexpr int kRingBytes = 32 * 1024;
 constexpr int kDigitBins = 2048;    // 11-bit digits (the last digit has 10 bits)
 constexpr int kSampleRows = 64;     // rows scored up front to place the first digit's bins
 constexpr int kMinSampled = 2048;   // smaller problems use the key's top bits as first digit
@@ -599,17 +598,22 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
     }
     std::stable_sort(order.pair, order.pair + n_pairs, [&](uint16_t x, uint16_t y) { return cand[x] > cand[y]; });
     const int tile_bytes = kRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
-    int n_stages = kRingBytes / tile_bytes;            // 32 KB of ring: four blocks per SM keep 128 KB in flight
+    // Ring depth: the SM's shared memory split among the blocks it will hold (four when the launch has
+    // that many per SM: 32 KB rings, 128 KB in flight; fewer blocks get deeper rings).
+    const size_t fixed = 1024 + kDigitBins * sizeof(int) + sizeof(WaveSmem);
+    int per_sm = (n_units + c->sm_count - 1) / c->sm_count;
+    per_sm = per_sm < 1 ? 1 : per_sm > 4 ? 4 : per_sm;
+    int n_stages = (int)(((size_t)224 * 1024 / per_sm - 1024 - fixed) / tile_bytes);
     if (n_stages > kStagesMax) n_stages = kStagesMax;
     if (n_stages < 2) n_stages = 2;
-    const size_t smem = 1024 + (size_t)n_stages * tile_bytes + kDigitBins * sizeof(int) + sizeof(WaveSmem);
+    const size_t smem = fixed + (size_t)n_stages * tile_bytes;
 
 #define TB_SEL(T, DP)                                                                                                   \
     do {                                                                                                                \
         static unsigned char seen[64];                                                                                  \
         if (first_use_on_this_device(seen)) {                                                                           \
             cudaError_t e = cudaFuncSetAttribute(select_wave_kernel<T, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                                 80 * 1024);                                                            \
+                                                 200 * 1024);                                                            \
             if (e != cudaSuccess) return e;                                                                             \
         }                                                                                                               \
         select_wave_kernel<T, DP><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, c->st.idx, c->st.cnt, \

@@ -36,6 +36,7 @@ UNIT = "tokens/s"
 NCU_TRAFFIC_BYTES = {
     ("cfg2_llama8b_32k", "select_kernel"): 67_197_184 + 755_200,   # profiles/select_kernel_cfg2_32k.md
     ("cfg2_llama8b_32k", "attn_kernel"): 13_575_936,               # profiles/attn_mma_kernel_cfg2_32k.md
+    ("cfg3_batched_serving", "select_kernel"): 398_913_792 + 4_822_528,   # profiles/select_wave_kernel_cfg3_batched.md
 }
 
 

@@ -346,6 +346,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     // predecessor; otherwise only before the queries are read, so that the row map, the list fetch
     // and the first gathers overlap the predecessor's tail.
     if (!a.early_ok) pdl_wait();
+    pdl_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gid = lane >> 2, tig = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y;
@@ -421,7 +422,6 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     attn_stamp(2);
 
     if (a.early_ok) pdl_wait();                        // the queries are this call's input
-    pdl_launch_dependents();
     // Q^T as the B operand of S = K Q^T: k = channels, n = query heads (gid; heads >= g are zero padding)
     uint32_t qb[8][2];
     {
@@ -689,6 +689,14 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
 #ifdef TB_FORCE_ATTN_CLUSTER
         n = TB_FORCE_ATTN_CLUSTER;
 #else
+        // First choice: a launch that takes at most half of the SMs, so that the next layer's blocks
+        // (programmatic dependent launch) can fetch their lists and first rows on free SMs while this
+        // layer still computes (config 2, 8 problems: clusters of 9 run at 7.36 us per layer, the largest
+        // that fits, 10, at 7.86, 8 at 8.65).  Otherwise the largest cluster that fits once.
+        {
+            const int cand = c->sm_count / (2 * units);
+            if (cand >= 6 && cand <= 16 && cand <= by_rows && clusters_that_fit(cand) >= units) n = cand;
+        }
         for (int cand = 16; cand >= 1 && !n; cand = cand > 8 ? cand - 2 : cand - 1)
             if (cand <= by_rows && units * cand <= c->sm_count && (cand <= 8 || clusters_that_fit(cand) >= units)) n = cand;
 #endif

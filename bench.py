@@ -34,8 +34,8 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
-    ("cfg2_llama8b_32k", "select_kernel"): 67_197_184 + 755_200,   # profiles/select_kernel_cfg2_32k.md
-    ("cfg2_llama8b_32k", "attn_kernel"): 13_575_936,               # profiles/attn_mma_kernel_cfg2_32k.md
+    ("cfg2_llama8b_32k", "select_kernel"): 67_198_720 + 815_872,   # profiles/select_kernel_cfg2_32k.md
+    ("cfg2_llama8b_32k", "attn_kernel"): 13_579_264,               # profiles/attn_mma_kernel_cfg2_32k.md
     ("cfg3_batched_serving", "select_kernel"): 398_913_792 + 4_822_528,   # profiles/select_wave_kernel_cfg3_batched.md
 }
 

@@ -101,8 +101,11 @@ __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
 // attribute may start while its predecessor in the stream still runs.  pdl_wait() blocks until the
 // predecessor has completed and its writes are visible (a no-op for ordinary launches);
 // pdl_launch_dependents() lets the successor begin.  Every kernel here waits before it touches
-// anything its predecessor may have produced and before its own global writes, and only then
-// releases its successor, so completion stays transitive along the stream.
+// anything its predecessor may have produced and before its own global writes; a successor's wait
+// ends only when this kernel has completed, which it cannot before its own wait has, so completion
+// stays transitive along the stream.  A kernel whose predecessor wrote what its prologue reads waits
+// first and releases afterwards; the others release at once, and by induction everything older than
+// their predecessor had already completed when they started.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

@@ -488,6 +488,15 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     }
     phase_stamp(6);
     int out_pos = gt_before + min(eq_before, krem);
+    const uint32_t lt = (1u << lane) - 1u;
+    // Exclusive prefix over the warp of a per-lane count 0..4, and the warp total, from three ballots
+    // (one per bit of the count) instead of a five-step chain of dependent shuffles.
+    auto warp_prefix_small = [&](int n, int& total) {
+        const uint32_t b0 = __ballot_sync(0xffffffffu, n & 1), b1 = __ballot_sync(0xffffffffu, n & 2),
+                       b2 = __ballot_sync(0xffffffffu, n & 4);
+        total = __popc(b0) + 2 * __popc(b1) + 4 * __popc(b2);
+        return __popc(b0 & lt) + 2 * __popc(b1 & lt) + 4 * __popc(b2 & lt);
+    };
 #pragma unroll 2
     for (int i0 = seg_begin; i0 < seg_end; i0 += 128) {
         const int base = i0 + 4 * lane;
@@ -495,24 +504,23 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         classify(base, gb, eb);
         int take = gb;
         if (__any_sync(0xffffffffu, eb != 0)) {        // class members here: hand out what is left of the quota in order
-            const int ne = __popc(eb);
-            int before = eq_before + warp_incl_scan(ne, lane) - ne;
+            int ne_warp;
+            int before = eq_before + warp_prefix_small(__popc(eb), ne_warp);
 #pragma unroll
             for (int e = 0; e < 4; ++e)
                 if ((eb >> e) & 1) {
                     if (before < krem) take |= 1 << e;
                     ++before;
                 }
-            eq_before += warp_sum_int(ne);
+            eq_before += ne_warp;
         }
-        const int nt = __popc(take);
-        if (__any_sync(0xffffffffu, nt != 0)) {
-            const int incl = warp_incl_scan(nt, lane);
-            int o = out_pos + incl - nt;
+        if (__any_sync(0xffffffffu, take != 0)) {
+            int nt_warp;
+            int o = out_pos + warp_prefix_small(__popc(take), nt_warp);
 #pragma unroll
             for (int e = 0; e < 4; ++e)
                 if ((take >> e) & 1) idx_dst[o++] = tok0 + base + e;
-            out_pos += __shfl_sync(0xffffffffu, incl, 31);
+            out_pos += nt_warp;
         }
     }
     if (rank == 0 && tid == 0) *cnt_dst = k;

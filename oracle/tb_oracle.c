@@ -20,6 +20,9 @@
  *   orc_attended_set   Sink | Important | Local-Window      Sec. 3.3 (three buffers)
  *   orc_attention      softmax(q K^T / sqrt(D)) V           Sec. 3.3 ("standard attention kernel")
  *   orc_step_units     the steps above chained per unit     Sec. 3.3 / 3.4
+ *   orc_predict_queries  Q_imp = f(LN(H)), two-layer MLP    Sec. 3.1 "Query prediction", App. A (hidden
+ *                                                           size 512), Table 6 (bias-free linears, LN
+ *                                                           with weight and bias)
  *
  * Parity pins live in tests/test_oracle_pins.py.  The placement rule of the CLUSTER neighbour
  * mode (which side of a run the extra positions go to) is a reading of one sentence of Sec. 3.4:
@@ -320,6 +323,45 @@ void orc_step_units(orc_unit* units, int n_units, const orc_params* p, int n_thr
         orc_attention(un->q, un->K, un->V, A, nA, p->g, p->D, p->dtype, p->sm_scale, un->out, un->lse);
         free(A);
     }
+}
+
+/* ---------- importance-query predictor (Sec. 3.1 "Query prediction", App. A) --------------------
+ * For each token: x = LN(h) (mean and biased variance over the E channels, eps inside the root,
+ * weight and bias), u = act(W1 x), q = W2 u.  Linears have no bias (the parameter counts of Table 6
+ * leave no room for one).  The paper does not name the activation: act 0 = GELU in its exact erf
+ * form (this build's reading), 1 = SiLU, 2 = ReLU.  W1 is [hid][E], W2 is [out][hid], both row-major
+ * (one row per output), out = slots * heads * d'.  Everything in fp64 on values the caller widened. */
+enum { ORC_ACT_GELU = 0, ORC_ACT_SILU = 1, ORC_ACT_RELU = 2 };
+
+void orc_predict_queries(const double* H, int n_tok, int E, const double* ln_w, const double* ln_b, double eps,
+                         const double* W1, int hid, const double* W2, int out, int act, double* q) {
+    double* x = (double*)malloc(sizeof(double) * (size_t)E);
+    double* u = (double*)malloc(sizeof(double) * (size_t)hid);
+    for (int t = 0; t < n_tok; ++t) {
+        const double* h = H + (size_t)t * E;
+        double mean = 0.0, var = 0.0;
+        for (int c = 0; c < E; ++c) mean += h[c];
+        mean /= E;
+        for (int c = 0; c < E; ++c) var += (h[c] - mean) * (h[c] - mean);
+        var /= E;
+        const double rstd = 1.0 / sqrt(var + eps);
+        for (int c = 0; c < E; ++c) x[c] = (h[c] - mean) * rstd * ln_w[c] + ln_b[c];
+        for (int j = 0; j < hid; ++j) {
+            double a = 0.0;
+            for (int c = 0; c < E; ++c) a += W1[(size_t)j * E + c] * x[c];
+            if (act == ORC_ACT_GELU) a = 0.5 * a * (1.0 + erf(a / sqrt(2.0)));
+            else if (act == ORC_ACT_SILU) a = a / (1.0 + exp(-a));
+            else a = a > 0.0 ? a : 0.0;
+            u[j] = a;
+        }
+        for (int o = 0; o < out; ++o) {
+            double a = 0.0;
+            for (int j = 0; j < hid; ++j) a += W2[(size_t)o * hid + j] * u[j];
+            q[(size_t)t * out + o] = a;
+        }
+    }
+    free(x);
+    free(u);
 }
 
 int orc_max_threads(void) {

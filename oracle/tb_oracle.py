@@ -200,5 +200,22 @@ def step_units(units, Ls, q_imps, qs, refresh, *, g, D, dp, dtype, budget, sinks
     return (out, lse) if want_lse else out
 
 
+ACT_GELU, ACT_SILU, ACT_RELU = 0, 1, 2
+
+
+def predict_queries(H: np.ndarray, ln_w: np.ndarray, ln_b: np.ndarray, W1: np.ndarray, W2: np.ndarray, dtype: int,
+                    eps: float = 1e-5, act: int = ACT_GELU) -> np.ndarray:
+    """Importance queries of the predictor (Sec. 3.1 "Query prediction", App. A): q = W2 act(W1 LN(h)) per
+    token.  All inputs are stored values (``dtype``): H [tokens, E], ln_w / ln_b [E], W1 [hidden, E],
+    W2 [out, hidden]; returns float64 [tokens, out]."""
+    H, ln_w, ln_b, W1, W2 = (widen(_chk(a, dtype), dtype) for a in (H, ln_w, ln_b, W1, W2))
+    n_tok, E = H.shape
+    hid, out = W1.shape[0], W2.shape[0]
+    assert W1.shape == (hid, E) and W2.shape == (out, hid) and ln_w.shape == (E,) and ln_b.shape == (E,)
+    q = np.empty((n_tok, out), np.float64)
+    lib().orc_predict_queries(_p(H), n_tok, E, _p(ln_w), _p(ln_b), C.c_double(eps), _p(W1), hid, _p(W2), out, act, _p(q))
+    return q
+
+
 def max_threads() -> int:
     return lib().orc_max_threads()

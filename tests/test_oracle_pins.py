@@ -364,3 +364,58 @@ def test_planted_tokens_are_all_recalled(orc):
     I = orc.select(s, w.sinks, w.recent, w.budget)
     assert len(I) == w.budget
     assert set(pos[0]) <= set(I)
+
+
+# ------------------------------------------------------------------ importance-query predictor (Sec. 3.1, App. A)
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_predictor_is_layernorm_then_two_float64_matmuls(orc, dtype, act):
+    """q = W2 act(W1 LN(h)): every stage against numpy / math library routines in float64, with a
+    layer norm that has both weight and bias and linears without bias (Table 6)."""
+    import math
+    r = rng(310 + act)
+    n_tok, E, hid, heads, slots, dp = 3, 96, 40, 4, 2, 8
+    out = slots * heads * dp
+    H = rand_storage(r, (n_tok, E), dtype, 2.0)
+    H[1] = wl.to_storage((wl.storage_to_f32(H[1], dtype) + 7.0).astype(np.float32), dtype)    # a token with a large mean
+    ln_w, ln_b = rand_storage(r, (E,), dtype), rand_storage(r, (E,), dtype, 0.3)
+    W1, W2 = rand_storage(r, (hid, E), dtype, E ** -0.5), rand_storage(r, (out, hid), dtype, hid ** -0.5)
+    q = orc.predict_queries(H, ln_w, ln_b, W1, W2, dtype, eps=1e-5, act=act)
+    h = f64(H, dtype)
+    x = (h - h.mean(axis=1, keepdims=True)) / np.sqrt(h.var(axis=1, keepdims=True) + 1e-5) * f64(ln_w, dtype) + f64(ln_b, dtype)
+    pre = x @ f64(W1, dtype).T
+    if act == 0:
+        u = np.array([[0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))) for v in row] for row in pre])
+    elif act == 1:
+        u = pre / (1.0 + np.exp(-pre))
+    else:
+        u = np.maximum(pre, 0.0)
+    ref = u @ f64(W2, dtype).T
+    assert q.shape == (n_tok, out)
+    assert np.allclose(q, ref, rtol=1e-12, atol=1e-12)
+
+
+def test_predictor_closed_forms(orc):
+    """Special cases with known answers: a constant hidden state normalises to the LN bias alone; GELU
+    at 0, +1, -1 (0, Phi(1), -Phi(-1)); identity-like weights pass the normalised input through."""
+    E = 8
+    one = np.ones((1, E), np.float32)
+    eye = np.eye(E, dtype=np.float32)
+    # constant token: (h - mean) = 0, so x = ln_b whatever ln_w is; ReLU and identity weights return it
+    b = np.linspace(0.5, 4.0, E).astype(np.float32)
+    q = orc.predict_queries(3.25 * one, 9.0 * one[0], b, eye, eye, F32, act=2)
+    assert np.allclose(q[0], b, rtol=0, atol=1e-12)
+    # h = (+1, -1, +1, -1, ...): mean 0, variance 1, so x = h / sqrt(1 + eps); GELU(x) by its closed form
+    h = np.tile(np.array([1.0, -1.0], np.float32), E // 2)[None]
+    q = orc.predict_queries(h, one[0], 0 * one[0], eye, eye, F32, eps=0.0, act=0)
+    assert np.allclose(q[0, 0], 0.8413447460685429, atol=1e-12) and np.allclose(q[0, 1], -0.15865525393145707, atol=1e-12)
+    q = orc.predict_queries(h, one[0], 0 * one[0], eye, eye, F32, eps=0.0, act=1)
+    assert np.allclose(q[0, 0], 1.0 / (1.0 + np.exp(-1.0)), atol=1e-12) and np.allclose(q[0, 1], -1.0 / (1.0 + np.exp(1.0)), atol=1e-12)
+    # scale invariance of the layer norm (eps = 0): 5 h gives the same queries as h
+    r = rng(311)
+    H = r.standard_normal((2, E)).astype(np.float32)
+    W1, W2 = r.standard_normal((6, E)).astype(np.float32), r.standard_normal((4, 6)).astype(np.float32)
+    qa = orc.predict_queries(H, one[0], b, W1, W2, F32, eps=0.0)
+    qb = orc.predict_queries((4.0 * H).astype(np.float32), one[0], b, W1, W2, F32, eps=0.0)   # 4 h is exact in fp32
+    assert np.allclose(qa, qb, rtol=1e-12, atol=1e-12)

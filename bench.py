@@ -317,6 +317,21 @@ def run_ours(args, w):
         g_all = capture(lambda: (ctx.select_topk(0, w.n_layers, None, w.batch, qi, p),
                                  [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)]))
         ms_all = timed(g_all.replay, max(20, args.steps // 4), 3)
+        # The step before the path, reported beside it (not inside the timed step): the importance-query
+        # predictor of one producer layer, 8B-shaped (model dim 4096, hidden 512), random weights; 16 weight
+        # sets are cycled so that every call reads its 8 MB from HBM, not from L2.
+        E, HID, n_sets = 4096, 512, 16
+        n_out = GROUP_LAYERS * w.n_q_heads * w.imp_dim
+        pw = [(torch.randn(E, generator=gen, device="cuda").to(dt), torch.randn(E, generator=gen, device="cuda").to(dt),
+               (torch.randn(HID, E, generator=gen, device="cuda") * E ** -0.5).to(dt),
+               (torch.randn(n_out, HID, generator=gen, device="cuda") * HID ** -0.5).to(dt)) for _ in range(n_sets)]
+        hs = torch.randn(w.batch, E, generator=gen, device="cuda").to(dt)
+        p_scratch = torch.empty(w.batch * HID, device="cuda")
+        p_out = torch.empty(GROUP_LAYERS, w.batch, w.n_q_heads, w.imp_dim, device="cuda")
+        g_pred = capture(lambda: [tbh.predict_importance_queries(hs, a, b, w1, w2, w.dtype, w.n_q_heads, GROUP_LAYERS, w.imp_dim,
+                                                                 p_scratch, p_out, stream=stream) for (a, b, w1, w2) in pw])
+        ms_pred = timed(g_pred.replay, 20, 3) / n_sets
+        pred_bytes = (HID * E + n_out * HID + 2 * E + w.batch * E) * (2 if w.dtype == wl.BF16 else 4)
         assert ctx.get_status(stream) == 0, "device status set during the timed region"
 
     peak, peak_kind = measured_peaks()
@@ -352,6 +367,10 @@ def run_ours(args, w):
                                                     "step_frac_of_peak": step_bytes / (ms_all * 1e-3) / 1e9 / peak,
                                                     "note": "selection for all layers in one call; needs every layer's importance "
                                                             "query up front, which the per-producer schedule does not have"},
+        "predictor_forward": {"us_per_producer": ms_pred * 1e3, "bytes_per_producer": pred_bytes,
+                              "gbs": pred_bytes / (ms_pred * 1e-3) / 1e9, "producers_per_step": len(groups),
+                              "note": "importance-query MLP of one producer layer (two launches); the step before the path, "
+                                      "not part of the timed step"},
         "prefill_projection": proj_info,
         "clocks": sampler.summary(),
     }

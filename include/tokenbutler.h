@@ -192,6 +192,37 @@ tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32_t kv_dtype
                                             int32_t sinks, int32_t recent, float sm_scale, float* out_dev,
                                             float* lse_dev, void* stream);
 
+/* Importance-query predictor forward (paper Sec. 3.1 "Query prediction"; App. A: a two-layer MLP with
+ * hidden size 512 at every producer layer; Table 6's parameter counts fix bias-free linears and a layer
+ * norm with weight and bias).  For each of n_tokens hidden states h [model_dim] (one per decoding
+ * sequence):   q = W2 . act(W1 . LN(h)),   LN over the model_dim channels with biased variance and
+ * ln_eps inside the root.  The paper does not name the activation; TB_ACT_GELU (exact erf form) is this
+ * library's reading, SiLU and ReLU are offered.  It is the step right before tb_select_topk: the output
+ *   q_imp_dev [n_slots][n_tokens][n_q_heads][imp_dim] fp32
+ * is laid out so that the n_slots consumer layers of a producer can be selected with one
+ * tb_select_topk(layer_begin = first consumer, layer_count = n_slots, q_imp_dev).
+ *   hidden_dev   [n_tokens][model_dim] in `dtype`
+ *   ln_weight, ln_bias [model_dim]; w1 [hidden_dim][model_dim]; w2 [n_slots][n_q_heads][imp_dim][hidden_dim],
+ *                row-major (one row per output), all in `dtype`, device memory owned by the caller
+ *   scratch_dev  n_tokens * hidden_dim floats of device memory (contents undefined afterwards)
+ * All device pointers 16-byte aligned; model_dim and hidden_dim multiples of 8 (bf16) or 4 (fp32) and
+ * hidden_dim <= 1536, else TB_ERR_UNSUPPORTED; n_tokens <= 64, else TB_ERR_CAPACITY.  Needs no tb_ctx, keeps no pointer, enqueues two
+ * kernels on `stream` and returns. */
+typedef enum { TB_ACT_GELU = 0, TB_ACT_SILU = 1, TB_ACT_RELU = 2 } tb_activation;
+typedef struct {
+    int32_t dtype;                        /* tb_dtype of the hidden states and of every weight */
+    int32_t model_dim, hidden_dim;
+    int32_t n_q_heads, n_slots, imp_dim;  /* outputs per token = n_slots * n_q_heads * imp_dim */
+    int32_t activation;                   /* tb_activation */
+    float ln_eps;
+    const void* ln_weight;
+    const void* ln_bias;
+    const void* w1;
+    const void* w2;
+} tb_predictor;
+tb_status tb_predict_importance_queries(const tb_predictor* p, const void* hidden_dev, int32_t n_tokens,
+                                        float* scratch_dev, float* q_imp_dev, void* stream);
+
 /* Synchronise `stream`, return the device status word (TB_OK, TB_ERR_TIMEOUT or TB_ERR_BAD_INDEX)
  * in *device_status and clear it. */
 tb_status tb_get_status(tb_ctx* ctx, void* stream, int32_t* device_status);

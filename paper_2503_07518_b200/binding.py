@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libtokenbutler.so")
 
 EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb_set_projection", "tb_reset_sequence",
            "tb_get_length", "tb_append_kv", "tb_project_keys", "tb_score_tokens", "tb_select_topk",
-           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
+           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_predict_importance_queries", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
 
 
 class tb_config(C.Structure):
@@ -31,6 +31,14 @@ class tb_config(C.Structure):
 class tb_select_params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("budget", "sinks", "recent", "radius", "nmode", "interval", "step", "reduce")] + \
                [("score_scale", C.c_float)]
+
+
+class tb_predictor(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("dtype", "model_dim", "hidden_dim", "n_q_heads", "n_slots", "imp_dim", "activation")] + \
+               [("ln_eps", C.c_float)] + [(n, C.c_void_p) for n in ("ln_weight", "ln_bias", "w1", "w2")]
+
+
+TB_ACT_GELU, TB_ACT_SILU, TB_ACT_RELU = 0, 1, 2
 
 
 class TBError(RuntimeError):
@@ -70,6 +78,7 @@ def lib():
                                                  vp, vp, vp]
         L.tb_sparse_decode_attention_static.argtypes = [vp, i32, i32, i32, i32, i32, ip, ip, i32, vp, vp, vp, i32, i32, i32,
                                                         C.c_float, vp, vp, vp]
+        L.tb_predict_importance_queries.argtypes = [vp, vp, i32, vp, vp, vp]
         L.tb_get_status.argtypes = [vp, vp, ip]
         L.tb_last_step_bytes.argtypes = [vp]
         L.tb_launch_count.argtypes = [vp]
@@ -114,6 +123,16 @@ def sparse_decode_attention_static(kv, kv_dtype, n_q_heads, n_kv_heads, head_dim
                                                    _ints(seq_slots), _ints(seq_lens), len(seq_lens), _ptr(q), _ptr(idx),
                                                    _ptr(cnt), idx_stride, sinks, recent, sm_scale, _ptr(out), _ptr(lse),
                                                    _stream(stream))
+
+
+def predict_importance_queries(hidden, ln_weight, ln_bias, w1, w2, dtype, n_q_heads, n_slots, imp_dim, scratch, q_imp,
+                               ln_eps=1e-5, activation=TB_ACT_GELU, stream=None):
+    """Predictor forward q = W2 act(W1 LN(h)) for the rows of `hidden` [tokens, model_dim]; writes q_imp
+    [n_slots, tokens, n_q_heads, imp_dim].  Only marshals arguments for tb_predict_importance_queries;
+    returns its status code."""
+    p = tb_predictor(dtype, hidden.shape[1], w1.shape[0], n_q_heads, n_slots, imp_dim, activation, ln_eps,
+                     ln_weight.data_ptr(), ln_bias.data_ptr(), w1.data_ptr(), w2.data_ptr())
+    return lib().tb_predict_importance_queries(C.byref(p), _ptr(hidden), hidden.shape[0], _ptr(scratch), _ptr(q_imp), _stream(stream))
 
 
 class Context:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtokenbutler.so")
-SOURCES = ["tb_api.cu", "tb_cache.cu", "tb_select.cu", "tb_select_wave.cu", "tb_select_aux.cu", "tb_attention.cu"]
+SOURCES = ["tb_api.cu", "tb_cache.cu", "tb_select.cu", "tb_select_wave.cu", "tb_select_aux.cu", "tb_attention.cu", "tb_predictor.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
               "--expt-relaxed-constexpr", "--expt-extended-lambda"]
 

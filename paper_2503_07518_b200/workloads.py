@@ -14,7 +14,7 @@ from dataclasses import dataclass, field
 import numpy as np
 
 F32, BF16 = 0, 1
-TAG_K, TAG_V, TAG_Q, TAG_QIMP, TAG_W, TAG_AUX = 1, 2, 3, 4, 5, 6
+TAG_K, TAG_V, TAG_Q, TAG_QIMP, TAG_W, TAG_AUX, TAG_PRED = 1, 2, 3, 4, 5, 6, 7
 BASE_SEED = 250307518
 
 
@@ -178,3 +178,20 @@ def plant_keys(w: Workload, layer: int, seq: int, K: np.ndarray, W: np.ndarray, 
             K[h, p] = to_storage(k.astype(np.float32), w.dtype)
         pos_all.append(pos)
     return np.stack(pos_all)
+
+
+def gen_predictor(w: Workload, producer: int, model_dim: int = 4096, hidden_dim: int = 512, slots: int = 4, step: int = 0):
+    """Inputs of one producer layer's importance-query predictor, in the storage type: hidden states
+    [batch, model_dim] (unit-variance channels, a shared offset and 8 channels scaled by 20: residual
+    streams have a few massive channels), layer-norm weight ~ 1 and bias ~ 0, W1 [hidden, model_dim]
+    ~ N(0, 1/model_dim), W2 [slots * q_heads * imp_dim, hidden] ~ N(0, 4/hidden)."""
+    r = _rng(w.cfg_id, producer, 0, TAG_PRED)
+    ln_w = 1.0 + 0.1 * r.standard_normal(model_dim)
+    ln_b = 0.02 * r.standard_normal(model_dim)
+    W1 = r.standard_normal((hidden_dim, model_dim)) * model_dim ** -0.5
+    W2 = r.standard_normal((slots * w.n_q_heads * w.imp_dim, hidden_dim)) * 2.0 * hidden_dim ** -0.5
+    big = r.choice(model_dim, size=8, replace=False)
+    rh = _rng(w.cfg_id, producer, step, TAG_PRED + 8)
+    H = rh.standard_normal((w.batch, model_dim)) + 0.25
+    H[:, big] *= 20.0
+    return tuple(to_storage(np.ascontiguousarray(a, dtype=np.float32), w.dtype) for a in (H, ln_w, ln_b, W1, W2))

@@ -51,3 +51,23 @@ def test_host_validation_needs_no_gpu(libpath):
     bad = b.tb_config(2, 9, 8, 128, 32, b.TB_BF16, 1, 1024, 64, 1, 0)
     assert L.tb_query_sizes(ctypes.byref(bad), *[ctypes.byref(s) for s in sizes]) == b.TB_ERR_INVALID_ARG
     assert L.tb_status_string(b.TB_ERR_UNPROJECTED) == b"candidate keys not projected"
+
+
+def test_predictor_host_validation_needs_no_gpu(libpath):
+    from paper_2503_07518_b200 import binding as b
+    L = b.lib()
+    one = ctypes.c_void_p(16)                           # any aligned non-null address: never dereferenced on these paths
+    ok = dict(dtype=b.TB_BF16, model_dim=4096, hidden_dim=512, n_q_heads=32, n_slots=4, imp_dim=32, activation=b.TB_ACT_GELU,
+              ln_eps=1e-5, ln_weight=16, ln_bias=16, w1=16, w2=16)
+
+    def call(n_tokens=1, hidden=one, **over):
+        p = b.tb_predictor(**{**ok, **over})
+        return L.tb_predict_importance_queries(ctypes.byref(p), hidden, n_tokens, one, one, None)
+
+    assert call(w1=None) == b.TB_ERR_INVALID_ARG
+    assert call(hidden=None) == b.TB_ERR_INVALID_ARG
+    assert call(n_tokens=0) == b.TB_ERR_INVALID_ARG
+    assert call(activation=7) == b.TB_ERR_INVALID_ARG
+    assert call(ln_weight=24) == b.TB_ERR_INVALID_ARG      # not 16-byte aligned
+    assert call(model_dim=4100) == b.TB_ERR_UNSUPPORTED    # rows are read 16 bytes at a time
+    assert call(n_tokens=65) == b.TB_ERR_CAPACITY

@@ -418,3 +418,46 @@ def test_selection_beyond_cluster_capacity(H):
     one-block-per-problem kernel, whose bitmask does not fit its scratch either: the general path."""
     r = np.random.Generator(np.random.PCG64(79))
     _crafted_scores_case(H, _bf16_exact(r.standard_normal((1, 270001))), budget=5000, sinks=4, recent=64)
+
+
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_predictor_forward_matches_oracle(H, act):
+    """q = W2 act(W1 LN(h)) against the fp64 oracle on the same stored bytes: fp32 accumulation over
+    4096 and 512 terms of O(1) values, so 2e-4 absolute on outputs of magnitude ~2 is ample."""
+    import torch
+    for cfg, over, E, hid in ((2, dict(batch=5), 4096, 512), (1, dict(batch=3), 1000, 72)):   # bf16 8B shapes; fp32, odd sizes
+        w = wl.workload(cfg, **over)
+        Hs, ln_w, ln_b, W1, W2 = wl.gen_predictor(w, 1, model_dim=E, hidden_dim=hid, slots=4)
+        ref = H.orc.predict_queries(Hs, ln_w, ln_b, W1, W2, w.dtype, eps=1e-5, act=act)       # [tokens, slots * heads * d']
+        dev = [H.to_dev(a, w.dtype) for a in (Hs, ln_w, ln_b, W1, W2)]
+        scratch = torch.empty(w.batch * hid, dtype=torch.float32, device="cuda")
+        q = torch.full((4, w.batch, w.n_q_heads, w.imp_dim), float("nan"), dtype=torch.float32, device="cuda")
+        st = tb().predict_importance_queries(*dev, w.dtype, w.n_q_heads, 4, w.imp_dim, scratch, q, ln_eps=1e-5, activation=act)
+        assert st == tb().TB_OK
+        torch.cuda.synchronize()
+        got = q.cpu().numpy()                                                                  # [slot, token, head, d']
+        want = ref.reshape(w.batch, 4, w.n_q_heads, w.imp_dim).transpose(1, 0, 2, 3)
+        assert np.isfinite(got).all()
+        assert np.abs(got - want).max() <= 2e-4, np.abs(got - want).max()
+
+
+def test_predictor_output_feeds_selection(H):
+    """The predictor's output block is the q_imp argument of tb_select_topk for its consumer layers:
+    selecting with it on the GPU equals selecting with the oracle's queries in the oracle."""
+    import torch
+    w = wl.workload(2, n_layers=4, batch=2, lengths=[3000, 1800], budget=200)
+    case = H.Case(w)
+    Hs, ln_w, ln_b, W1, W2 = wl.gen_predictor(w, 0, model_dim=1024, hidden_dim=512, slots=4)
+    dev = [H.to_dev(a, w.dtype) for a in (Hs, ln_w, ln_b, W1, W2)]
+    scratch = torch.empty(w.batch * 512, dtype=torch.float32, device="cuda")
+    q = torch.empty((4, w.batch, w.n_q_heads, w.imp_dim), dtype=torch.float32, device="cuda")
+    assert tb().predict_importance_queries(*dev, w.dtype, w.n_q_heads, 4, w.imp_dim, scratch, q) == tb().TB_OK
+    p = tb().select_params(w.budget)
+    lists = H.gpu_select(case, q.cpu().numpy(), p)
+    assert case.ctx.get_status() == 0
+    ref = H.orc.predict_queries(Hs, ln_w, ln_b, W1, W2, w.dtype).reshape(w.batch, 4, w.n_q_heads, w.imp_dim).transpose(1, 0, 2, 3)
+    for l in range(4):
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                _, full, s = case.oracle_select(l, b, h, np.ascontiguousarray(ref[l, b], dtype=np.float32), p)
+                H.check_selection(lists[l][b][h], full, s, "layer %d seq %d head %d" % (l, b, h))

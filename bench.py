@@ -224,7 +224,7 @@ def run_ours(args, w):
 
     p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode)
     ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + 8,
-                      w.budget, w.radius, device=local)
+                      w.budget, w.radius, device=local, kv_on_host=args.offload_kv)
     proj_info = fill_caches(ctx, w, torch, tbh)
     dt = tbh.torch_dtype(w.dtype)
     gen = torch.Generator(device="cuda")
@@ -314,6 +314,17 @@ def run_ours(args, w):
         ms_att = timed(g_att.replay, max(20, args.steps // 4), 3) / w.n_layers
         # Upper bound, not the method's schedule: the importance queries of all layers at once, so the
         # selection runs as one call over every layer (many problems per launch) before the attentions.
+        offload_info = None
+        if args.offload_kv:
+            # the comparison the paper draws for offloaded KV: the same step attending to every cached token
+            p_dense = tbh.select_params(-1)
+            g_dense = capture(lambda: [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p_dense, out[l]) for l in range(w.n_layers)])
+            ms_dense = timed(g_dense.replay, 3, 1)
+            dense_bytes = float(sum(w.lengths)) * w.n_layers * w.n_kv_heads * 2 * w.head_dim * (2 if w.dtype == wl.BF16 else 4)
+            offload_info = {"kv_placement": "page-locked host memory, rows fetched by the attention kernel over the host link",
+                            "dense_step_us": ms_dense * 1e3, "dense_link_gbs": dense_bytes / (ms_dense * 1e-3) / 1e9,
+                            "sparse_link_gbs": float(np.sum(att_bytes)) / (ms_step * 1e-3) / 1e9,
+                            "sparse_speedup_over_dense": ms_dense / ms_step}
         g_all = capture(lambda: (ctx.select_topk(0, w.n_layers, None, w.batch, qi, p),
                                  [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)]))
         ms_all = timed(g_all.replay, max(20, args.steps // 4), 3)
@@ -344,7 +355,8 @@ def run_ours(args, w):
         "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "q_heads": w.n_q_heads,
+        "config": {"workload": w.name + ("+offloaded_kv" if args.offload_kv else ""), "layers": w.n_layers, "batch_per_gpu": w.batch,
+                   "q_heads": w.n_q_heads,
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "imp_dim": w.imp_dim,
                    "kv_storage": "bf16" if w.dtype == wl.BF16 else "f32", "context": w.lengths if len(set(w.lengths)) > 1 else w.lengths[0],
                    "budget": w.budget, "sinks": w.sinks, "recent": w.recent, "radius": w.radius, "interval": w.interval,
@@ -371,6 +383,7 @@ def run_ours(args, w):
                               "gbs": pred_bytes / (ms_pred * 1e-3) / 1e9, "producers_per_step": len(groups),
                               "note": "importance-query MLP of one producer layer (two launches); the step before the path, "
                                       "not part of the timed step"},
+        "offloaded_kv": offload_info,
         "prefill_projection": proj_info,
         "clocks": sampler.summary(),
     }
@@ -547,6 +560,8 @@ def main():
     ap.add_argument("--cpu-layers", type=int, default=2, help="layers in the CPU oracle's sample")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--profile", action="store_true", help="only warm-up + steps of plain launches (for ncu)")
+    ap.add_argument("--offload-kv", action="store_true",
+                    help="K|V cache in page-locked host memory (selected rows cross the host link); also times the dense step")
     ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
                     help="neighbour rule of the interval workload (default: its own, +-r dilation)")
     args = ap.parse_args()

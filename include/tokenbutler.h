@@ -92,7 +92,12 @@ tb_status tb_query_sizes(const tb_config* cfg, size_t* kv_bytes, size_t* kimp_by
 
 /* Bind the four regions (256-byte aligned device pointers; contents of kv/kimp may be anything,
  * state and workspace are cleared here with a synchronous memset).  The context owns nothing on the
- * device; tb_destroy frees only host memory.  All sequences start empty. */
+ * device; tb_destroy frees only host memory.  All sequences start empty.
+ * Offloaded KV (paper Sec. 4.4 "CPU-offloaded KV"): kv_dev alone may instead be page-locked host
+ * memory that the device addresses through the same pointer (cudaHostAlloc under unified addressing).
+ * Every call then works unchanged: appends and projections cross the host link, and attention fetches
+ * only the rows it attends to; the projected keys, lists and workspace stay in device memory.  Any
+ * pointer that is neither is refused here with TB_ERR_INVALID_ARG (it would fault in a kernel later). */
 tb_status tb_create(const tb_config* cfg, void* kv_dev, void* kimp_dev, void* state_dev,
                     void* workspace_dev, tb_ctx** out);
 tb_status tb_destroy(tb_ctx* ctx);

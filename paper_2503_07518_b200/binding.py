@@ -140,7 +140,7 @@ class Context:
     names of the C entry points and only marshal arguments."""
 
     def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, imp_dim, kv_dtype, max_batch, max_seq_len,
-                 max_budget, max_radius=0, device=0):
+                 max_budget, max_radius=0, device=0, kv_on_host=False):
         L = lib()
         self.cfg = tb_config(n_layers, n_q_heads, n_kv_heads, head_dim, imp_dim, kv_dtype, max_batch, max_seq_len,
                              max_budget, max_radius, device)
@@ -154,8 +154,10 @@ class Context:
         dt = torch_dtype(kv_dtype)
         es = 2 if kv_dtype == TB_BF16 else 4
         # caller-owned regions; kv / kimp exposed as typed views in the documented layouts
-        self.kv = torch.empty(self.sizes[0] // es, dtype=dt, device=self.device).view(
-            n_layers, max_batch, n_kv_heads, max_seq_len, 2, head_dim)
+        # (kv_on_host: the cache in page-locked host memory, addressed by the device through the same pointer)
+        kv_flat = torch.empty(self.sizes[0] // es, dtype=dt, pin_memory=True) if kv_on_host else \
+            torch.empty(self.sizes[0] // es, dtype=dt, device=self.device)
+        self.kv = kv_flat.view(n_layers, max_batch, n_kv_heads, max_seq_len, 2, head_dim)
         self.kimp = torch.empty(self.sizes[1] // es, dtype=dt, device=self.device).view(
             n_layers, max_batch, n_kv_heads, max_seq_len, imp_dim)
         self.state = torch.empty(self.sizes[2], dtype=torch.uint8, device=self.device)

@@ -146,6 +146,22 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return TB_ERR_CUDA;
     if (dev != cfg->device) return TB_ERR_INVALID_ARG;
+    {
+        // kimp, state and workspace must be device memory.  The KV cache may also be page-locked host
+        // memory that the device addresses through the same pointer (offloaded KV, paper Sec. 4.4):
+        // the attention kernels then fetch just the selected rows over the host link.  Anything else
+        // would fault in a kernel later, so it is refused here.
+        cudaPointerAttributes pa;
+        const void* dev_only[3] = {kimp, state, workspace};
+        for (const void* ptr : dev_only) {
+            if (cudaPointerGetAttributes(&pa, ptr) != cudaSuccess) { (void)cudaGetLastError(); return TB_ERR_INVALID_ARG; }
+            if (pa.type != cudaMemoryTypeDevice && pa.type != cudaMemoryTypeManaged) return TB_ERR_INVALID_ARG;
+        }
+        if (cudaPointerGetAttributes(&pa, kv) != cudaSuccess) { (void)cudaGetLastError(); return TB_ERR_INVALID_ARG; }
+        const bool on_device = pa.type == cudaMemoryTypeDevice || pa.type == cudaMemoryTypeManaged;
+        const bool mapped_host = pa.type == cudaMemoryTypeHost && pa.devicePointer == kv;
+        if (!on_device && !mapped_host) return TB_ERR_INVALID_ARG;
+    }
     tb_ctx* c = new (std::nothrow) tb_ctx();
     if (!c) return TB_ERR_INVALID_ARG;
     c->cfg = *cfg;

@@ -36,12 +36,12 @@ def to_host(t: torch.Tensor, dtype: int) -> np.ndarray:
 class Case:
     """A workload instantiated on the host (numpy) and on the device (tb.Context)."""
 
-    def __init__(self, w: wl.Workload, max_budget=None, max_radius=None, extra_len=0, project="device"):
+    def __init__(self, w: wl.Workload, max_budget=None, max_radius=None, extra_len=0, project="device", kv_on_host=False):
         self.w = w
         self.lengths = list(w.lengths)
         self.cap = max(self.lengths) + extra_len
         self.ctx = tb.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, self.cap,
-                              max_budget or max(1, w.budget), w.radius if max_radius is None else max_radius)
+                              max_budget or max(1, w.budget), w.radius if max_radius is None else max_radius, kv_on_host=kv_on_host)
         self.K = [[None] * w.batch for _ in range(w.n_layers)]     # [layer][seq] -> [Hkv, cap, D] storage
         self.V = [[None] * w.batch for _ in range(w.n_layers)]
         self.Kimp = [[None] * w.batch for _ in range(w.n_layers)]  # oracle's projection, [Hkv, cap, d']

@@ -461,3 +461,41 @@ def test_predictor_output_feeds_selection(H):
             for h in range(w.n_kv_heads):
                 _, full, s = case.oracle_select(l, b, h, np.ascontiguousarray(ref[l, b], dtype=np.float32), p)
                 H.check_selection(lists[l][b][h], full, s, "layer %d seq %d head %d" % (l, b, h))
+
+
+def test_kv_cache_in_pinned_host_memory(H):
+    """Offloaded KV: with the K|V cache in page-locked host memory every call works unchanged and gives
+    the same bits as with the cache on the device (same kernels, same order of operations); a pointer
+    the device cannot address is refused at tb_create."""
+    import ctypes
+    import torch
+    w = wl.workload(2, n_layers=2, batch=2, lengths=[2500, 1111], budget=150, sinks=2, recent=9)
+    p = tb().select_params(w.budget, w.sinks, w.recent)
+    q, qi = H.queries(w, 0)
+    res = []
+    for on_host in (False, True):
+        case = H.Case(w, extra_len=4, kv_on_host=on_host)
+        assert case.ctx.kv.is_cuda != on_host
+        lists = H.gpu_select(case, qi, p)
+        out, lse = H.gpu_attention(case, q, p)
+        case.append_step(0)                                   # one decode step: append (over the link), project, attend
+        out2, lse2 = H.gpu_attention(case, q, p)
+        assert case.ctx.get_status() == 0
+        res.append((lists, out, lse, out2, lse2))
+        if on_host:
+            case.project_all()                                # the new token's projected key (reads K over the link)
+            full_pipeline_check(H, case, p, step=1)           # and it matches the oracle
+    (la, oa, sa, oa2, sa2), (lb, ob, sb, ob2, sb2) = res
+    assert all(np.array_equal(x, y) for l in range(2) for s in range(2) for x, y in zip(la[l][s], lb[l][s]))
+    assert np.array_equal(oa, ob) and np.array_equal(sa, sb) and np.array_equal(oa2, ob2) and np.array_equal(sa2, sb2)
+    # pageable host memory is not addressable by the device: refused, nothing launched
+    b = tb()
+    cfg = b.tb_config(1, 8, 8, 128, 32, b.TB_BF16, 1, 256, 16, 0, 0)
+    sizes = [ctypes.c_size_t() for _ in range(4)]
+    assert b.lib().tb_query_sizes(ctypes.byref(cfg), *[ctypes.byref(s) for s in sizes]) == b.TB_OK
+    dev = [torch.empty(s.value + 256, dtype=torch.uint8, device="cuda") for s in sizes]
+    pageable = torch.empty(sizes[0].value + 256, dtype=torch.uint8)
+    al = lambda t: ctypes.c_void_p((t.data_ptr() + 255) & ~255)
+    h = ctypes.c_void_p()
+    assert b.lib().tb_create(ctypes.byref(cfg), al(pageable), al(dev[1]), al(dev[2]), al(dev[3]), ctypes.byref(h)) == b.TB_ERR_INVALID_ARG
+    assert b.lib().tb_create(ctypes.byref(cfg), al(dev[0]), al(pageable), al(dev[2]), al(dev[3]), ctypes.byref(h)) == b.TB_ERR_INVALID_ARG

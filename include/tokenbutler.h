@@ -53,7 +53,9 @@ typedef enum {
 } tb_status;
 
 typedef enum { TB_F32 = 0, TB_BF16 = 1 } tb_dtype;
-/* How the g importance queries of a GQA group become one ranking per KV head. */
+/* How the g importance queries of a GQA group become one ranking per KV head: a token's score is the
+ * sum (default) or the largest of the group's g head scores.  TB_PER_QHEAD (one list per query head, no
+ * row sharing) is named for completeness; the library answers TB_ERR_UNSUPPORTED to it. */
 typedef enum { TB_GROUP_SUM = 0, TB_GROUP_MAX = 1, TB_PER_QHEAD = 2 } tb_group_reduce;
 /* Neighbour fetching (Sec. 3.4): DILATE = every position within +-radius of a selected one;
  * CLUSTER = runs of consecutive selected positions get radius*len extra positions just outside the

@@ -308,14 +308,14 @@ tb_status tb_project_keys(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_
 tb_status tb_score_tokens(tb_ctx* c, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const float* q_imp, int32_t reduce,
                           float score_scale, float* scores, void* stream) {
     if (!c || !q_imp || !scores || bad_layers(c, layer, 1)) return TB_ERR_INVALID_ARG;
-    if (reduce != TB_GROUP_SUM) return TB_ERR_UNSUPPORTED;
+    if (reduce != TB_GROUP_SUM && reduce != TB_GROUP_MAX) return TB_ERR_UNSUPPORTED;   // per-query-head lists: not built
     int seqs[kMaxLaunchSeq];
     tb_status st = resolve_seqs(c, seq_ids, n_seq, seqs);
     if (st != TB_OK) return st;
     UnitTable ut;
     fill_table(c, &ut, layer, 1, seqs, n_seq);
     for (int i = 0; i < n_seq; ++i) ut.len[i] = c->len_proj[(size_t)layer * c->cfg.max_batch + seqs[i]];   // projected tokens only
-    if (launch_score(c, ut, q_imp, score_scale, scores, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+    if (launch_score(c, ut, q_imp, reduce, score_scale, scores, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     c->launches++;
     return TB_OK;
 }
@@ -325,7 +325,7 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
     if (!c || !p || bad_layers(c, lb, lc)) return TB_ERR_INVALID_ARG;
     if (p->budget < 0 || p->sinks < 0 || p->recent < 0 || p->radius < 0 || p->interval < 1 || p->step < 0) return TB_ERR_INVALID_ARG;
     if (p->nmode != TB_NEIGHBOR_DILATE && p->nmode != TB_NEIGHBOR_CLUSTER) return TB_ERR_INVALID_ARG;
-    if (p->reduce != TB_GROUP_SUM) return TB_ERR_UNSUPPORTED;
+    if (p->reduce != TB_GROUP_SUM && p->reduce != TB_GROUP_MAX) return TB_ERR_UNSUPPORTED;   // per-query-head lists: not built
     if (p->budget > c->cfg.max_budget || p->radius > c->cfg.max_radius) return TB_ERR_CAPACITY;
     int seqs[kMaxLaunchSeq];
     tb_status st = resolve_seqs(c, seq_ids, n_seq, seqs);
@@ -358,7 +358,7 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
         if (refresh) {
             SelectArgs a;
             a.q_imp = q_imp + (size_t)(l0 - lb) * n_seq * c->cfg.n_q_heads * c->cfg.imp_dim;
-            a.budget = p->budget, a.sinks = p->sinks, a.recent = p->recent;
+            a.budget = p->budget, a.sinks = p->sinks, a.recent = p->recent, a.reduce = p->reduce;
             if (p->radius == 0) {
                 a.idx_dst = nullptr, a.cnt_dst = nullptr, a.dst_is_state = 1, a.idx_stride = c->geom.idx_cap;
             } else {

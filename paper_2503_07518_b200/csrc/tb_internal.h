@@ -38,6 +38,7 @@ struct SelectArgs {
     int dst_is_state;     // 1: rows indexed by (layer, seq_id, head) in the context's lists; 0: by launch unit
     int idx_stride;
     int budget, sinks, recent;
+    int reduce;           // tb_group_reduce: TB_GROUP_SUM or TB_GROUP_MAX
 };
 
 struct NeighborArgs {
@@ -122,7 +123,7 @@ cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new
 cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, cudaStream_t s);
 
 // tb_select.cu
-cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, float scale, float* scores,
+cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, int reduce, float scale, float* scores,
                          cudaStream_t s);
 cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
 // one block per problem; launch_select hands over to it when a launch holds at least two problems per SM

@@ -17,6 +17,8 @@
 // launches take the general path: every digit through cluster-merged histograms.
 #include <cooperative_groups.h>
 
+#include <cstddef>
+
 #include "tb_select.cuh"
 
 namespace cg = cooperative_groups;
@@ -62,7 +64,10 @@ struct __align__(16) SelSmem {
     int above[kMaxCluster];             // per rank: keys in bins above the threshold bin
     int inbin[kMaxCluster];             // per rank: keys in the threshold bin
     uint32_t lists[kMaxCluster][kListCap];   // (bin << 16 | count) of every rank's non-empty bins
+    alignas(16) float qs[kMaxGroup * 32];           // TB_GROUP_MAX: the group's importance queries
 };
+
+static_assert(offsetof(SelSmem, qs) % 16 == 0, "qs is read with 16-byte loads");
 
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -131,7 +136,7 @@ __device__ __forceinline__ void find_digit(const int* hist, int k, SelSmem* sm, 
     __syncthreads();                                  // bc_* and warp_a may be reused right away
 }
 
-template <typename T, int DP>
+template <typename T, int DP, int RED>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_constant__ CUtensorMap tmap, Geom gm, UnitTable ut,
                                                              SelectArgs a, int tiles_per_cta, int n_stages,
                                                              int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt,
@@ -208,8 +213,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             tma_load_2d(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kTileRows), &sm->full[i]);
         }
     }
-    float qr[DP];
-    load_group_query<DP>(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    if (RED != TB_GROUP_SUM) __syncthreads();
 
     // ---- stream + score + first digit histogram -------------------------------------------------
     bool timed_out = false;
@@ -221,7 +227,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         const int slot = i * kTileRows + tid;
         if (slot < n_local) {
             const uint32_t off = tid * RB;
-            float sc = row_score<T, DP>(qr, [&](int c) {
+            float sc = scorer.score([&](int c) {
                 uint32_t o = off + c * 16;
                 o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
                 return *reinterpret_cast<const uint4*>(tile + o);
@@ -604,16 +610,21 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     cfg.attrs = attr;
     cfg.numAttrs = 1;
 
-#define TB_SEL(T, DP)                                                                                              \
+#define TB_SEL_R(T, DP, RED)                                                                                       \
     do {                                                                                                           \
         static unsigned char seen[64];                                                                            \
         if (first_use_on_this_device(seen)) {                                                                                         \
-            cudaError_t e = cudaFuncSetAttribute(select_kernel<T, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+            cudaError_t e = cudaFuncSetAttribute(select_kernel<T, DP, RED>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                                  227 * 1024);                                                      \
             if (e != cudaSuccess) return e;                                                                        \
         }                                                                                                          \
-        return cudaLaunchKernelEx(&cfg, select_kernel<T, DP>, c->kimp_map, gm, ut, a, tiles_per_cta, n_stages, c->st.idx, \
+        return cudaLaunchKernelEx(&cfg, select_kernel<T, DP, RED>, c->kimp_map, gm, ut, a, tiles_per_cta, n_stages, c->st.idx, \
                                   c->st.cnt, c->st.status);                                                        \
+    } while (0)
+#define TB_SEL(T, DP)                                            \
+    do {                                                         \
+        if (a.reduce == TB_GROUP_MAX) TB_SEL_R(T, DP, TB_GROUP_MAX); \
+        else TB_SEL_R(T, DP, TB_GROUP_SUM);                      \
     } while (0)
     if (gm.dtype == TB_BF16) {
         if (gm.dp == 32) TB_SEL(__nv_bfloat16, 32); else TB_SEL(__nv_bfloat16, 16);
@@ -621,6 +632,7 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
         if (gm.dp == 32) TB_SEL(float, 32); else TB_SEL(float, 16);
     }
 #undef TB_SEL
+#undef TB_SEL_R
 }
 
 }  // namespace tb

@@ -43,6 +43,59 @@ __device__ __forceinline__ float row_score(const float* qr, LoadChunk ld) {
     return acc0 + acc1;
 }
 
+// The same for TB_GROUP_MAX: the row's score is the largest of the g heads' dot products.  `qs` holds
+// the g importance queries, [g][DP] floats in shared memory (every lane reads the same words: broadcast).
+// Each head's dot product is accumulated exactly as in row_score.
+template <typename T, int DP, typename LoadChunk>
+__device__ __forceinline__ float row_score_max(const float* qs, int g, LoadChunk ld) {
+    constexpr int P = Elem<T>::kPer16;
+    constexpr int NCH = DP / P;
+    float f[DP];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) Elem<T>::unpack16(ld(c), f + c * P);
+    float best = -INFINITY;
+    for (int u = 0; u < g; ++u) {
+        const float4* q4 = reinterpret_cast<const float4*>(qs + u * DP);
+        float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+#pragma unroll
+            for (int e = 0; e < P; e += 4) {
+                const float4 q = q4[(c * P + e) / 4];
+                float& acc = (c & 1) ? acc1 : acc0;
+                acc = fmaf(q.x, f[c * P + e], acc), acc = fmaf(q.y, f[c * P + e + 1], acc);
+                acc = fmaf(q.z, f[c * P + e + 2], acc), acc = fmaf(q.w, f[c * P + e + 3], acc);
+            }
+        }
+        best = fmaxf(best, acc0 + acc1);
+    }
+    return best;
+}
+
+// How a selection kernel scores a row under the reduction RED (TB_GROUP_SUM: one dot product with the
+// summed query held in registers; TB_GROUP_MAX: g dot products against the queries in shared memory).
+template <typename T, int DP, int RED>
+struct GroupScorer {
+    float qr[RED == TB_GROUP_SUM ? DP : 1];
+    const float* qs;
+    int g;
+    // q_unit: the group's g queries [g][DP] in global memory; qs_smem: room for kMaxGroup * DP floats.
+    // All threads of the block call it; with TB_GROUP_MAX a block barrier must follow before score().
+    __device__ __forceinline__ void load(const float* __restrict__ q_unit, int g_, float* qs_smem) {
+        g = g_, qs = qs_smem;
+        if constexpr (RED == TB_GROUP_SUM) {
+            load_group_query<DP>(q_unit, g_, qr);
+        } else {
+            for (int i = threadIdx.x; i < g_ * DP; i += blockDim.x) qs_smem[i] = q_unit[i];
+        }
+    }
+    template <typename LoadChunk>
+    __device__ __forceinline__ float score(LoadChunk ld) const {
+        if constexpr (RED == TB_GROUP_SUM) return row_score<T, DP>(qr, ld);
+        else return row_score_max<T, DP>(qs, g, ld);
+    }
+};
+
 __device__ __forceinline__ void decode_unit(const Geom& gm, const UnitTable& ut, int u, int& ll, int& s, int& h) {
     h = u % gm.Hkv;
     s = (u / gm.Hkv) % ut.n_seq;

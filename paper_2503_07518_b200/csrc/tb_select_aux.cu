@@ -6,32 +6,38 @@ namespace tb {
 
 // ---- standalone scores ---------------------------------------------------------------------------
 
-template <typename T, int DP>
+template <typename T, int DP, int RED>
 __global__ void __launch_bounds__(256) score_kernel(Geom gm, UnitTable ut, const float* __restrict__ q_imp, float scale,
                                                     const T* __restrict__ kimp, float* __restrict__ scores) {
     constexpr int NCH = DP / Elem<T>::kPer16;
+    __shared__ __align__(16) float qs[kMaxGroup * 32];
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
     const int L = ut.len[ll * ut.n_seq + s];
-    float qr[DP];
-    load_group_query<DP>(q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load(q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qs);
+    if (RED != TB_GROUP_SUM) __syncthreads();
     const uint4* base = reinterpret_cast<const uint4*>(kimp + cache_unit(gm, ut, ll, s, h) * gm.max_seq_len * DP);
     float* out = scores + ((size_t)(ll * ut.n_seq + s) * gm.Hkv + h) * gm.max_seq_len;
     for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < L; t += gridDim.x * blockDim.x) {
         const uint4* row = base + (size_t)t * NCH;
-        float sc = row_score<T, DP>(qr, [&](int c) { return __ldg(row + c); });
+        float sc = scorer.score([&](int c) { return __ldg(row + c); });
         out[t] = scale * sc;
     }
 }
 
-cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, float scale, float* scores, cudaStream_t s) {
+cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, int reduce, float scale, float* scores, cudaStream_t s) {
     const Geom& gm = c->geom;
     int maxL = 0;
     for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) maxL = ut.len[i] > maxL ? ut.len[i] : maxL;
     if (maxL == 0) return cudaSuccess;
     dim3 grid((maxL + 255) / 256, ut.layer_count * ut.n_seq * gm.Hkv);
     if (grid.x > 64) grid.x = 64;
-#define TB_SCORE(T, DP) score_kernel<T, DP><<<grid, 256, 0, s>>>(gm, ut, q_imp, scale, (const T*)c->kimp, scores)
+#define TB_SCORE(T, DP)                                                                                                   \
+    do {                                                                                                                  \
+        if (reduce == TB_GROUP_MAX) score_kernel<T, DP, TB_GROUP_MAX><<<grid, 256, 0, s>>>(gm, ut, q_imp, scale, (const T*)c->kimp, scores); \
+        else score_kernel<T, DP, TB_GROUP_SUM><<<grid, 256, 0, s>>>(gm, ut, q_imp, scale, (const T*)c->kimp, scores);     \
+    } while (0)
     if (gm.dtype == TB_BF16) {
         if (gm.dp == 32) TB_SCORE(__nv_bfloat16, 32); else TB_SCORE(__nv_bfloat16, 16);
     } else {

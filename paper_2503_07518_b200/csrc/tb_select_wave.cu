@@ -74,8 +74,9 @@ struct __align__(16) WaveSmem {
     int warp_b[kWarps];
     int bc_bin, bc_krem, bc_count, n_list;
     uint32_t s_lo, s_hi;            // sample keys bracketing the expected threshold
+    alignas(16) float qs[kMaxGroup * 32];       // TB_GROUP_MAX: the group's importance queries
 };
-static_assert(offsetof(WaveSmem, sample) % 16 == 0, "sample is read as uint4");
+static_assert(offsetof(WaveSmem, sample) % 16 == 0 && offsetof(WaveSmem, qs) % 16 == 0, "read with 16-byte loads");
 
 // First digit of the radix select: 2048 bins, monotone in the key.  Bin 0 = below `base`, bins
 // 1..2046 = equal slices of 2^shift keys from `base` up, bin 2047 = everything above.  With base = 0
@@ -161,8 +162,7 @@ __device__ __forceinline__ void wave_find_digit(const int* hist, int k, WaveSmem
 __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const Digit dg, const uint32_t* __restrict__ keys,
                                                  unsigned char* scratch, int scratch_bytes, int ncand, int k, int lo,
                                                  int32_t* __restrict__ idx_dst, int32_t* __restrict__ cnt_dst) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t lt = (1u << lane) - 1u;
+    const int tid = threadIdx.x, lane = tid & 31;
 #ifdef TB_PHASE_TIMING
     unsigned long long tf0 = wave_now();
 #define FIN_MARK(i) do { if (tid == 0) { unsigned long long tn = wave_now(); atomicAdd(&g_fin_ns[i], tn - tf0); tf0 = tn; } } while (0)
@@ -311,7 +311,7 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
     return true;
 }
 
-template <typename T, int DP>
+template <typename T, int DP, int RED>
 __global__ void __launch_bounds__(kThreads, 4)
     select_wave_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut,
                        WaveOrder order, SelectArgs a, int n_stages,
@@ -381,8 +381,9 @@ __global__ void __launch_bounds__(kThreads, 4)
 #pragma unroll
         for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
     }
-    float qr[DP];
-    load_group_query<DP>(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qr);
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    if (RED != TB_GROUP_SUM) __syncthreads();
     if (tid == 0)
         for (int i = 0; i < n_stages && i < n_tiles; ++i) {
             mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
@@ -395,7 +396,7 @@ __global__ void __launch_bounds__(kThreads, 4)
     // open-ended bin, which sends the problem down the general path.
     Digit dg = {0u, 21};
     if (sampled) {
-        if (tid < kSampleRows) sm->sample[tid] = order_key(row_score<T, DP>(qr, [&](int c) { return srow[c]; }));
+        if (tid < kSampleRows) sm->sample[tid] = order_key(scorer.score([&](int c) { return srow[c]; }));
         __syncthreads();
         if (tid < kSampleRows) {   // descending rank of this thread's sample key (equal keys by index)
             const uint32_t mine = sm->sample[tid];
@@ -436,7 +437,7 @@ __global__ void __launch_bounds__(kThreads, 4)
         if (i == 0) wave_stamp(1);
         if (slot < ncand) {
             const uint32_t off = tid * RB;
-            const float sc = row_score<T, DP>(qr, [&](int c) {
+            const float sc = scorer.score([&](int c) {
                 uint32_t o = off + c * 16;
                 o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
                 return *reinterpret_cast<const uint4*>(tile + o);
@@ -608,17 +609,22 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
     if (n_stages < 2) n_stages = 2;
     const size_t smem = fixed + (size_t)n_stages * tile_bytes;
 
-#define TB_SEL(T, DP)                                                                                                   \
+#define TB_SEL_R(T, DP, RED)                                                                                                   \
     do {                                                                                                                \
         static unsigned char seen[64];                                                                                  \
         if (first_use_on_this_device(seen)) {                                                                           \
-            cudaError_t e = cudaFuncSetAttribute(select_wave_kernel<T, DP>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+            cudaError_t e = cudaFuncSetAttribute(select_wave_kernel<T, DP, RED>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                                  200 * 1024);                                                            \
             if (e != cudaSuccess) return e;                                                                             \
         }                                                                                                               \
-        select_wave_kernel<T, DP><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, c->st.idx, c->st.cnt, \
+        select_wave_kernel<T, DP, RED><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, c->st.idx, c->st.cnt, \
                                                                   c->st.status, c->wk.sel_keys);                        \
         return cudaGetLastError();                                                                                      \
+    } while (0)
+#define TB_SEL(T, DP)                                            \
+    do {                                                         \
+        if (a.reduce == TB_GROUP_MAX) TB_SEL_R(T, DP, TB_GROUP_MAX); \
+        else TB_SEL_R(T, DP, TB_GROUP_SUM);                      \
     } while (0)
     if (gm.dtype == TB_BF16) {
         if (gm.dp == 32) TB_SEL(__nv_bfloat16, 32); else TB_SEL(__nv_bfloat16, 16);
@@ -626,6 +632,7 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
         if (gm.dp == 32) TB_SEL(float, 32); else TB_SEL(float, 16);
     }
 #undef TB_SEL
+#undef TB_SEL_R
 }
 
 }  // namespace tb

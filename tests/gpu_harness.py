@@ -116,7 +116,8 @@ class Case:
     def oracle_select(self, l, b, h, q_imp, p):
         """Oracle list (after neighbours) and the fp64 scores, on the oracle's K_imp bytes."""
         w, L = self.w, self.cur[b]
-        s = orc.score(q_imp[h * w.group:(h + 1) * w.group], np.ascontiguousarray(self.Kimp[l][b][h, :L]), w.dtype)
+        s = orc.score(q_imp[h * w.group:(h + 1) * w.group], np.ascontiguousarray(self.Kimp[l][b][h, :L]), w.dtype,
+                      reduce=getattr(p, "reduce", orc.GROUP_SUM))
         base = orc.select(s, p.sinks, p.recent, p.budget)
         lo, hi = orc.candidate_range(L, p.sinks, p.recent)
         full = orc.neighbors(base, p.radius, p.nmode, lo, hi) if p.radius > 0 else base

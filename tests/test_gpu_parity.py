@@ -499,3 +499,45 @@ def test_kv_cache_in_pinned_host_memory(H):
     h = ctypes.c_void_p()
     assert b.lib().tb_create(ctypes.byref(cfg), al(pageable), al(dev[1]), al(dev[2]), al(dev[3]), ctypes.byref(h)) == b.TB_ERR_INVALID_ARG
     assert b.lib().tb_create(ctypes.byref(cfg), al(dev[0]), al(pageable), al(dev[2]), al(dev[3]), ctypes.byref(h)) == b.TB_ERR_INVALID_ARG
+
+
+def test_group_max_reduction(H):
+    """TB_GROUP_MAX (a token's score is the largest of its group's g head scores): materialised scores
+    against the oracle, the fused selection = exact top-k of those very fp32 values, on the cluster
+    kernel (one long sequence), on the many-problem kernel (40 sequences) and through the whole pipeline."""
+    b_ = tb()
+    # cluster kernel + score kernel, g = 4
+    w = wl.workload(2, n_layers=1, batch=2, lengths=[9000, 700], budget=300, sinks=2, recent=5)
+    case = H.Case(w)
+    q, qi = H.queries(w)
+    p = b_.select_params(w.budget, w.sinks, w.recent, reduce=b_.TB_GROUP_MAX)
+    scores = torch.full((w.batch, w.n_kv_heads, case.cap), float("nan"), device="cuda")
+    case.ctx.score_tokens(0, None, w.batch, torch.from_numpy(qi[0]).cuda(), scores, reduce=b_.TB_GROUP_MAX)
+    lists = H.gpu_select(case, qi, p)
+    sc = scores.cpu().numpy()
+    for b in range(w.batch):
+        L = case.cur[b]
+        for h in range(w.n_kv_heads):
+            _, _, s = case.oracle_select(0, b, h, qi[0, b], p)
+            assert np.allclose(sc[b, h, :L], s, rtol=1e-5, atol=1e-5)
+            ssum = H.orc.score(qi[0, b][h * w.group:(h + 1) * w.group], np.ascontiguousarray(case.Kimp[0][b][h, :L]), w.dtype)
+            assert not np.allclose(s, ssum)                                # and it is not the sum reduction
+            lo, hi = H.orc.candidate_range(L, p.sinks, p.recent)
+            cand = np.arange(lo, hi)
+            order = np.lexsort((cand, -sc[b, h, lo:hi].astype(np.float64)))
+            assert np.array_equal(lists[0][b][h], np.sort(cand[order[:w.budget]]))
+    full_pipeline_check(H, case, p)
+    # many-problem kernel: 40 sequences x 8 KV heads in one launch, fp32 storage and d' = 16 as well
+    for cfg, over in ((2, dict(n_layers=1, batch=40, lengths=[2300 + 37 * i for i in range(40)], budget=128)),
+                      (1, dict(n_layers=1, n_q_heads=16, n_kv_heads=8, imp_dim=16, batch=40, lengths=[2100 + 11 * i for i in range(40)],
+                               budget=64, sinks=1, recent=3))):
+        w = wl.workload(cfg, **over)
+        case = H.Case(w)
+        q, qi = H.queries(w)
+        p = b_.select_params(w.budget, w.sinks, w.recent, reduce=b_.TB_GROUP_MAX)
+        lists = H.gpu_select(case, qi, p)
+        assert case.ctx.get_status() == 0
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                _, full, s = case.oracle_select(0, b, h, qi[0, b], p)
+                H.check_selection(lists[0][b][h], full, s, "seq %d head %d" % (b, h))

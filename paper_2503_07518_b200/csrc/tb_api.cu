@@ -59,7 +59,8 @@ void compute_layout(const tb_config* c, Layout* l) {
     l->off_part_ml = o, o = align_up(o + units_q * kMaxSplits * 2 * 4, 256);
     l->off_sel_idx = o, o = align_up(o + units * l->sel_stride * 4, 256);
     l->off_sel_cnt = o, o = align_up(o + units * 4, 256);
-    l->off_sel_keys = o, o = align_up(o + units * align_up((size_t)c->max_seq_len, 4) * 4, 256);   // one 32-bit key per token
+    const size_t row = align_up((size_t)c->max_seq_len, 256);
+    l->off_sel_keys = o, o = align_up(o + units * row * 4, 256);       // one 32-bit key per token
     l->work_bytes = o;
 }
 

@@ -79,7 +79,7 @@ struct DevWork {
     int32_t* sel_idx;     // [n_layers*max_batch*Hkv][max_budget rounded]  pre-expansion selection
     int32_t* sel_cnt;
     int sel_stride;
-    uint32_t* sel_keys;   // [n_layers*max_batch*Hkv][max_seq_len rounded up to 4]  score keys of a many-problem selection launch
+    uint32_t* sel_keys;   // [n_layers*max_batch*Hkv][max_seq_len rounded up to 256]  score keys of a many-problem selection launch
 };
 
 }  // namespace tb

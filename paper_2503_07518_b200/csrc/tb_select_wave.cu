@@ -311,160 +311,14 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
     return true;
 }
 
-template <typename T, int DP, int RED>
-__global__ void __launch_bounds__(kThreads, 4)
-    select_wave_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut,
-                       WaveOrder order, SelectArgs a, int n_stages,
-                       int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt, int32_t* __restrict__ status,
-                       uint32_t* __restrict__ keys_g) {
-    constexpr int RB = DP * Elem<T>::kBytes;          // bytes per projected-key row: 32, 64 or 128
-    constexpr int NCH = RB / 16;
-    constexpr uint32_t kTileBytes = kRows * RB;
-
-    extern __shared__ unsigned char smem_raw[];
-    // swizzled TMA boxes need their shared-memory base on the swizzle period (up to 1024 bytes)
-    unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    int* hist = reinterpret_cast<int*>(stage_base + n_stages * kTileBytes);       // one digit at a time
-    WaveSmem* sm = reinterpret_cast<WaveSmem*>(hist + kDigitBins);
-    // The ring is idle once the rows are streamed; it then caches the problem's keys (as many as fit).
-    uint4* key_cache = reinterpret_cast<uint4*>(stage_base);
-    const int cache_vecs = n_stages * (int)kTileBytes / 16;                      // 16-byte vectors of 4 keys
-
+// General path: exact radix select (11 + 11 + 10 bits of the key itself) over all of a problem's
+// parked keys, then an ordered compaction with the lower-position tie rule.  The first pass over the
+// keys leaves them in `key_cache` (shared memory, `cache_vecs` 16-byte vectors; 0 = none).  `hist` is
+// scratch.  Called by all threads of the block.
+__device__ __forceinline__ void wave_general(int* hist, WaveSmem* sm, const uint32_t* __restrict__ keys_unit, uint4* key_cache,
+                                             int cache_vecs, int ncand, int k, int lo, int32_t* __restrict__ idx_dst,
+                                             int32_t* __restrict__ cnt_dst) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int pair = order.pair[blockIdx.x / gm.Hkv], h = blockIdx.x % gm.Hkv;
-    const int ll = pair / ut.n_seq, s = pair % ut.n_seq;
-    const int L = ut.len[pair];
-    const int lo = min(a.sinks, L);
-    const int hi = max(lo, L - a.recent);
-    const int ncand = hi - lo;
-    const int k = min(a.budget, ncand);
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
-    const size_t dst_row = a.dst_is_state ? cu : (size_t)pair * gm.Hkv + h;
-    int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
-    int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
-
-    if (k <= 0) {
-        if (tid == 0) *cnt_dst = 0;
-        return;
-    }
-    if (k == ncand) {                                  // budget covers every candidate: no ranking needed
-        for (int i = tid; i < ncand; i += kThreads) idx_dst[i] = lo + i;
-        if (tid == 0) *cnt_dst = k;
-        return;
-    }
-
-    // ---- set-up -------------------------------------------------------------------------------
-    wave_stamp(0);
-    for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
-    if (tid == 0) {
-        prefetch_tmap(&tmap);
-        for (int i = 0; i < n_stages; ++i) mbar_init(&sm->full[i], 1);
-        fence_mbar_init();
-    }
-    __syncthreads();
-
-    const int n_tiles = (ncand + kRows - 1) / kRows;
-    const long long row_base = (long long)cu * gm.max_seq_len + lo;              // row of candidate 0 in the 2-D view
-    uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 3) & ~3);     // by candidate index, 16-byte aligned
-    // The projected keys stream through L2 once; the score keys parked there must still be there when
-    // the block comes back for them.
-    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
-    // The sample row and the query are requested before the ring's first tiles: behind the whole
-    // grid's opening burst of bulk copies they would wait for microseconds.
-    const bool sampled = ncand >= kMinSampled;
-    uint4 srow[NCH];
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) srow[c] = make_uint4(0u, 0u, 0u, 0u);
-    if (sampled && tid < kSampleRows) {
-        const int slot = (int)(((long long)tid * ncand) / kSampleRows);
-        const uint4* rowp = reinterpret_cast<const uint4*>(kimp + (size_t)(row_base + slot) * RB);
-#pragma unroll
-        for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
-    }
-    GroupScorer<T, DP, RED> scorer;
-    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
-    if (RED != TB_GROUP_SUM) __syncthreads();
-    if (tid == 0)
-        for (int i = 0; i < n_stages && i < n_tiles; ++i) {
-            mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
-            tma_load_2d_hint(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kRows), &sm->full[i], stream_policy);
-        }
-
-    // ---- where to put the first digit's bins: a look at 256 rows spread over the problem ----------------
-    // Only the bins' resolution depends on the sample, never the result: the digit is monotone in the
-    // key whatever base and shift are, and a threshold that falls outside the sampled range lands in an
-    // open-ended bin, which sends the problem down the general path.
-    Digit dg = {0u, 21};
-    if (sampled) {
-        if (tid < kSampleRows) sm->sample[tid] = order_key(scorer.score([&](int c) { return srow[c]; }));
-        __syncthreads();
-        if (tid < kSampleRows) {   // descending rank of this thread's sample key (equal keys by index)
-            const uint32_t mine = sm->sample[tid];
-            const uint4* s4 = reinterpret_cast<const uint4*>(sm->sample);
-            int r = 0;
-#pragma unroll 8
-            for (int j4 = 0; j4 < kSampleRows / 4; ++j4) {
-                const uint4 x = s4[j4];
-                const int j = j4 * 4;
-                r += (x.x > mine) | ((x.x == mine) & (j < tid));
-                r += (x.y > mine) | ((x.y == mine) & (j + 1 < tid));
-                r += (x.z > mine) | ((x.z == mine) & (j + 2 < tid));
-                r += (x.w > mine) | ((x.w == mine) & (j + 3 < tid));
-            }
-            // about p * kSampleRows sample keys lie above the threshold (p = k / candidates); bracket it widely
-            const float p = (float)k / (float)ncand, mean = p * kSampleRows, sd = sqrtf(mean * (1.f - p));
-            const int r_hi = max(0, (int)floorf(mean - 6.f * sd) - 3), r_lo = min(kSampleRows - 1, (int)ceilf(mean + 6.f * sd) + 3);
-            if (r == r_hi) sm->s_hi = mine;
-            if (r == r_lo) sm->s_lo = mine;
-        }
-        __syncthreads();
-        const uint32_t s_lo = sm->s_lo, s_hi = sm->s_hi;
-        uint32_t range = s_hi - s_lo;
-        range += range >> 1;                           // room above the highest bracketing sample
-        if (range < s_hi - s_lo) range = 0xffffffffu;
-        dg.base = s_lo, dg.shift = 0;
-        while ((range >> dg.shift) >= 2046u) ++dg.shift;
-    }
-
-    // ---- stream + score + first digit histogram -------------------------------------------------
-    bool timed_out = false;
-    int st = 0;
-    uint32_t phase = 0;
-    for (int i = 0; i < n_tiles; ++i) {
-        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;   // keep going: control flow stays uniform
-        const unsigned char* tile = stage_base + st * kTileBytes;
-        const int slot = i * kRows + tid;
-        if (i == 0) wave_stamp(1);
-        if (slot < ncand) {
-            const uint32_t off = tid * RB;
-            const float sc = scorer.score([&](int c) {
-                uint32_t o = off + c * 16;
-                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
-                return *reinterpret_cast<const uint4*>(tile + o);
-            });
-            const uint32_t key = order_key(sc);
-            st_global_hint(keys_unit + slot, key, keep_policy);
-            hist_add(&hist[dg.bin(key)]);
-        }
-        __syncthreads();                               // all reads of this stage are done
-        if (tid == 0 && i + n_stages < n_tiles) {
-            fence_proxy_async();
-            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
-            tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kRows), &sm->full[st],
-                             stream_policy);
-        }
-        if (++st == n_stages) st = 0, phase ^= 1u;
-    }
-    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
-    __syncthreads();                                   // histogram complete, own keys visible to the block
-    wave_stamp(2);
-
-    // ---- finish -----------------------------------------------------------------------------------
-    if (wave_finish_mask(hist, sm, dg, keys_unit, stage_base, n_stages * (int)kTileBytes, ncand, k, lo, idx_dst, cnt_dst)) {
-        wave_stamp(3);
-        return;
-    }
-    // general path: exact radix select over all of the problem's keys
     const uint4* keys4 = reinterpret_cast<const uint4*>(keys_unit);
     const int n_vec = (ncand + 3) / 4;
     bool cached = false;                               // key_cache holds vectors [0, min(n_vec, cache_vecs))
@@ -580,6 +434,163 @@ __global__ void __launch_bounds__(kThreads, 4)
         }
     }
     if (tid == 0) *cnt_dst = k;
+
+}
+
+template <typename T, int DP, int RED>
+__global__ void __launch_bounds__(kThreads, 4)
+    select_wave_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut,
+                       WaveOrder order, SelectArgs a, int n_stages,
+                       int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt, int32_t* __restrict__ status,
+                       uint32_t* __restrict__ keys_g) {
+    constexpr int RB = DP * Elem<T>::kBytes;          // bytes per projected-key row: 32, 64 or 128
+    constexpr int NCH = RB / 16;
+    constexpr uint32_t kTileBytes = kRows * RB;
+
+    extern __shared__ unsigned char smem_raw[];
+    // swizzled TMA boxes need their shared-memory base on the swizzle period (up to 1024 bytes)
+    unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    int* hist = reinterpret_cast<int*>(stage_base + n_stages * kTileBytes);       // one digit at a time
+    WaveSmem* sm = reinterpret_cast<WaveSmem*>(hist + kDigitBins);
+    // The ring is idle once the rows are streamed; it then caches the problem's keys (as many as fit).
+    uint4* key_cache = reinterpret_cast<uint4*>(stage_base);
+    const int cache_vecs = n_stages * (int)kTileBytes / 16;                      // 16-byte vectors of 4 keys
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int pair = order.pair[blockIdx.x / gm.Hkv], h = blockIdx.x % gm.Hkv;
+    const int ll = pair / ut.n_seq, s = pair % ut.n_seq;
+    const int L = ut.len[pair];
+    const int lo = min(a.sinks, L);
+    const int hi = max(lo, L - a.recent);
+    const int ncand = hi - lo;
+    const int k = min(a.budget, ncand);
+    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t dst_row = a.dst_is_state ? cu : (size_t)pair * gm.Hkv + h;
+    int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
+    int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
+
+    if (k <= 0) {
+        if (tid == 0) *cnt_dst = 0;
+        return;
+    }
+    if (k == ncand) {                                  // budget covers every candidate: no ranking needed
+        for (int i = tid; i < ncand; i += kThreads) idx_dst[i] = lo + i;
+        if (tid == 0) *cnt_dst = k;
+        return;
+    }
+
+    // ---- set-up -------------------------------------------------------------------------------
+    wave_stamp(0);
+    for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
+    if (tid == 0) {
+        prefetch_tmap(&tmap);
+        for (int i = 0; i < n_stages; ++i) mbar_init(&sm->full[i], 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    const int n_tiles = (ncand + kRows - 1) / kRows;
+    const long long row_base = (long long)cu * gm.max_seq_len + lo;              // row of candidate 0 in the 2-D view
+    uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255); // by candidate index, 16-byte aligned
+    // The projected keys stream through L2 once; the score keys parked there must still be there when
+    // the block comes back for them.
+    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
+    // The sample row and the query are requested before the ring's first tiles: behind the whole
+    // grid's opening burst of bulk copies they would wait for microseconds.
+    const bool sampled = ncand >= kMinSampled;
+    uint4 srow[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) srow[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (sampled && tid < kSampleRows) {
+        const int slot = (int)(((long long)tid * ncand) / kSampleRows);
+        const uint4* rowp = reinterpret_cast<const uint4*>(kimp + (size_t)(row_base + slot) * RB);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
+    }
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    if (RED != TB_GROUP_SUM) __syncthreads();
+    if (tid == 0)
+        for (int i = 0; i < n_stages && i < n_tiles; ++i) {
+            mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
+            tma_load_2d_hint(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kRows), &sm->full[i], stream_policy);
+        }
+
+    // ---- where to put the first digit's bins: a look at 256 rows spread over the problem ----------------
+    // Only the bins' resolution depends on the sample, never the result: the digit is monotone in the
+    // key whatever base and shift are, and a threshold that falls outside the sampled range lands in an
+    // open-ended bin, which sends the problem down the general path.
+    Digit dg = {0u, 21};
+    if (sampled) {
+        if (tid < kSampleRows) sm->sample[tid] = order_key(scorer.score([&](int c) { return srow[c]; }));
+        __syncthreads();
+        if (tid < kSampleRows) {   // descending rank of this thread's sample key (equal keys by index)
+            const uint32_t mine = sm->sample[tid];
+            const uint4* s4 = reinterpret_cast<const uint4*>(sm->sample);
+            int r = 0;
+#pragma unroll 8
+            for (int j4 = 0; j4 < kSampleRows / 4; ++j4) {
+                const uint4 x = s4[j4];
+                const int j = j4 * 4;
+                r += (x.x > mine) | ((x.x == mine) & (j < tid));
+                r += (x.y > mine) | ((x.y == mine) & (j + 1 < tid));
+                r += (x.z > mine) | ((x.z == mine) & (j + 2 < tid));
+                r += (x.w > mine) | ((x.w == mine) & (j + 3 < tid));
+            }
+            // about p * kSampleRows sample keys lie above the threshold (p = k / candidates); bracket it widely
+            const float p = (float)k / (float)ncand, mean = p * kSampleRows, sd = sqrtf(mean * (1.f - p));
+            const int r_hi = max(0, (int)floorf(mean - 6.f * sd) - 3), r_lo = min(kSampleRows - 1, (int)ceilf(mean + 6.f * sd) + 3);
+            if (r == r_hi) sm->s_hi = mine;
+            if (r == r_lo) sm->s_lo = mine;
+        }
+        __syncthreads();
+        const uint32_t s_lo = sm->s_lo, s_hi = sm->s_hi;
+        uint32_t range = s_hi - s_lo;
+        range += range >> 1;                           // room above the highest bracketing sample
+        if (range < s_hi - s_lo) range = 0xffffffffu;
+        dg.base = s_lo, dg.shift = 0;
+        while ((range >> dg.shift) >= 2046u) ++dg.shift;
+    }
+
+    // ---- stream + score + first digit histogram -------------------------------------------------
+    bool timed_out = false;
+    int st = 0;
+    uint32_t phase = 0;
+    for (int i = 0; i < n_tiles; ++i) {
+        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;   // keep going: control flow stays uniform
+        const unsigned char* tile = stage_base + st * kTileBytes;
+        const int slot = i * kRows + tid;
+        if (i == 0) wave_stamp(1);
+        if (slot < ncand) {
+            const uint32_t off = tid * RB;
+            const float sc = scorer.score([&](int c) {
+                uint32_t o = off + c * 16;
+                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
+                return *reinterpret_cast<const uint4*>(tile + o);
+            });
+            const uint32_t key = order_key(sc);
+            st_global_hint(keys_unit + slot, key, keep_policy);
+            hist_add(&hist[dg.bin(key)]);
+        }
+        __syncthreads();                               // all reads of this stage are done
+        if (tid == 0 && i + n_stages < n_tiles) {
+            fence_proxy_async();
+            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+            tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kRows), &sm->full[st],
+                             stream_policy);
+        }
+        if (++st == n_stages) st = 0, phase ^= 1u;
+    }
+    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    __syncthreads();                                   // histogram complete, own keys visible to the block
+    wave_stamp(2);
+
+    // ---- finish -----------------------------------------------------------------------------------
+    if (wave_finish_mask(hist, sm, dg, keys_unit, stage_base, n_stages * (int)kTileBytes, ncand, k, lo, idx_dst, cnt_dst)) {
+        wave_stamp(3);
+        return;
+    }
+    wave_general(hist, sm, keys_unit, key_cache, cache_vecs, ncand, k, lo, idx_dst, cnt_dst);
     wave_stamp(3);
 }
 
@@ -614,7 +625,7 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
         static unsigned char seen[64];                                                                                  \
         if (first_use_on_this_device(seen)) {                                                                           \
             cudaError_t e = cudaFuncSetAttribute(select_wave_kernel<T, DP, RED>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                                 200 * 1024);                                                            \
+                                                 226 * 1024);                                                            \
             if (e != cudaSuccess) return e;                                                                             \
         }                                                                                                               \
         select_wave_kernel<T, DP, RED><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, c->st.idx, c->st.cnt, \

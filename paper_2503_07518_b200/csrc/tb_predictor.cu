@@ -9,6 +9,8 @@
 // in registers.  Two launches: hidden units (layer norm folded in; each block recomputes the few
 // tokens' statistics rather than exchanging them), then outputs written in the layout
 // tb_select_topk reads.  No context: weights and scratch belong to the caller.
+#include <cooperative_groups.h>
+
 #include "tb_common.cuh"
 #include "tb_internal.h"
 
@@ -207,6 +209,184 @@ __global__ void __launch_bounds__(kPredThreads) predictor_out_kernel(const T* __
     }
 }
 
+// ---- several tokens at once (bf16): both linears on the tensor cores ---------------------------------
+// With 5 or more tokens the products above re-walk a weight row once per token chunk; a tile of 16
+// tokens x 8 outputs per mma.sync.m16n8k16 reads each weight once for all of them.  The left operand
+// (normalised hidden states, resp. hidden units) is fp32: it is split into a bf16 high and low part
+// and multiplied twice, so the products keep ~16 bits of it and accumulate in fp32.
+// The 16 k-indices of an MMA step are mapped to channels so that every thread's operands are 16
+// contiguous bytes: over a run of 32 channels, thread (row gid, column pair tig) takes channels
+// 8 tig .. 8 tig + 7; the first four feed the first MMA step (k = 2 tig, 2 tig + 1, 2 tig + 8, 2 tig + 9),
+// the last four the second.  Both operands use the same mapping, so the sum over channels is unchanged.
+__device__ __forceinline__ void mma_bf16_16x8x16(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// fp32 pair -> bf16x2 high parts and bf16x2 of what they leave
+__device__ __forceinline__ void split_bf16x2(float x, float y, uint32_t& hi, uint32_t& lo) {
+    const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+    const __nv_bfloat16 xl = __float2bfloat16_rn(x - __bfloat162float(xh)), yl = __float2bfloat16_rn(y - __bfloat162float(yh));
+    hi = (uint32_t)__bfloat16_as_ushort(xh) | ((uint32_t)__bfloat16_as_ushort(yh) << 16);
+    lo = (uint32_t)__bfloat16_as_ushort(xl) | ((uint32_t)__bfloat16_as_ushort(yl) << 16);
+}
+// One run of 32 channels: x0 / x1 = this thread's 8 left-operand values of rows gid / gid + 8 (zeros for
+// rows past the tokens), w = its 8 right-operand values (16 bytes of the weight row of output gid).
+__device__ __forceinline__ void mma_run32(float* acc, const float* x0, const float* x1, const uint4& w) {
+    const uint32_t wb[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int st = 0; st < 2; ++st) {
+        uint32_t h0, l0, h1, l1, h2, l2, h3, l3;
+        split_bf16x2(x0[4 * st], x0[4 * st + 1], h0, l0);          // row gid,     k = 2 tig, 2 tig + 1
+        split_bf16x2(x1[4 * st], x1[4 * st + 1], h1, l1);          // row gid + 8
+        split_bf16x2(x0[4 * st + 2], x0[4 * st + 3], h2, l2);      // row gid,     k = 2 tig + 8, 2 tig + 9
+        split_bf16x2(x1[4 * st + 2], x1[4 * st + 3], h3, l3);
+        mma_bf16_16x8x16(acc, h0, h1, h2, h3, wb[2 * st], wb[2 * st + 1]);
+        mma_bf16_16x8x16(acc, l0, l1, l2, l3, wb[2 * st], wb[2 * st + 1]);
+    }
+}
+
+constexpr int kSplitK = 4;           // thread blocks (one cluster) that share the channels of a hidden-unit tile
+
+// hidden[t][j] for 8 hidden units per cluster of kSplitK blocks: block r takes a quarter of the channels,
+// its 8 warps a run of 32 channels at a time; partial tiles are summed in rank 0's shared memory
+// (distributed shared memory, fixed order).  The layer-norm statistics of the tokens are split over
+// the cluster the same way.
+__global__ void __launch_bounds__(kPredThreads) predictor_hidden_mma_kernel(const __nv_bfloat16* __restrict__ H,
+                                                                            const __nv_bfloat16* __restrict__ ln_w,
+                                                                            const __nv_bfloat16* __restrict__ ln_b,
+                                                                            const __nv_bfloat16* __restrict__ W1,
+                                                                            float* __restrict__ hidden, int n_tok, int E, int hid,
+                                                                            float eps, int act) {
+    using EB = Elem<__nv_bfloat16>;
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();        // == blockIdx.x
+    pdl_launch_dependents();
+    __shared__ float s_mean[kPredMaxTokens], s_rstd[kPredMaxTokens];
+    __shared__ float s_acc[kSplitK][kPredWarps][16][8];   // rank 0 receives every block's per-warp tiles
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
+    // statistics of tokens rank*8+warp, +32, ...: shifted one-pass sums, sixteen 16-byte loads in flight
+    for (int t = rank * kPredWarps + warp; t < n_tok; t += kSplitK * kPredWarps) {
+        const uint4* h4 = reinterpret_cast<const uint4*>(H + (size_t)t * E);
+        const float shift = __bfloat162float(H[(size_t)t * E]);
+        float f[8], s1 = 0.f, s2 = 0.f;
+#pragma unroll 4
+        for (int v = lane; v < E / 8; v += 32) {
+            EB::unpack16(__ldg(h4 + v), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float d = f[e] - shift;
+                s1 += d, s2 = fmaf(d, d, s2);
+            }
+        }
+        s1 = warp_sum(s1), s2 = warp_sum(s2);
+        if (lane < kSplitK) {                          // lane r tells block r
+            const float m = s1 / (float)E;
+            *cluster.map_shared_rank(&s_mean[t], lane) = shift + m;
+            *cluster.map_shared_rank(&s_rstd[t], lane) = rsqrtf(fmaxf(s2 / (float)E - m * m, 0.f) + eps);
+        }
+    }
+    cluster.sync();
+    const int j0 = blockIdx.y * 8;                     // the cluster's hidden units; hid is a multiple of 8
+    const __nv_bfloat16* wrow = W1 + (size_t)(j0 + gid) * E;
+    const int n_runs = E / 32, runs_per_block = (n_runs + kSplitK - 1) / kSplitK;
+    const int r_begin = rank * runs_per_block, r_end = min(n_runs, r_begin + runs_per_block);
+    float(*acc0)[kPredWarps][16][8] = cluster.map_shared_rank(s_acc, 0);
+    for (int t0 = 0; t0 < n_tok; t0 += 16) {
+        const int ta = t0 + gid, tb_ = t0 + gid + 8;
+        const bool va = ta < n_tok, vb = tb_ < n_tok;
+        const float ma = va ? s_mean[ta] : 0.f, ra = va ? s_rstd[ta] : 0.f, mb = vb ? s_mean[tb_] : 0.f, rb = vb ? s_rstd[tb_] : 0.f;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int r0 = r_begin + warp; r0 < r_end; r0 += 2 * kPredWarps) {       // two runs' loads in flight
+            uint4 wv[2], gv[2], bv[2], hav[2], hbv[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int r = r0 + i * kPredWarps;
+                const int c = min(r, r_end - 1) * 32 + 8 * tig;
+                wv[i] = __ldg(reinterpret_cast<const uint4*>(wrow + c));
+                gv[i] = __ldg(reinterpret_cast<const uint4*>(ln_w + c));
+                bv[i] = __ldg(reinterpret_cast<const uint4*>(ln_b + c));
+                hav[i] = va ? __ldg(reinterpret_cast<const uint4*>(H + (size_t)ta * E + c)) : make_uint4(0u, 0u, 0u, 0u);
+                hbv[i] = vb ? __ldg(reinterpret_cast<const uint4*>(H + (size_t)tb_ * E + c)) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                if (r0 + i * kPredWarps >= r_end) break;   // warp-uniform
+                float g[8], b[8], ha[8], hb[8];
+                EB::unpack16(gv[i], g), EB::unpack16(bv[i], b), EB::unpack16(hav[i], ha), EB::unpack16(hbv[i], hb);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    ha[e] = va ? fmaf((ha[e] - ma) * ra, g[e], b[e]) : 0.f;
+                    hb[e] = vb ? fmaf((hb[e] - mb) * rb, g[e], b[e]) : 0.f;
+                }
+                mma_run32(acc, ha, hb, wv[i]);
+            }
+        }
+        // acc: rows gid (acc[0..1]) and gid + 8 (acc[2..3]), units 2 tig, 2 tig + 1 -> rank 0
+        acc0[rank][warp][gid][2 * tig] = acc[0], acc0[rank][warp][gid][2 * tig + 1] = acc[1];
+        acc0[rank][warp][gid + 8][2 * tig] = acc[2], acc0[rank][warp][gid + 8][2 * tig + 1] = acc[3];
+        cluster.sync();
+        if (rank == 0 && tid < 128) {
+            const int row = tid >> 3, col = tid & 7;
+            float a = 0.f;
+#pragma unroll
+            for (int r = 0; r < kSplitK; ++r)
+#pragma unroll
+                for (int w = 0; w < kPredWarps; ++w) a += s_acc[r][w][row][col];
+            if (t0 + row < n_tok) hidden[(size_t)(t0 + row) * hid + j0 + col] = activate(a, act);
+        }
+        cluster.sync();                                // rank 0 has read the tiles before the next round overwrites them
+    }
+}
+
+// q_imp for 8 output rows per half block: a block's 8 warps are 2 output tiles x 4 quarters of the row.
+__global__ void __launch_bounds__(kPredThreads) predictor_out_mma_kernel(const __nv_bfloat16* __restrict__ W2, const float* __restrict__ hidden,
+                                                                         float* __restrict__ q_imp, int n_tok, int hid, int n_out,
+                                                                         int per_slot) {
+    __shared__ float s_acc[2][4][16][8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
+    const int tile = warp >> 2, quarter = warp & 3;
+    const int o0 = (blockIdx.x * 2 + tile) * 8;        // n_out is a multiple of 8
+    const bool live = o0 < n_out;
+    const __nv_bfloat16* wrow = W2 + (size_t)(live ? o0 + gid : 0) * hid;
+    const int n_runs = hid / 32, runs_per_q = (n_runs + 3) / 4;
+    const int r_begin = quarter * runs_per_q, r_end = min(n_runs, r_begin + runs_per_q);
+    // the weights of this warp's first two runs do not depend on the hidden units: fetch them, then wait
+    uint4 wpre[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) wpre[i] = __ldg(reinterpret_cast<const uint4*>(wrow + min(r_begin + i, max(n_runs - 1, 0)) * 32 + 8 * tig));
+    pdl_wait();                                        // the hidden units come from the previous kernel
+    for (int t0 = 0; t0 < n_tok; t0 += 16) {
+        const int ta = t0 + gid, tb_ = t0 + gid + 8;
+        const bool va = ta < n_tok, vb = tb_ < n_tok;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int r = r_begin; r < r_end; ++r) {
+            const int c = r * 32 + 8 * tig;
+            const uint4 wv = r - r_begin < 2 ? wpre[r - r_begin] : __ldg(reinterpret_cast<const uint4*>(wrow + c));
+            float ha[8], hb[8];
+#pragma unroll
+            for (int e = 0; e < 8; e += 4) {
+                const float4 xa = va ? __ldcg(reinterpret_cast<const float4*>(hidden + (size_t)ta * hid + c + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 xb = vb ? __ldcg(reinterpret_cast<const float4*>(hidden + (size_t)tb_ * hid + c + e)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                ha[e] = xa.x, ha[e + 1] = xa.y, ha[e + 2] = xa.z, ha[e + 3] = xa.w;
+                hb[e] = xb.x, hb[e + 1] = xb.y, hb[e + 2] = xb.z, hb[e + 3] = xb.w;
+            }
+            mma_run32(acc, ha, hb, wv);
+        }
+        s_acc[tile][quarter][gid][2 * tig] = acc[0], s_acc[tile][quarter][gid][2 * tig + 1] = acc[1];
+        s_acc[tile][quarter][gid + 8][2 * tig] = acc[2], s_acc[tile][quarter][gid + 8][2 * tig + 1] = acc[3];
+        __syncthreads();
+        {
+            const int tl = tid >> 7, row = (tid >> 3) & 15, col = tid & 7;   // 256 threads = 2 tiles x 16 rows x 8 columns
+            const int t = t0 + row, o = (blockIdx.x * 2 + tl) * 8 + col;
+            const float a = s_acc[tl][0][row][col] + s_acc[tl][1][row][col] + s_acc[tl][2][row][col] + s_acc[tl][3][row][col];
+            if (t < n_tok && o < n_out) q_imp[((size_t)(o / per_slot) * n_tok + t) * per_slot + o % per_slot] = a;
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 }  // namespace tb
@@ -241,7 +421,25 @@ extern "C" tb_status tb_predict_importance_queries(const tb_predictor* p, const 
     cfg.attrs = attr, cfg.numAttrs = 1;
     const int per_slot = p->n_q_heads * p->imp_dim, n_out_i = (int)n_out;
     cudaError_t e;
-    if (p->dtype == TB_BF16) {
+    if (p->dtype == TB_BF16 && n_tokens >= 5 && p->model_dim % 32 == 0 && p->hidden_dim % 32 == 0 && n_out % 8 == 0) {
+        // several tokens: tensor-core tiles of 16 tokens x 8 outputs
+        {
+            cudaLaunchConfig_t c1 = {};
+            c1.gridDim = dim3(kSplitK, p->hidden_dim / 8, 1), c1.blockDim = dim3(kPredThreads, 1, 1), c1.stream = s;
+            cudaLaunchAttribute a1[1];
+            a1[0].id = cudaLaunchAttributeClusterDimension;
+            a1[0].val.clusterDim.x = kSplitK, a1[0].val.clusterDim.y = 1, a1[0].val.clusterDim.z = 1;
+            c1.attrs = a1, c1.numAttrs = 1;
+            if (cudaLaunchKernelEx(&c1, predictor_hidden_mma_kernel, (const __nv_bfloat16*)hidden_dev, (const __nv_bfloat16*)p->ln_weight,
+                                   (const __nv_bfloat16*)p->ln_bias, (const __nv_bfloat16*)p->w1, scratch_dev, (int)n_tokens,
+                                   (int)p->model_dim, (int)p->hidden_dim, p->ln_eps, (int)p->activation) != cudaSuccess)
+                return TB_ERR_CUDA;
+        }
+        cfg.gridDim = dim3((unsigned)((n_out / 8 + 1) / 2), 1, 1);
+        cfg.dynamicSmemBytes = 0;
+        e = cudaLaunchKernelEx(&cfg, predictor_out_mma_kernel, (const __nv_bfloat16*)p->w2, (const float*)scratch_dev, q_imp_dev,
+                               (int)n_tokens, (int)p->hidden_dim, n_out_i, per_slot);
+    } else if (p->dtype == TB_BF16) {
         predictor_hidden_kernel<__nv_bfloat16><<<g1, kPredThreads, 0, s>>>(
             (const __nv_bfloat16*)hidden_dev, (const __nv_bfloat16*)p->ln_weight, (const __nv_bfloat16*)p->ln_bias,
             (const __nv_bfloat16*)p->w1, scratch_dev, n_tokens, p->model_dim, p->hidden_dim, p->ln_eps, p->activation);

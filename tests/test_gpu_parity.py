@@ -425,7 +425,10 @@ def test_predictor_forward_matches_oracle(H, act):
     """q = W2 act(W1 LN(h)) against the fp64 oracle on the same stored bytes: fp32 accumulation over
     4096 and 512 terms of O(1) values, so 2e-4 absolute on outputs of magnitude ~2 is ample."""
     import torch
-    for cfg, over, E, hid in ((2, dict(batch=5), 4096, 512), (1, dict(batch=3), 1000, 72)):   # bf16 8B shapes; fp32, odd sizes
+    # bf16 8B shapes at 1 token (matrix-vector kernels), 5 and 20 tokens (tensor-core tiles, one and two of them);
+    # bf16 with sizes the tiles do not divide; fp32, odd sizes
+    for cfg, over, E, hid in ((2, dict(batch=1), 4096, 512), (2, dict(batch=5), 4096, 512), (2, dict(batch=20), 4096, 512),
+                              (2, dict(batch=7), 1000, 72), (1, dict(batch=3), 1000, 72)):
         w = wl.workload(cfg, **over)
         Hs, ln_w, ln_b, W1, W2 = wl.gen_predictor(w, 1, model_dim=E, hidden_dim=hid, slots=4)
         ref = H.orc.predict_queries(Hs, ln_w, ln_b, W1, W2, w.dtype, eps=1e-5, act=act)       # [tokens, slots * heads * d']

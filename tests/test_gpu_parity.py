@@ -544,3 +544,13 @@ def test_group_max_reduction(H):
             for h in range(w.n_kv_heads):
                 _, full, s = case.oracle_select(0, b, h, qi[0, b], p)
                 H.check_selection(lists[0][b][h], full, s, "seq %d head %d" % (b, h))
+
+
+@pytest.mark.parametrize("nmode", [0, 1])
+def test_many_problem_selection_with_neighbours_and_attention(H, nmode):
+    """The one-block-per-problem selection kernel in the full pipeline: 32 sequences x 8 KV heads per
+    launch, neighbour expansion from its pre-expansion lists, attention from the stored lists."""
+    w = wl.workload(5, n_layers=1, batch=32, lengths=[2100 + 29 * i for i in range(32)], budget=120, sinks=2, recent=16, radius=1)
+    case = H.Case(w)
+    p = tb().select_params(w.budget, w.sinks, w.recent, radius=1, nmode=nmode)
+    full_pipeline_check(H, case, p)

@@ -624,8 +624,10 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
 }
 
 static int pick_nsplit(const tb_ctx* c, int units, int max_rows) {
-    int target = 4 * c->sm_count;
-    int n = (target + units - 1) / units;
+    // about two blocks per SM and never a thin second wave: with 64 problems of 9.8K rows, 4 splits
+    // (256 blocks) ran at 58.5 us, 5 at 63.6, 6 at 61.5, 7 (448 blocks, four more than fit at once) at 75.7,
+    // 10 at 65.0
+    int n = 2 * c->sm_count / units;
     int by_rows = max_rows / 64;
     if (n > by_rows) n = by_rows;
     if (n > kMaxSplits) n = kMaxSplits;

@@ -128,6 +128,8 @@ cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_im
 cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
 // one block per problem; launch_select hands over to it when a launch holds at least two problems per SM
 cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
+// few, long problems: a cluster per problem on parked keys
+cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
 cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s);
 cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s);
 

@@ -33,6 +33,8 @@ constexpr int kBins = 2048;         // 11-bit digits (the last digit has 10 bits
 constexpr int kMaxCluster = 8;
 constexpr int kMaxKeysPerBlock = 32768;   // 128 KB of on-chip keys per block at most
 constexpr int kListCap = 256;       // non-empty first-digit bins a block may publish on the fast path
+constexpr int kCwFrom = 48 * 1024;   // candidates from which the parked-key cluster kernel takes over
+constexpr int kCwLimit = 8 * 32768;  // ... and up to which it can (8 blocks x 64 KB of first digits)
 constexpr int kCandCap = 4096;      // keys of the threshold bin gathered at rank 0 (aliases merged[1..2])
 
 // Optional per-phase timestamps of the first and last block of unit 0, for tuning builds only
@@ -565,6 +567,10 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     // fill the GPU by themselves: one block each, no clusters.  So do problems too long for a cluster's
     // on-chip key arrays.
     if (2 * n_units >= 3 * c->sm_count || max_cand > kMaxCluster * kMaxKeysPerBlock) return launch_select_wave(c, ut, a, s);
+    // Long problems (beyond ~48K candidates) go to the cluster kernel that parks the keys in memory and
+    // keeps 2 bytes per row on chip: two blocks per SM where this one, with 4 bytes per row, has room for
+    // one (128K tokens: 70.1 -> 59.1 us per launch; at 32K the two are level, below that this one wins).
+    if (max_cand > kCwFrom && max_cand <= kCwLimit) return launch_select_cw(c, ut, a, s);
     const int n_tiles = (max_cand + kTileRows - 1) / kTileRows;
     // Cluster size: enough blocks to cover the GPU about twice, at least 4 tiles per block, and a
     // key array per block of at most 32 KB where the cluster limit allows (64 KB otherwise).

@@ -1,4 +1,5 @@
-// Fused importance scoring + exact top-B selection for launches with many problems (paper Sec. 3.4
+// Fused importance scoring + exact top-B selection on parked keys: the kernel for launches with many
+// problems (below) and, at the end of the file, the cluster kernel for few long problems (paper Sec. 3.4
 // "score computation against all projected keys ... top-B selection", Sec. 4 "Token Selection
 // Policy"): batched serving, where one launch holds several hundred (layer, sequence, KV head)
 // problems and the GPU is filled by problems, not by splitting one.
@@ -50,6 +51,7 @@ struct WaveOrder {
 
 #ifdef TB_PHASE_TIMING
 __device__ unsigned long long g_fin_ns[8];
+__device__ unsigned long long g_cw_ns[8];
 __device__ unsigned long long g_wave_ns[4][1024];       // per block: start, first tile landed, rows streamed, end
 __device__ __forceinline__ unsigned long long wave_now() {
     unsigned long long t;
@@ -595,6 +597,7 @@ __global__ void __launch_bounds__(kThreads, 4)
 }
 
 #ifdef TB_PHASE_TIMING
+extern "C" int tb_debug_cw_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_cw_ns, sizeof(g_cw_ns)); }
 extern "C" int tb_debug_fin_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_fin_ns, sizeof(g_fin_ns)); }
 extern "C" int tb_debug_wave_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_wave_ns, sizeof(g_wave_ns)); }
 #endif
@@ -644,6 +647,432 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
     }
 #undef TB_SEL
 #undef TB_SEL_R
+}
+
+// ===================================================================================================
+// Few, long problems (one sequence, or a small batch, at 32K tokens and beyond): a thread-block cluster
+// per problem, built from the same pieces as the kernel above.  Every block of the cluster places the
+// first digit from the same 64-row sample, streams its share of the rows, parks the keys in the
+// workspace row and keeps, on chip, only each row's first digit (2 bytes) and the digit histogram.
+// Barrier 1.  Every block sums the cluster's histograms through distributed shared memory, finds the
+// threshold bin itself, turns its own digits into a bitmask, fetches the full keys of its few rows
+// in the threshold bin and sends them, with its count of selected rows, to every peer.  Barrier 2.
+// Every block ranks the (tiny) list itself, knows every rank's count, and writes its part of the
+// ascending list.  Two cluster barriers after the stream, no serial section, 2 bytes of shared memory
+// per row (so two blocks per SM at 128K tokens).  A crowded or open-below threshold bin sends the
+// problem to the general path, run by rank 0 on the parked keys.
+constexpr int kCwListCap = 256;      // keys of the threshold bin set aside per problem (more: the bin is cut again)
+constexpr int kCwMaxCluster = 8;
+
+struct __align__(16) CwSmem {
+    WaveSmem w;
+    int take[kCwMaxCluster];         // per rank: rows its bitmask selects by the first digit alone
+    int n_in[kCwMaxCluster];         // per rank: entries in its region of the list
+    int winners[kCwMaxCluster];      // per rank: list entries that made it
+    int my_n;
+    int fine8[8];
+    int coarse[kThreads];            // this block's histogram, 8 first-digit bins per entry
+};
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+template <typename P>
+__device__ __forceinline__ P* peer_ptr(P* p, int rank) {       // the same shared-memory object in block `rank` of the cluster
+    uint64_t out;
+    asm volatile("mapa.u64 %0, %1, %2;" : "=l"(out) : "l"(reinterpret_cast<uint64_t>(p)), "r"(rank));
+    return reinterpret_cast<P*>(out);
+}
+
+template <typename T, int DP, int RED>
+__global__ void __launch_bounds__(kThreads, 2)
+    select_cw_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut, SelectArgs a,
+                     int tiles_per_cta, int n_stages, int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt,
+                     int32_t* __restrict__ status, uint32_t* __restrict__ keys_g) {
+    constexpr int RB = DP * Elem<T>::kBytes;
+    constexpr int NCH = RB / 16;
+    constexpr uint32_t kTileBytes = kRows * RB;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    const int ring_bytes = n_stages * (int)kTileBytes;
+    int* hist = reinterpret_cast<int*>(stage_base + ring_bytes);                 // this block's first-digit histogram
+    uint16_t* bins = reinterpret_cast<uint16_t*>(hist + kDigitBins);             // first digit of every row of this block
+    uint32_t* mask = reinterpret_cast<uint32_t*>(bins + (size_t)tiles_per_cta * kRows);   // tiles_per_cta * 8 words
+    CwSmem* cs = reinterpret_cast<CwSmem*>(mask + tiles_per_cta * (kRows / 32));
+    WaveSmem* sm = &cs->w;
+    // after the stream the ring holds the list (one region per rank)
+    uint2* list = reinterpret_cast<uint2*>(stage_base);
+
+    unsigned C, rank;
+    asm volatile("mov.u32 %0, %%cluster_nctaid.x;" : "=r"(C));
+    asm volatile("mov.u32 %0, %%cluster_ctaid.x;" : "=r"(rank));
+    const int tid = threadIdx.x, lane = tid & 31;
+    int ll, s, h;
+    decode_unit(gm, ut, blockIdx.y, ll, s, h);
+    const int L = ut.len[ll * ut.n_seq + s];
+    const int lo = min(a.sinks, L), ncand = max(lo, L - a.recent) - lo, k = min(a.budget, ncand);
+    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t dst_row = a.dst_is_state ? cu : (size_t)blockIdx.y;
+    int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
+    int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
+    // uniform over the cluster: all of its blocks leave together
+    if (k <= 0) {
+        if (rank == 0 && tid == 0) *cnt_dst = 0;
+        return;
+    }
+    if (k == ncand) {
+        for (int i = rank * kThreads + tid; i < ncand; i += C * kThreads) idx_dst[i] = lo + i;
+        if (rank == 0 && tid == 0) *cnt_dst = k;
+        return;
+    }
+
+#ifdef TB_PHASE_TIMING
+    const unsigned long long tc0 = wave_now();
+#define CW_MARK(i) do { if (tid == 0) { const int bb = blockIdx.y * gridDim.x + blockIdx.x; if (bb < 1024) g_wave_ns[(i) & 3][bb] = ((i) < 4 ? 0 : 0) + wave_now() - ((i) == 0 ? 0 : tc0); } } while (0)
+#else
+#define CW_MARK(i) do {} while (0)
+#endif
+    CW_MARK(0);
+    for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
+    if (tid == 0) {
+        prefetch_tmap(&tmap);
+        for (int i = 0; i < n_stages; ++i) mbar_init(&sm->full[i], 1);
+        fence_mbar_init();
+        cs->my_n = 0;
+    }
+    if (tid < kCwMaxCluster) cs->winners[tid] = 0;
+    __syncthreads();
+
+    const int n_tiles = (ncand + kRows - 1) / kRows;
+    const int tile0 = rank * tiles_per_cta, my_tiles = max(0, min(tiles_per_cta, n_tiles - tile0));
+    const int slot0 = tile0 * kRows;                   // candidate index of this block's first row
+    const int n_local = max(0, min(my_tiles * kRows, ncand - slot0));
+    const long long row_base = (long long)cu * gm.max_seq_len + lo;              // row of candidate 0
+    uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255);
+    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
+
+    // sample row and query first, then the ring's opening requests (see the kernel above)
+    const bool sampled = ncand >= kMinSampled;
+    uint4 srow[NCH];
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) srow[c] = make_uint4(0u, 0u, 0u, 0u);
+    if (sampled && tid < kSampleRows) {
+        const int slot = (int)(((long long)tid * ncand) / kSampleRows);
+        const uint4* rowp = reinterpret_cast<const uint4*>(kimp + (size_t)(row_base + slot) * RB);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
+    }
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    if (RED != TB_GROUP_SUM) __syncthreads();
+    if (tid == 0)
+        for (int i = 0; i < n_stages && i < my_tiles; ++i) {
+            mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
+            tma_load_2d_hint(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + slot0 + (long long)i * kRows), &sm->full[i], stream_policy);
+        }
+    Digit dg = {0u, 21};
+    if (sampled) {                                     // identical in every block of the cluster: same rows, same arithmetic
+        if (tid < kSampleRows) sm->sample[tid] = order_key(scorer.score([&](int c) { return srow[c]; }));
+        __syncthreads();
+        if (tid < kSampleRows) {
+            const uint32_t mine = sm->sample[tid];
+            const uint4* s4 = reinterpret_cast<const uint4*>(sm->sample);
+            int r = 0;
+#pragma unroll 8
+            for (int j4 = 0; j4 < kSampleRows / 4; ++j4) {
+                const uint4 x = s4[j4];
+                const int j = j4 * 4;
+                r += (x.x > mine) | ((x.x == mine) & (j < tid));
+                r += (x.y > mine) | ((x.y == mine) & (j + 1 < tid));
+                r += (x.z > mine) | ((x.z == mine) & (j + 2 < tid));
+                r += (x.w > mine) | ((x.w == mine) & (j + 3 < tid));
+            }
+            const float p = (float)k / (float)ncand, mean = p * kSampleRows, sd = sqrtf(mean * (1.f - p));
+            const int r_hi = max(0, (int)floorf(mean - 6.f * sd) - 3), r_lo = min(kSampleRows - 1, (int)ceilf(mean + 6.f * sd) + 3);
+            if (r == r_hi) sm->s_hi = mine;
+            if (r == r_lo) sm->s_lo = mine;
+        }
+        __syncthreads();
+        const uint32_t s_lo = sm->s_lo, s_hi = sm->s_hi;
+        uint32_t range = s_hi - s_lo;
+        // room above the highest bracketing sample; twice as much when that is the sample's largest key
+        // (few sample keys above the threshold: it may well lie beyond them)
+        const float pm = (float)k / (float)ncand * kSampleRows;
+        const bool clipped = (int)floorf(pm - 6.f * sqrtf(pm * (1.f - (float)k / (float)ncand))) - 3 <= 0;
+        const uint64_t wide = (uint64_t)range * (clipped ? 3u : 1u) + (range >> 1);
+        range = wide > 0xffffffffull ? 0xffffffffu : (uint32_t)wide;
+        dg.base = s_lo, dg.shift = 0;
+        while ((range >> dg.shift) >= 2046u) ++dg.shift;
+    }
+
+    CW_MARK(1);
+    // ---- stream: score, park the key, keep the first digit ---------------------------------------------
+    bool timed_out = false;
+    int st = 0;
+    uint32_t phase = 0;
+    for (int i = 0; i < my_tiles; ++i) {
+        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;
+        const unsigned char* tile = stage_base + st * kTileBytes;
+        const int slot = i * kRows + tid;
+        uint16_t b = 0;                                // rows past the end: below everything
+        if (slot < n_local) {
+            const uint32_t off = tid * RB;
+            const float sc = scorer.score([&](int c) {
+                uint32_t o = off + c * 16;
+                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
+                return *reinterpret_cast<const uint4*>(tile + o);
+            });
+            const uint32_t key = order_key(sc);
+#ifdef TB_NOHINT
+            keys_unit[slot0 + slot] = key;
+#else
+            st_global_hint(keys_unit + slot0 + slot, key, keep_policy);
+#endif
+            b = (uint16_t)dg.bin(key);
+            hist_add(&hist[b]);
+        }
+        bins[slot] = b;
+        __syncthreads();
+        if (tid == 0 && i + n_stages < my_tiles) {
+            fence_proxy_async();
+            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+            tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + slot0 + (long long)(i + n_stages) * kRows),
+                             &sm->full[st], stream_policy);
+        }
+        if (++st == n_stages) st = 0, phase ^= 1u;
+    }
+    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    __syncthreads();
+    CW_MARK(2);
+#ifdef TB_PHASE_TIMING
+    unsigned long long tp = wave_now();
+#define CW_PH(i) do { if (tid == 0) { unsigned long long tn = wave_now(); atomicAdd(&g_cw_ns[i], tn - tp); tp = tn; } } while (0)
+#else
+#define CW_PH(i) do {} while (0)
+#endif
+    // ---- threshold bin: the cluster's histogram in two levels ---------------------------------------------
+    // Every block sums, through distributed shared memory, first a coarse histogram (256 bins of 8
+    // first-digit bins each: one remote word per thread and peer), finds the coarse bin of the threshold,
+    // then the 8 fine bins inside it.  If the threshold's bin holds more keys than the list takes (a
+    // bracket stretched by an outlier in the sample, the open bin above it, many near-equal scores), the
+    // bin itself is cut into 2046 slices and the rows inside it are re-digitised from their parked keys:
+    // another round, two more barriers, only for the cluster that needs it.
+    int bin = 0, krem = k, bc = 0;
+    bool exact = false;
+    uint32_t bin_base = 0;
+    Digit cur = dg;
+#pragma unroll 1
+    for (int level = 0;; ++level) {
+        cs->coarse[tid] = [&] {
+            const int4* hp = reinterpret_cast<const int4*>(hist + tid * 8);
+            const int4 x0 = hp[0], x1 = hp[1];
+            return x0.x + x0.y + x0.z + x0.w + x1.x + x1.y + x1.z + x1.w;
+        }();
+        __syncthreads();
+        cluster_sync_all();                            // every block's histograms are complete (level 0: every ring idle)
+        if (level == 0) CW_PH(0);
+        int mine = 0;
+        for (unsigned r = 0; r < C; ++r) mine += peer_ptr(cs, (int)r)->coarse[tid];
+        int total;
+        const int excl = wave_excl_scan(mine, sm->warp_a, total);
+        const int above = total - excl - mine;         // keys in coarse bins above this thread's
+        if (above < krem && krem <= above + mine) sm->bc_bin = tid, sm->bc_krem = krem - above;   // exactly one thread
+        __syncthreads();
+        const int cb = sm->bc_bin, kc = sm->bc_krem;
+        if (tid < 8) {
+            int f = 0;
+            for (unsigned r = 0; r < C; ++r) f += peer_ptr(hist, (int)r)[cb * 8 + tid];
+            cs->fine8[tid] = f;
+        }
+        __syncthreads();
+        {
+            int run = 0, e = 7;
+            while (e > 0 && run + cs->fine8[e] < kc) run += cs->fine8[e], --e;
+            bin = cb * 8 + e, bc = cs->fine8[e], krem = kc - run;
+        }
+        exact = bc == krem;
+        bin_base = cur.base + ((uint32_t)(bin - 1) << cur.shift);
+        __syncthreads();                               // bc_*, fine8 and warp_a may be reused
+        if (exact || bc <= kCwListCap) break;
+        const bool open_top = bin == 2047;
+        if (bin == 0 || level == 3 || (cur.shift == 0 && !open_top)) {
+            // below the bracket, or more equal keys than the list takes: general path on the parked keys, rank 0 alone
+            cluster_sync_all();                        // nobody reads a peer's histogram any more
+            if (rank == 0)
+                wave_general(hist, sm, keys_unit, reinterpret_cast<uint4*>(stage_base), ring_bytes / 16, ncand, k, lo, idx_dst, cnt_dst);
+            return;
+        }
+        cluster_sync_all();                            // every block has read what it needs of the old histograms
+        // the open bin above the bracket: first try twice the bracket's width again (what lies beyond
+        // lands in the new digit's own open bin), then everything up to the largest key
+        const uint64_t twice = (uint64_t)2 * (2046ull << cur.shift);
+        const uint32_t rest = 0xffffffffu - bin_base;
+        const uint32_t range = open_top ? (level == 0 && twice < rest ? (uint32_t)twice : rest) : (1u << cur.shift) - 1u;
+        Digit nxt = {bin_base, 0};
+        while ((range >> nxt.shift) >= 2046u) ++nxt.shift;
+        for (int i = tid; i < kDigitBins; i += kThreads) hist[i] = 0;
+        __syncthreads();
+        for (int sl = tid; sl < my_tiles * kRows; sl += kThreads) {   // rows above the bin: 0xffff from now on; below: 0
+            const int d = bins[sl];
+            uint16_t nb = d > bin ? (uint16_t)0xffff : (uint16_t)0;
+            if (d == bin) {
+                nb = (uint16_t)nxt.bin(__ldcg(keys_unit + slot0 + sl));   // >= 1: the key is not below the bin's base
+                hist_add(&hist[nb]);
+            }
+            bins[sl] = nb;
+        }
+        cur = nxt;
+        __syncthreads();
+    }
+    CW_PH(1);
+
+    // ---- own digits -> bitmask; own rows of the threshold bin -> every peer's list ------------------------
+    int my_take = 0;
+    {
+        const uint4* bins4 = reinterpret_cast<const uint4*>(bins);
+        for (int v = tid; v < my_tiles * (kRows / 8); v += kThreads) {          // 8 digits per 16-byte load
+            const uint4 x = bins4[v];
+            const uint32_t w4[4] = {x.x, x.y, x.z, x.w};
+            uint32_t take = 0, eq = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int d = (int)((w4[e >> 1] >> (16 * (e & 1))) & 0xffffu);
+                take |= (uint32_t)(d > bin || (d == bin && exact)) << e;
+                eq |= (uint32_t)(d == bin && !exact) << e;
+            }
+            my_take += __popc(take);
+            uint32_t word = take << (8 * (lane & 3));  // four lanes' bytes make a mask word
+            word |= __shfl_xor_sync(0xffffffffu, word, 1);
+            word |= __shfl_xor_sync(0xffffffffu, word, 2);
+            if ((lane & 3) == 0) mask[v >> 2] = word;
+            while (eq) {                               // rare: a handful of rows per block
+                const int e = __ffs(eq) - 1;
+                eq &= eq - 1;
+                const int ls = v * 8 + e;
+                const int i = atomicAdd(&cs->my_n, 1);
+                const uint2 ent = make_uint2(__ldcg(keys_unit + slot0 + ls) - bin_base, (uint32_t)(slot0 + ls));
+                for (unsigned r = 0; r < C; ++r) peer_ptr(list, (int)r)[rank * kCwListCap + i] = ent;
+            }
+        }
+    }
+    {
+        int total;
+        wave_excl_scan(my_take, sm->warp_a, total);
+        __syncthreads();
+        if (tid < (int)C) peer_ptr(cs, tid)->take[rank] = total, peer_ptr(cs, tid)->n_in[rank] = cs->my_n;
+    }
+    CW_PH(2);
+    cluster_sync_all();                                // barrier 2: lists and counts are everywhere
+    CW_PH(3);
+
+    // ---- every block ranks the list itself ------------------------------------------------------------
+    if (!exact) {
+        int r_of = 0, i_of = tid;                      // thread t takes entry t of the concatenated regions
+        while (r_of < (int)C && i_of >= cs->n_in[r_of]) i_of -= cs->n_in[r_of], ++r_of;
+        if (r_of < (int)C) {
+            const uint2 it = list[r_of * kCwListCap + i_of];
+            int before = 0;                            // larger key, or equal key at a lower position
+            for (unsigned r = 0; r < C; ++r)
+                for (int j = 0; j < cs->n_in[r]; ++j) {
+                    const uint2 o = list[r * kCwListCap + j];
+                    before += (o.x > it.x) | ((o.x == it.x) & (o.y < it.y));
+                }
+            if (before < krem) {
+                atomicAdd(&cs->winners[r_of], 1);
+                if (r_of == (int)rank) {
+                    const int ls = (int)it.y - slot0;
+                    atomicOr(&mask[ls >> 5], 1u << (ls & 31));
+                }
+            }
+        }
+        __syncthreads();
+    }
+    CW_PH(4);
+    int out_base = 0;
+    for (unsigned r = 0; r < rank; ++r) out_base += cs->take[r] + cs->winners[r];
+    {
+        const int n_words = my_tiles * (kRows / 32);
+        const int per = (n_words + kThreads - 1) / kThreads;
+        const int w0 = min(n_words, tid * per), w1 = min(n_words, w0 + per);
+        int cnt = 0;
+        for (int w = w0; w < w1; ++w) cnt += __popc(mask[w]);
+        int total;
+        int o = out_base + wave_excl_scan(cnt, sm->warp_a, total);
+        for (int w = w0; w < w1; ++w) {
+            uint32_t bits = mask[w];
+            while (bits) {
+                const int b = __ffs(bits) - 1;
+                bits &= bits - 1;
+                if (o < k) idx_dst[o] = lo + slot0 + w * 32 + b;
+                ++o;
+            }
+        }
+    }
+    if (rank == 0 && tid == 0) *cnt_dst = k;
+    CW_PH(5);
+#ifdef TB_PHASE_TIMING
+    if (tid == 0) atomicAdd(&g_cw_ns[7], 1ull);
+#endif
+    CW_MARK(3);
+}
+
+cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
+    const Geom& gm = c->geom;
+    const int n_units = ut.layer_count * ut.n_seq * gm.Hkv;
+    int max_cand = 0;
+    for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) {
+        const int L = ut.len[i], lo = a.sinks < L ? a.sinks : L, hi = L - a.recent > lo ? L - a.recent : lo;
+        if (hi - lo > max_cand) max_cand = hi - lo;
+    }
+    const int n_tiles = (max_cand + kRows - 1) / kRows;
+    // cluster size: two resident blocks per SM over the whole GPU, at least 8 tiles per block
+    int C = 2 * c->sm_count / n_units;
+    if (C > kCwMaxCluster) C = kCwMaxCluster;
+    while (C > 1 && n_tiles / C < 8) --C;
+    if (C < 1) C = 1;
+    const int tiles_per_cta = (n_tiles + C - 1) / C > 0 ? (n_tiles + C - 1) / C : 1;
+    const int tile_bytes = kRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
+    const size_t fixed = 1024 + kDigitBins * sizeof(int) + (size_t)tiles_per_cta * kRows * 2 + (size_t)tiles_per_cta * (kRows / 32) * 4 +
+                         sizeof(CwSmem);
+    const size_t ring_min = (size_t)C * kCwListCap * sizeof(uint2);   // list regions
+    const size_t budget = (size_t)(C * n_units > c->sm_count ? 113 : 224) * 1024;
+    if (fixed + ring_min > 224 * 1024) return cudaErrorInvalidConfiguration;
+    int n_stages = fixed < budget ? (int)((budget - fixed) / tile_bytes) : 0;
+    if (n_stages > kStagesMax) n_stages = kStagesMax;
+    if (n_stages < 2) n_stages = 2;
+    while ((size_t)n_stages * tile_bytes < ring_min) ++n_stages;
+    const size_t smem = fixed + (size_t)n_stages * tile_bytes;
+    if (smem > 226 * 1024 || n_stages > kStagesMax) return cudaErrorInvalidConfiguration;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(C, n_units, 1), cfg.blockDim = dim3(kThreads, 1, 1), cfg.dynamicSmemBytes = smem, cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C, attr[0].val.clusterDim.y = 1, attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+#define TB_CW_R(T, DP, RED)                                                                                              \
+    do {                                                                                                                 \
+        static unsigned char seen[64];                                                                                   \
+        if (first_use_on_this_device(seen)) {                                                                            \
+            cudaError_t e = cudaFuncSetAttribute(select_cw_kernel<T, DP, RED>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                 226 * 1024);                                                            \
+            if (e != cudaSuccess) return e;                                                                              \
+        }                                                                                                                \
+        return cudaLaunchKernelEx(&cfg, select_cw_kernel<T, DP, RED>, c->kimp_map, (const unsigned char*)c->kimp, gm, ut, a, \
+                                  tiles_per_cta, n_stages, c->st.idx, c->st.cnt, c->st.status, c->wk.sel_keys);          \
+    } while (0)
+#define TB_CW(T, DP)                                                \
+    do {                                                            \
+        if (a.reduce == TB_GROUP_MAX) TB_CW_R(T, DP, TB_GROUP_MAX); \
+        else TB_CW_R(T, DP, TB_GROUP_SUM);                          \
+    } while (0)
+    if (gm.dtype == TB_BF16) {
+        if (gm.dp == 32) TB_CW(__nv_bfloat16, 32); else TB_CW(__nv_bfloat16, 16);
+    } else {
+        if (gm.dp == 32) TB_CW(float, 32); else TB_CW(float, 16);
+    }
+#undef TB_CW
+#undef TB_CW_R
 }
 
 }  // namespace tb

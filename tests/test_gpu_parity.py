@@ -554,3 +554,34 @@ def test_many_problem_selection_with_neighbours_and_attention(H, nmode):
     case = H.Case(w)
     p = tb().select_params(w.budget, w.sinks, w.recent, radius=1, nmode=nmode)
     full_pipeline_check(H, case, p)
+
+
+def test_long_problem_cluster_kernel_unusual_distributions(H):
+    """Problems beyond 48K candidates take the cluster kernel that parks its keys (70001 tokens, 2 heads
+    here).  Cases for each way its threshold search can go: a bin cut again, the open bin above the
+    sampled bracket, the open bin below it and massive ties (general path on the parked keys)."""
+    r = np.random.Generator(np.random.PCG64(80))
+    L = 70001
+    _crafted_scores_case(H, _bf16_exact(r.standard_normal((2, L))), budget=3000, sinks=3, recent=40)
+    # every score equal; a few distinct values (tens of thousands of ties at the threshold)
+    _crafted_scores_case(H, np.full((2, L), 2.25, np.float32), budget=500, sinks=5, recent=9)
+    _crafted_scores_case(H, r.integers(0, 4, size=(2, L)).astype(np.float32), budget=20000)
+    # a hundred huge scores where the sample does not look, budget below their number: the threshold is far
+    # above the bracket
+    s = _bf16_exact(r.standard_normal((2, L)))
+    s[:, 11::701] = _bf16_exact(1000.0 + 8.0 * r.integers(0, 64, size=s[:, 11::701].shape))
+    _crafted_scores_case(H, s, budget=37)
+    # 3000 scores just above everything else, spread so thinly that the bracket's top slice holds them all
+    s = _bf16_exact(r.standard_normal((2, L)))
+    s[:, 5::23] = _bf16_exact(6.0 + 0.5 * r.random(s[:, 5::23].shape))
+    _crafted_scores_case(H, s, budget=1500)
+    # the sampled positions hold large scores, the rest small ones, and the budget reaches deep into the
+    # small ones: the threshold lies below the bracket
+    s = _bf16_exact(0.01 * r.standard_normal((2, L)))
+    for i in range(64):
+        s[:, (i * L) // 64] = 50.0 + i
+    _crafted_scores_case(H, s, budget=30000)
+    # ~400 binades, both signs
+    expo = r.integers(-100, 101, size=(2, L))
+    sign = r.choice([-1.0, 1.0], size=(2, L))
+    _crafted_scores_case(H, (sign * np.exp2(expo)).astype(np.float32), budget=9000)

@@ -26,7 +26,7 @@
  *
  * Device layouts (row-major, element = kv_dtype)
  *   kv    [n_layers][max_batch][Hkv][max_seq_len][2][D]   K row then V row of a token, adjacent
- *   kimp  [n_layers][max_batch][Hkv][max_seq_len][d']
+ *   kimp  [n_layers][max_batch][Hkv][max_seq_len][d']     ([1] in place of [Hkv] under TB_SCOPE_LAYER)
  *   W_K   [Hkv][D][d'] per layer (one D x d' matrix per layer AND per KV head)
  *   index lists: int32 rows of tb_index_capacity() entries, ascending token positions
  */
@@ -54,9 +54,25 @@ typedef enum {
 
 typedef enum { TB_F32 = 0, TB_BF16 = 1 } tb_dtype;
 /* How the g importance queries of a GQA group become one ranking per KV head: a token's score is the
- * sum (default) or the largest of the group's g head scores.  TB_PER_QHEAD (one list per query head, no
- * row sharing) is named for completeness; the library answers TB_ERR_UNSUPPORTED to it. */
+ * sum (default) or the largest of the group's g head scores.  TB_PER_QHEAD asks for no reduction: it is
+ * accepted by a context whose lists are per query head (TB_SCOPE_Q_HEAD below), where it is the only
+ * meaning there is, and refused with TB_ERR_UNSUPPORTED by a context whose lists are per KV head.  On a
+ * context with one importance query per list (TB_SCOPE_Q_HEAD, TB_SCOPE_LAYER) all three mean the same. */
 typedef enum { TB_GROUP_SUM = 0, TB_GROUP_MAX = 1, TB_PER_QHEAD = 2 } tb_group_reduce;
+/* Which heads share one index list (paper Sec. 3.1: importance is predicted per head; App. "additional
+ * evaluation": a head-less predictor with one importance per token and layer).  Fixed per context,
+ * since it sizes the projected-key cache and the lists:
+ *   TB_SCOPE_KV_HEAD  one list per KV head; the g query heads of a group share the gathered rows.
+ *                     q_imp [..][Hq][d'], kimp [..][Hkv][max_seq_len][d'], lists [..][Hkv].
+ *   TB_SCOPE_Q_HEAD   one list per query head, ranked by that head's importance query against its KV
+ *                     head's projected keys; no row sharing in attention.  q_imp [..][Hq][d'], kimp as
+ *                     above, lists [..][Hq].
+ *   TB_SCOPE_LAYER    one list per layer, shared by every head.  One importance query per layer,
+ *                     q_imp [..][1][d'], and one projected key per token, kimp [..][1][max_seq_len][d'] =
+ *                     sum over KV heads h of K[h] . W_K[h] (the [Hkv*D] x d' projection of the token's
+ *                     concatenated key); lists [..][1].
+ * In the calls below, "[Hl]" stands for the number of lists per (layer, sequence): Hkv, Hq or 1. */
+typedef enum { TB_SCOPE_KV_HEAD = 0, TB_SCOPE_Q_HEAD = 1, TB_SCOPE_LAYER = 2 } tb_list_scope;
 /* Neighbour fetching (Sec. 3.4): DILATE = every position within +-radius of a selected one;
  * CLUSTER = runs of consecutive selected positions get radius*len extra positions just outside the
  * run (ceil half after it, floor half before it). */
@@ -70,6 +86,7 @@ typedef struct {
     int32_t max_budget;    /* largest `budget` any select call will use                      */
     int32_t max_radius;    /* largest neighbour radius; lists hold (2*max_radius+1)*max_budget */
     int32_t device;        /* CUDA device ordinal the regions live on                        */
+    int32_t list_scope;    /* tb_list_scope; 0 = one list per KV head                        */
 } tb_config;
 
 typedef struct {
@@ -135,21 +152,23 @@ tb_status tb_project_keys(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count,
 
 /* Sec. 3.4 / App. E importance scores of ALL projected tokens, materialised:
  * scores_dev[i][h][t] = score_scale * sum_j qr[i][h][j] * K_imp[seq_i][h][t][j], t < projected length,
- * row stride max_seq_len, entries past the projected length untouched.  q_imp_dev [n_seq][Hq][d'] fp32;
- * qr = sum of the g importance queries that share KV head h (TB_GROUP_SUM; the other modes return
- * TB_ERR_UNSUPPORTED).  The fast path (tb_select_topk) never materialises scores. */
+ * h < Hl, row stride max_seq_len, entries past the projected length untouched.  q_imp_dev [n_seq][Hq][d']
+ * fp32 ([n_seq][1][d'] under TB_SCOPE_LAYER); qr = sum of the importance queries that share list h
+ * (TB_GROUP_SUM), or the score is the largest of their dot products (TB_GROUP_MAX).  The fast path
+ * (tb_select_topk) never materialises scores. */
 tb_status tb_score_tokens(tb_ctx* ctx, int32_t layer, const int32_t* seq_ids, int32_t n_seq,
                           const float* q_imp_dev, int32_t reduce, float score_scale, float* scores_dev, void* stream);
 
 /* Sec. 4 "Token Selection Policy" + Sec. 3.4 interval / neighbour fetching, fused with scoring, for
  * layers [layer_begin, layer_begin+layer_count) (Sec. 3.3: predictor work is batched over the
  * consumer layers of a producer).  If params->step % params->interval != 0 nothing is launched and
- * the stored lists stay (stale reuse).  Otherwise, per (layer, sequence, KV head): candidates are
+ * the stored lists stay (stale reuse).  Otherwise, per (layer, sequence, list): candidates are
  * positions [min(S,L), max(min(S,L), L-W)); the `budget` highest scores are kept (all candidates if
  * fewer), equal scores resolved toward the LOWER position, -0.0 == +0.0; the list is expanded by the
  * neighbour rule, clipped to the candidates, and stored ascending in the context.
- * q_imp_dev: [layer_count][n_seq][Hq][d'] fp32.  idx_out_dev / cnt_out_dev (optional, may be NULL):
- * copies of the stored lists, [layer_count][n_seq][Hkv][tb_index_capacity()] and [..][Hkv].
+ * q_imp_dev: [layer_count][n_seq][Hq][d'] fp32 ([..][1][d'] under TB_SCOPE_LAYER).  idx_out_dev /
+ * cnt_out_dev (optional, may be NULL): copies of the stored lists, [layer_count][n_seq][Hl][tb_index_capacity()]
+ * and [..][Hl].
  * TB_ERR_UNPROJECTED if a candidate range is not fully projected; TB_ERR_CAPACITY if budget or radius
  * exceed the configured maxima. */
 tb_status tb_select_topk(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, const int32_t* seq_ids,
@@ -158,7 +177,9 @@ tb_status tb_select_topk(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, 
 
 /* Sec. 3.3 attention of one decode token per listed sequence over
  * sinks [0,min(S,L)) + index list + window [max(min(S,L),L-W), L) of the full cache, each gathered
- * K/V row shared by the g query heads of its KV head; split over the rows with a fixed partition and
+ * K/V row shared by the g query heads of its KV head (by no one under TB_SCOPE_Q_HEAD, where every
+ * query head gathers its own list's rows; under TB_SCOPE_LAYER every KV head reads the layer's one
+ * list); split over the rows with a fixed partition and
  * merged in a fixed order (bit-reproducible).  q_dev [layer_count][n_seq][Hq][D] kv_dtype;
  * out_dev [layer_count][n_seq][Hq][D] fp32; lse_dev (optional) [layer_count][n_seq][Hq] natural-log
  * sum-exp of the scaled logits.  idx_dev/cnt_dev: caller lists laid out like tb_select_topk's

@@ -13,6 +13,7 @@ TB_ERR_INVALID_ARG, TB_ERR_UNSUPPORTED, TB_ERR_CAPACITY, TB_ERR_UNPROJECTED = -1
 TB_ERR_STATE, TB_ERR_CUDA, TB_ERR_TIMEOUT, TB_ERR_BAD_INDEX = -5, -6, -7, -8
 TB_F32, TB_BF16 = 0, 1
 TB_GROUP_SUM, TB_GROUP_MAX, TB_PER_QHEAD = 0, 1, 2
+TB_SCOPE_KV_HEAD, TB_SCOPE_Q_HEAD, TB_SCOPE_LAYER = 0, 1, 2
 TB_NEIGHBOR_DILATE, TB_NEIGHBOR_CLUSTER = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -25,7 +26,8 @@ EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb
 
 class tb_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "n_q_heads", "n_kv_heads", "head_dim", "imp_dim", "kv_dtype",
-                                         "max_batch", "max_seq_len", "max_budget", "max_radius", "device")]
+                                         "max_batch", "max_seq_len", "max_budget", "max_radius", "device",
+                                         "list_scope")]
 
 
 class tb_select_params(C.Structure):
@@ -140,10 +142,13 @@ class Context:
     names of the C entry points and only marshal arguments."""
 
     def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, imp_dim, kv_dtype, max_batch, max_seq_len,
-                 max_budget, max_radius=0, device=0, kv_on_host=False):
+                 max_budget, max_radius=0, device=0, kv_on_host=False, list_scope=TB_SCOPE_KV_HEAD):
         L = lib()
         self.cfg = tb_config(n_layers, n_q_heads, n_kv_heads, head_dim, imp_dim, kv_dtype, max_batch, max_seq_len,
-                             max_budget, max_radius, device)
+                             max_budget, max_radius, device, list_scope)
+        # heads of the projected-key cache / lists per (layer, sequence) under the selection scope
+        self.n_key_heads = 1 if list_scope == TB_SCOPE_LAYER else n_kv_heads
+        self.n_lists = {TB_SCOPE_KV_HEAD: n_kv_heads, TB_SCOPE_Q_HEAD: n_q_heads, TB_SCOPE_LAYER: 1}.get(list_scope, n_kv_heads)
         sizes = [C.c_size_t() for _ in range(4)]
         st = L.tb_query_sizes(C.byref(self.cfg), *[C.byref(s) for s in sizes])
         if st != TB_OK:
@@ -159,7 +164,7 @@ class Context:
             torch.empty(self.sizes[0] // es, dtype=dt, device=self.device)
         self.kv = kv_flat.view(n_layers, max_batch, n_kv_heads, max_seq_len, 2, head_dim)
         self.kimp = torch.empty(self.sizes[1] // es, dtype=dt, device=self.device).view(
-            n_layers, max_batch, n_kv_heads, max_seq_len, imp_dim)
+            n_layers, max_batch, self.n_key_heads, max_seq_len, imp_dim)
         self.state = torch.empty(self.sizes[2], dtype=torch.uint8, device=self.device)
         self.workspace = torch.empty(self.sizes[3], dtype=torch.uint8, device=self.device)
         h = C.c_void_p()

@@ -21,6 +21,14 @@ struct Layout {
     int idx_cap, sel_stride;
 };
 
+// Heads per (layer, sequence) of the projected-key cache (hi), the index lists (hl) and the
+// attention units (ha) under the configuration's selection scope.
+void scope_heads(const tb_config* c, int* hi, int* hl, int* ha) {
+    *hi = c->list_scope == TB_SCOPE_LAYER ? 1 : c->n_kv_heads;
+    *hl = c->list_scope == TB_SCOPE_LAYER ? 1 : c->list_scope == TB_SCOPE_Q_HEAD ? c->n_q_heads : c->n_kv_heads;
+    *ha = c->list_scope == TB_SCOPE_Q_HEAD ? c->n_q_heads : c->n_kv_heads;
+}
+
 tb_status check_config(const tb_config* c) {
     if (!c) return TB_ERR_INVALID_ARG;
     if (c->n_layers <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->max_batch <= 0 || c->max_seq_len <= 0 ||
@@ -28,6 +36,7 @@ tb_status check_config(const tb_config* c) {
         return TB_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads != 0) return TB_ERR_INVALID_ARG;
     if (c->kv_dtype != TB_F32 && c->kv_dtype != TB_BF16) return TB_ERR_INVALID_ARG;
+    if (c->list_scope != TB_SCOPE_KV_HEAD && c->list_scope != TB_SCOPE_Q_HEAD && c->list_scope != TB_SCOPE_LAYER) return TB_ERR_INVALID_ARG;
     if (c->head_dim != 128) return TB_ERR_UNSUPPORTED;
     if (c->imp_dim != 16 && c->imp_dim != 32) return TB_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > kMaxGroup) return TB_ERR_UNSUPPORTED;
@@ -40,10 +49,12 @@ tb_status check_config(const tb_config* c) {
 
 void compute_layout(const tb_config* c, Layout* l) {
     const size_t es = elem_size(c->kv_dtype);
-    const size_t units = (size_t)c->n_layers * c->max_batch * c->n_kv_heads;
-    const size_t slots = units * c->max_seq_len;
-    l->kv_bytes = slots * 2 * c->head_dim * es;
-    l->kimp_bytes = slots * c->imp_dim * es;
+    int hi, hl, ha;
+    scope_heads(c, &hi, &hl, &ha);
+    const size_t pairs = (size_t)c->n_layers * c->max_batch;
+    const size_t units = pairs * hl;                                   // index lists
+    l->kv_bytes = pairs * c->n_kv_heads * c->max_seq_len * 2 * c->head_dim * es;
+    l->kimp_bytes = pairs * hi * c->max_seq_len * c->imp_dim * es;
     l->idx_cap = (int)align_up((size_t)(2 * c->max_radius + 1) * c->max_budget, 4);
     l->sel_stride = (int)align_up((size_t)c->max_budget, 4);
     size_t o = 0;
@@ -51,7 +62,7 @@ void compute_layout(const tb_config* c, Layout* l) {
     l->off_idx = o, o = align_up(o + units * l->idx_cap * 4, 256);
     l->off_cnt = o, o = align_up(o + units * 4, 256);
     l->off_status = o, o = align_up(o + 4, 256);
-    l->off_counter = o, o = align_up(o + units * 4, 256);
+    l->off_counter = o, o = align_up(o + pairs * ha * 4, 256);
     l->state_bytes = o;
     const size_t units_q = (size_t)c->n_layers * c->max_batch * c->n_q_heads;
     o = 0;
@@ -79,7 +90,7 @@ tb_status make_kimp_map(tb_ctx* c) {
     const tb_config& g = c->cfg;
     const int es = elem_size(g.kv_dtype);
     const int row_bytes = g.imp_dim * es;
-    cuuint64_t dims[2] = {(cuuint64_t)g.imp_dim, (cuuint64_t)g.n_layers * g.max_batch * g.n_kv_heads * g.max_seq_len};
+    cuuint64_t dims[2] = {(cuuint64_t)g.imp_dim, (cuuint64_t)g.n_layers * g.max_batch * c->geom.Hi * g.max_seq_len};
     cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
     cuuint32_t box[2] = {(cuuint32_t)g.imp_dim, 256u};
     cuuint32_t estr[2] = {1u, 1u};
@@ -90,6 +101,15 @@ tb_status make_kimp_map(tb_ctx* c) {
                                      2, c->kimp, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? TB_OK : TB_ERR_CUDA;
+}
+
+// The reduction the kernels run, or -1.  A list with a single importance query (one list per query
+// head, one per layer) has nothing to reduce: every mode means the same there.  TB_PER_QHEAD on a
+// context whose lists are per KV head is refused: the lists it asks for do not exist.
+int effective_reduce(const tb_ctx* c, int reduce) {
+    if (reduce != TB_GROUP_SUM && reduce != TB_GROUP_MAX && reduce != TB_PER_QHEAD) return -1;
+    if (c->geom.gl == 1) return TB_GROUP_SUM;
+    return reduce == TB_PER_QHEAD ? -1 : reduce;
 }
 
 bool bad_layers(const tb_ctx* c, int lb, int lc) { return lb < 0 || lc <= 0 || lb + lc > c->cfg.n_layers; }
@@ -185,6 +205,8 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->wk.sel_keys = (uint32_t*)(wp + l.off_sel_keys);
     Geom& g = c->geom;
     g.n_layers = cfg->n_layers, g.Hq = cfg->n_q_heads, g.Hkv = cfg->n_kv_heads, g.g = cfg->n_q_heads / cfg->n_kv_heads;
+    scope_heads(cfg, &g.Hi, &g.Hl, &g.Ha);
+    g.gl = cfg->list_scope == TB_SCOPE_KV_HEAD ? g.g : 1, g.ga = g.Hq / g.Ha;
     g.D = cfg->head_dim, g.dp = cfg->imp_dim, g.max_batch = cfg->max_batch, g.max_seq_len = cfg->max_seq_len;
     g.idx_cap = l.idx_cap, g.dtype = cfg->kv_dtype;
     const size_t n = (size_t)cfg->n_layers * cfg->max_batch;
@@ -309,7 +331,8 @@ tb_status tb_project_keys(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_
 tb_status tb_score_tokens(tb_ctx* c, int32_t layer, const int32_t* seq_ids, int32_t n_seq, const float* q_imp, int32_t reduce,
                           float score_scale, float* scores, void* stream) {
     if (!c || !q_imp || !scores || bad_layers(c, layer, 1)) return TB_ERR_INVALID_ARG;
-    if (reduce != TB_GROUP_SUM && reduce != TB_GROUP_MAX) return TB_ERR_UNSUPPORTED;   // per-query-head lists: not built
+    reduce = effective_reduce(c, reduce);
+    if (reduce < 0) return TB_ERR_UNSUPPORTED;
     int seqs[kMaxLaunchSeq];
     tb_status st = resolve_seqs(c, seq_ids, n_seq, seqs);
     if (st != TB_OK) return st;
@@ -326,7 +349,8 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
     if (!c || !p || bad_layers(c, lb, lc)) return TB_ERR_INVALID_ARG;
     if (p->budget < 0 || p->sinks < 0 || p->recent < 0 || p->radius < 0 || p->interval < 1 || p->step < 0) return TB_ERR_INVALID_ARG;
     if (p->nmode != TB_NEIGHBOR_DILATE && p->nmode != TB_NEIGHBOR_CLUSTER) return TB_ERR_INVALID_ARG;
-    if (p->reduce != TB_GROUP_SUM && p->reduce != TB_GROUP_MAX) return TB_ERR_UNSUPPORTED;   // per-query-head lists: not built
+    const int reduce = effective_reduce(c, p->reduce);
+    if (reduce < 0) return TB_ERR_UNSUPPORTED;
     if (p->budget > c->cfg.max_budget || p->radius > c->cfg.max_radius) return TB_ERR_CAPACITY;
     int seqs[kMaxLaunchSeq];
     tb_status st = resolve_seqs(c, seq_ids, n_seq, seqs);
@@ -343,7 +367,7 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                 int lo, hi;
                 cand_range(c->len[u], p->sinks, p->recent, &lo, &hi);
                 if (c->len_proj[u] < hi) return TB_ERR_UNPROJECTED;
-                bytes += (uint64_t)(hi - lo) * c->cfg.n_kv_heads * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);
+                bytes += (uint64_t)(hi - lo) * c->geom.Hl * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);   // every list streams its keys
             }
     } else {
         for (int l = lb; l < lb + lc; ++l)
@@ -355,11 +379,11 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
         const int n = l0 + step <= lb + lc ? step : lb + lc - l0;
         UnitTable ut;
         fill_table(c, &ut, l0, n, seqs, n_seq);
-        const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->cfg.n_kv_heads;
+        const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->geom.Hl;
         if (refresh) {
             SelectArgs a;
-            a.q_imp = q_imp + (size_t)(l0 - lb) * n_seq * c->cfg.n_q_heads * c->cfg.imp_dim;
-            a.budget = p->budget, a.sinks = p->sinks, a.recent = p->recent, a.reduce = p->reduce;
+            a.q_imp = q_imp + (size_t)(l0 - lb) * n_seq * c->geom.Hl * c->geom.gl * c->cfg.imp_dim;
+            a.budget = p->budget, a.sinks = p->sinks, a.recent = p->recent, a.reduce = reduce;
             if (p->radius == 0) {
                 a.idx_dst = nullptr, a.cnt_dst = nullptr, a.dst_is_state = 1, a.idx_stride = c->geom.idx_cap;
             } else {
@@ -428,7 +452,7 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
                 rows = (long long)(p->sinks < L ? p->sinks : L) + bound + p->recent;
                 if (rows > L) rows = L;
             }
-            bytes += (uint64_t)rows * c->cfg.n_kv_heads * 2 * c->cfg.head_dim * elem_size(c->cfg.kv_dtype);
+            bytes += (uint64_t)rows * c->geom.Ha * 2 * c->cfg.head_dim * elem_size(c->cfg.kv_dtype);
         }
     const int step = layers_per_launch(n_seq);
     const size_t es = elem_size(c->cfg.kv_dtype);
@@ -437,7 +461,7 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
         UnitTable ut;
         fill_table(c, &ut, l0, n, seqs, n_seq);
         const size_t hq_off = (size_t)(l0 - lb) * n_seq * c->cfg.n_q_heads;
-        const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->cfg.n_kv_heads;
+        const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->geom.Hl;
         AttnArgs a;
         a.q = (const char*)q + hq_off * c->cfg.head_dim * es;
         a.idx = idx ? idx + unit_off * c->geom.idx_cap : nullptr;

@@ -38,6 +38,24 @@ struct RowMap {
     }
 };
 
+// An attention unit is (layer, sequence, head h < Ha): one KV head with its group of query heads, or,
+// with one list per query head, a single query head.  It reads KV head h*Hkv/Ha and list h*Hl/Ha.
+struct AttnUnit {
+    size_t kv_c;      // unit row of the K|V cache
+    size_t list_c;    // row of the context's lists
+    int list_l;       // row of caller-supplied lists [layer_count][n_seq][Hl]
+    int lu;           // launch-local attention unit
+    __device__ __forceinline__ AttnUnit(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
+        const size_t pc = (size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s];
+        const int pl = ll * ut.n_seq + s;
+        const int lh = (h * gm.Hl) / gm.Ha;
+        kv_c = pc * gm.Hkv + (h * gm.Hkv) / gm.Ha;
+        list_c = pc * gm.Hl + lh;
+        list_l = pl * gm.Hl + lh;
+        lu = pl * gm.Ha + h;
+    }
+};
+
 // Publishes one split's (m, l, o) per query head and lets the last block to arrive for the
 // (sequence, KV head) merge all splits in split order:  M = max m_j;  l = sum l_j 2^(m_j-M);
 // out = sum o_j 2^(m_j-M) / l;  lse = (M + log2 l) ln 2.  Called by all 128 threads; thread = channel.
@@ -136,9 +154,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
     const int split = blockIdx.x, h = blockIdx.y;
     const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq;
     const int L = ut.len[ll * ut.n_seq + s];
-    const int g = gm.g;
-    const size_t cu = ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h;
-    const int lu = (ll * ut.n_seq + s) * gm.Hkv + h;                 // launch-local unit
+    const int g = gm.ga;
+    const AttnUnit au(gm, ut, ll, s, h);
+    const int lu = au.lu;
 
     RowMap rm;
     rm.L = L, rm.dense = a.dense;
@@ -147,11 +165,11 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
     int n_list = 0;
     if (!a.dense) {
         const int known = a.known_cnt[ll * ut.n_seq + s];
-        n_list = a.idx ? a.cnt[lu] : (known >= 0 ? known : state_cnt[cu]);
+        n_list = a.idx ? a.cnt[au.list_l] : (known >= 0 ? known : state_cnt[au.list_c]);
         n_list = max(0, min(n_list, gm.idx_cap));
     }
     rm.n_list = n_list;
-    rm.list = a.idx ? a.idx + (size_t)lu * gm.idx_cap : state_idx + cu * gm.idx_cap;
+    rm.list = a.idx ? a.idx + (size_t)au.list_l * gm.idx_cap : state_idx + au.list_c * gm.idx_cap;
     const int n_rows = a.dense ? L : rm.n_sink + n_list + (L - rm.w_begin);
 
     const int r_begin = (int)((long long)n_rows * split / a.nsplit);
@@ -181,7 +199,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
         acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
     }
 
-    const T* kv_unit = kv + cu * gm.max_seq_len * 2 * D;
+    const T* kv_unit = kv + au.kv_c * gm.max_seq_len * 2 * D;
     bool any_bad = false;
     for (int r0 = wb; r0 < we; r0 += kRowsPerIter) {
         RowVec<T> kr[kRowsPerIter], vr[kRowsPerIter];
@@ -352,9 +370,9 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const int split = blockIdx.x, h = blockIdx.y;
     const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq;
     const int L = ut.len[ll * ut.n_seq + s];
-    const int g = gm.g;
-    const size_t cu = ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h;
-    const int lu = (ll * ut.n_seq + s) * gm.Hkv + h;
+    const int g = gm.ga;
+    const AttnUnit au(gm, ut, ll, s, h);
+    const int lu = au.lu;
 
     RowMap rm;
     rm.L = L, rm.dense = a.dense;
@@ -363,11 +381,11 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     int n_list = 0;
     if (!a.dense) {
         const int known = a.known_cnt[ll * ut.n_seq + s];
-        n_list = a.idx ? a.cnt[lu] : (known >= 0 ? known : state_cnt[cu]);
+        n_list = a.idx ? a.cnt[au.list_l] : (known >= 0 ? known : state_cnt[au.list_c]);
         n_list = max(0, min(n_list, gm.idx_cap));
     }
     rm.n_list = n_list;
-    rm.list = a.idx ? a.idx + (size_t)lu * gm.idx_cap : state_idx + cu * gm.idx_cap;
+    rm.list = a.idx ? a.idx + (size_t)au.list_l * gm.idx_cap : state_idx + au.list_c * gm.idx_cap;
     const int n_rows = a.dense ? L : rm.n_sink + n_list + (L - rm.w_begin);
 
     // rows of this split, dealt to the warps in whole tiles of 16
@@ -380,7 +398,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const int n_tiles = (we - wb + kTileTok - 1) / kTileTok;
 
     unsigned char* my_stage = smem_dyn + (size_t)warp * kMmaStages * kStageBytes;
-    const unsigned char* kv_unit = reinterpret_cast<const unsigned char*>(kv) + cu * gm.max_seq_len * 2 * D * 2;
+    const unsigned char* kv_unit = reinterpret_cast<const unsigned char*>(kv) + au.kv_c * gm.max_seq_len * 2 * D * 2;
 
     bool any_bad = false;
     // Gather of one tile: the whole warp copies each 512-byte K|V row with one 16-byte cp.async per
@@ -645,7 +663,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         if (rows > L) rows = L;
         if (rows > max_rows) max_rows = rows;
     }
-    const int units = ut.layer_count * ut.n_seq * gm.Hkv;
+    const int units = ut.layer_count * ut.n_seq * gm.Ha;
     a.cluster_merge = 0;
     int nw = kAttnWarps;
     if (gm.dtype == TB_BF16) {
@@ -666,7 +684,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             if (max_active[csize] == 0) {
                 cudaLaunchConfig_t q = {};
                 q.gridDim = dim3(csize, 1, 1), q.blockDim = dim3(256, 1, 1);
-                const size_t mb = (size_t)csize * gm.g * 132 * sizeof(float);
+                const size_t mb = (size_t)csize * gm.ga * 132 * sizeof(float);
                 const bool three = csize <= 8 && 8 * 3 * kStageBytes + mb <= 220 * 1024;
                 q.dynamicSmemBytes = 8 * (three ? 3 : 2) * kStageBytes + mb;
                 cudaLaunchAttribute at[1];
@@ -707,7 +725,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             // more than two tiles per warp would leave the third waiting for a free stage: 12 warps
             // per block when their rings and the merge area still fit the SM
             const int rows_per_block = (max_rows + n - 1) / n;
-            if (rows_per_block > 8 * 2 * kTileTok && 12 * 2 * kStageBytes + (size_t)n * gm.g * 132 * sizeof(float) <= 224 * 1024) nw = 12;
+            if (rows_per_block > 8 * 2 * kTileTok && 12 * 2 * kStageBytes + (size_t)n * gm.ga * 132 * sizeof(float) <= 224 * 1024) nw = 12;
         } else {
             a.nsplit = pick_nsplit(c, units, max_rows);
             // clusters only when the whole launch is resident at once: in multi-wave launches the
@@ -717,19 +735,19 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
     } else {
         a.nsplit = pick_nsplit(c, units, max_rows);
     }
-    dim3 grid(a.nsplit, gm.Hkv, ut.layer_count * ut.n_seq);
+    dim3 grid(a.nsplit, gm.Ha, ut.layer_count * ut.n_seq);
 #define TB_ATTN(T, G)                                                                                                   \
     attn_kernel<T, G><<<grid, kAttnThreads, 0, s>>>(gm, ut, a, (const T*)c->kv, c->st.idx, c->st.cnt, c->wk.part_o,     \
                                                    c->wk.part_ml, c->st.attn_counter, c->st.status)
 #define TB_ATTN_G(T)                                  \
     do {                                              \
-        if (gm.g == 1) TB_ATTN(T, 1);                 \
-        else if (gm.g == 2) TB_ATTN(T, 2);            \
-        else if (gm.g <= 4) TB_ATTN(T, 4);            \
+        if (gm.ga == 1) TB_ATTN(T, 1);                \
+        else if (gm.ga == 2) TB_ATTN(T, 2);           \
+        else if (gm.ga <= 4) TB_ATTN(T, 4);           \
         else TB_ATTN(T, 8);                           \
     } while (0)
     if (gm.dtype == TB_BF16) {
-        const size_t merge_bytes = a.cluster_merge ? (size_t)a.nsplit * gm.g * 132 * sizeof(float) : 0;
+        const size_t merge_bytes = a.cluster_merge ? (size_t)a.nsplit * gm.ga * 132 * sizeof(float) : 0;
         // three stages per warp when the 8-warp block still fits the SM with them
         const int nst = (nw == 8 && 8 * 3 * kStageBytes + merge_bytes <= 220 * 1024 && a.nsplit <= 8) ? 3 : 2;
         const size_t smem = (size_t)nw * nst * kStageBytes + merge_bytes;
@@ -844,6 +862,7 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
 
     Geom gm;
     gm.n_layers = 1, gm.Hq = n_q_heads, gm.Hkv = n_kv_heads, gm.g = n_q_heads / n_kv_heads, gm.D = head_dim, gm.dp = 0;
+    gm.Hi = gm.Hl = gm.Ha = n_kv_heads, gm.gl = gm.ga = gm.g;
     gm.max_batch = 1 << 20, gm.max_seq_len = max_seq_len, gm.idx_cap = idx_dev ? idx_stride : 0, gm.dtype = kv_dtype;
     UnitTable ut;
     ut.layer_begin = 0, ut.layer_count = 1, ut.n_seq = n_seq;
@@ -886,7 +905,7 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
             gm, ut, a, (const __nv_bfloat16*)kv_dev, nullptr, nullptr, part_o, part_ml, counters, status);
     } else {
 #define TB_ATTN_S(G) attn_kernel<float, G><<<grid, kAttnThreads, 0, s>>>(gm, ut, a, (const float*)kv_dev, nullptr, nullptr, part_o, part_ml, counters, status)
-        if (gm.g == 1) TB_ATTN_S(1); else if (gm.g == 2) TB_ATTN_S(2); else if (gm.g <= 4) TB_ATTN_S(4); else TB_ATTN_S(8);
+        if (gm.ga == 1) TB_ATTN_S(1); else if (gm.ga == 2) TB_ATTN_S(2); else if (gm.ga <= 4) TB_ATTN_S(4); else TB_ATTN_S(8);
 #undef TB_ATTN_S
     }
     return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;

@@ -82,26 +82,36 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTabl
     if (t0 >= t_end) return;
     const int nt = min(kProjTokens, t_end - t0);
 
-    const T* W = Wall + ((size_t)layer * gm.Hkv + h) * D * DP;
-    for (int i = threadIdx.x; i < D * DP; i += kProjThreads) Ws[i] = Elem<T>::to_f32(W[i]);
-    const size_t row0 = (((size_t)layer * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h) * gm.max_seq_len + t0;
-    for (int i = threadIdx.x; i < nt * D; i += kProjThreads) {
-        int t = i / D, ch = i % D;
-        Ks[t][ch] = Elem<T>::to_f32(kv[(row0 + t) * 2 * D + ch]);
-    }
-    __syncthreads();
-
+    // One key stream per KV head, or (one list per layer) a single stream that sums the heads'
+    // projections: K_imp[t] = sum_h K[t][h] . W[h], heads in ascending order on one fp32 chain.
+    const int n_sum = gm.Hkv / gm.Hi;
+    const size_t pair = (size_t)layer * gm.max_batch + ut.seq_id[s];
     const int t = threadIdx.x / 4, jq = threadIdx.x % 4;
-    if (t >= nt) return;
     float acc[JPT];
 #pragma unroll
     for (int j = 0; j < JPT; ++j) acc[j] = 0.f;
+    for (int hs = 0; hs < n_sum; ++hs) {
+        const int hk = h * n_sum + hs;
+        const T* W = Wall + ((size_t)layer * gm.Hkv + hk) * D * DP;
+        if (hs) __syncthreads();
+        for (int i = threadIdx.x; i < D * DP; i += kProjThreads) Ws[i] = Elem<T>::to_f32(W[i]);
+        const size_t krow0 = (pair * gm.Hkv + hk) * gm.max_seq_len + t0;
+        for (int i = threadIdx.x; i < nt * D; i += kProjThreads) {
+            int tt = i / D, ch = i % D;
+            Ks[tt][ch] = Elem<T>::to_f32(kv[(krow0 + tt) * 2 * D + ch]);
+        }
+        __syncthreads();
+        if (t < nt) {
 #pragma unroll 4
-    for (int ch = 0; ch < D; ++ch) {
-        float kx = Ks[t][ch];
+            for (int ch = 0; ch < D; ++ch) {
+                float kx = Ks[t][ch];
 #pragma unroll
-        for (int j = 0; j < JPT; ++j) acc[j] = fmaf(kx, Ws[ch * DP + jq * JPT + j], acc[j]);
+                for (int j = 0; j < JPT; ++j) acc[j] = fmaf(kx, Ws[ch * DP + jq * JPT + j], acc[j]);
+            }
+        }
     }
+    if (t >= nt) return;
+    const size_t row0 = (pair * gm.Hi + h) * gm.max_seq_len + t0;
     T* dst = kimp + (row0 + t) * DP + jq * JPT;
 #pragma unroll
     for (int j = 0; j < JPT; ++j) dst[j] = Elem<T>::from_f32(acc[j]);
@@ -136,64 +146,79 @@ __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTa
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gid = lane >> 2, tig = lane & 3;
 
-    const size_t row0 = (((size_t)layer * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h) * gm.max_seq_len + t0;
-    const unsigned char* kbase = reinterpret_cast<const unsigned char*>(kv) + row0 * 2 * D * 2;
-    const unsigned char* wbase = reinterpret_cast<const unsigned char*>(Wall + ((size_t)layer * gm.Hkv + h) * D * DP);
+    // One key stream per KV head, or (one list per layer) a single stream that sums the heads'
+    // projections in the fp32 accumulators, heads in ascending order.
+    const int n_sum = gm.Hkv / gm.Hi;
+    const size_t pair = (size_t)layer * gm.max_batch + ut.seq_id[s];
     const uint32_t ks_u32 = smem_u32(Ks), ws_u32 = smem_u32(Ws);
-    for (int i = tid; i < kPmTokens * 16; i += kPmThreads) {          // 16 chunks of 16 B per K row
-        const int t = i >> 4, ch = i & 15;
-        const int tc = min(t, nt_valid - 1);                           // rows past the range repeat the last one
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ks_u32 + t * kPmKPitch + ch * 16),
-                     "l"(kbase + (size_t)tc * 512 + ch * 16) : "memory");
-    }
-    for (int i = tid; i < D * (DP / 8); i += kPmThreads) {             // DP/8 chunks per W row
-        const int r = i / (DP / 8), ch = i % (DP / 8);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ws_u32 + r * kWPitch + ch * 16),
-                     "l"(wbase + (size_t)r * DP * 2 + ch * 16) : "memory");
-    }
-    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
-
     const int mi = lane >> 3, r8 = lane & 7;
-    // B fragments (W: k = channel, n = output) for every k-step and output tile, loaded once per warp
-    uint32_t bw[8][NT][2];
+    float acc[2][NT][4];
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks)
+    for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-        for (int np = 0; np < NT / 2; ++np) {
-            // matrices: (ch lo, outs np*16+0..7), (ch hi, same), (ch lo, outs +8), (ch hi, outs +8)
-            const uint32_t addr = ws_u32 + (ks * 16 + (mi & 1) * 8 + r8) * kWPitch + (np * 16 + (mi >> 1) * 8) * 2;
-            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(bw[ks][2 * np][0]), "=r"(bw[ks][2 * np][1]), "=r"(bw[ks][2 * np + 1][0]), "=r"(bw[ks][2 * np + 1][1])
-                         : "r"(addr));
+        for (int n = 0; n < NT; ++n) acc[mt][n][0] = acc[mt][n][1] = acc[mt][n][2] = acc[mt][n][3] = 0.f;
+
+    for (int hs = 0; hs < n_sum; ++hs) {
+        const int hk = h * n_sum + hs;
+        const size_t krow0 = (pair * gm.Hkv + hk) * gm.max_seq_len + t0;
+        const unsigned char* kbase = reinterpret_cast<const unsigned char*>(kv) + krow0 * 2 * D * 2;
+        const unsigned char* wbase = reinterpret_cast<const unsigned char*>(Wall + ((size_t)layer * gm.Hkv + hk) * D * DP);
+        if (hs) __syncthreads();                                       // the previous head's tiles are consumed
+        for (int i = tid; i < kPmTokens * 16; i += kPmThreads) {          // 16 chunks of 16 B per K row
+            const int t = i >> 4, ch = i & 15;
+            const int tc = min(t, nt_valid - 1);                           // rows past the range repeat the last one
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ks_u32 + t * kPmKPitch + ch * 16),
+                         "l"(kbase + (size_t)tc * 512 + ch * 16) : "memory");
         }
-    __nv_bfloat16* out = kimp + row0 * DP;
+        for (int i = tid; i < D * (DP / 8); i += kPmThreads) {             // DP/8 chunks per W row
+            const int r = i / (DP / 8), ch = i % (DP / 8);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ws_u32 + r * kWPitch + ch * 16),
+                         "l"(wbase + (size_t)r * DP * 2 + ch * 16) : "memory");
+        }
+        asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+
+        // B fragments (W: k = channel, n = output) for every k-step and output tile, loaded once per warp
+        uint32_t bw[8][NT][2];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+            for (int np = 0; np < NT / 2; ++np) {
+                // matrices: (ch lo, outs np*16+0..7), (ch hi, same), (ch lo, outs +8), (ch hi, outs +8)
+                const uint32_t addr = ws_u32 + (ks * 16 + (mi & 1) * 8 + r8) * kWPitch + (np * 16 + (mi >> 1) * 8) * 2;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(bw[ks][2 * np][0]), "=r"(bw[ks][2 * np][1]), "=r"(bw[ks][2 * np + 1][0]), "=r"(bw[ks][2 * np + 1][1])
+                             : "r"(addr));
+            }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const int tok = warp * 32 + mt * 16;                           // first token of this 16-token tile
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                uint32_t a0, a1, a2, a3;
+                const uint32_t addr = ks_u32 + (tok + (mi & 1) * 8 + r8) * kPmKPitch + ks * 32 + (mi >> 1) * 16;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+#pragma unroll
+                for (int n = 0; n < NT; ++n)
+                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                 : "+f"(acc[mt][n][0]), "+f"(acc[mt][n][1]), "+f"(acc[mt][n][2]), "+f"(acc[mt][n][3])
+                                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bw[ks][n][0]), "r"(bw[ks][n][1]));
+            }
+        }
+    }
+    __nv_bfloat16* out = kimp + ((pair * gm.Hi + h) * gm.max_seq_len + t0) * DP;
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt) {
-        const int tok = warp * 32 + mt * 16;                           // first token of this 16-token tile
-        float acc[NT][4];
-#pragma unroll
-        for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            uint32_t a0, a1, a2, a3;
-            const uint32_t addr = ks_u32 + (tok + (mi & 1) * 8 + r8) * kPmKPitch + ks * 32 + (mi >> 1) * 16;
-            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
-#pragma unroll
-            for (int n = 0; n < NT; ++n)
-                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                             : "+f"(acc[n][0]), "+f"(acc[n][1]), "+f"(acc[n][2]), "+f"(acc[n][3])
-                             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bw[ks][n][0]), "r"(bw[ks][n][1]));
-        }
+        const int tok = warp * 32 + mt * 16;
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
             const int j = n * 8 + tig * 2;
             if (tok + gid < nt_valid) {
-                __nv_bfloat162 v = __floats2bfloat162_rn(acc[n][0], acc[n][1]);
+                __nv_bfloat162 v = __floats2bfloat162_rn(acc[mt][n][0], acc[mt][n][1]);
                 *reinterpret_cast<__nv_bfloat162*>(out + (size_t)(tok + gid) * DP + j) = v;
             }
             if (tok + gid + 8 < nt_valid) {
-                __nv_bfloat162 v = __floats2bfloat162_rn(acc[n][2], acc[n][3]);
+                __nv_bfloat162 v = __floats2bfloat162_rn(acc[mt][n][2], acc[mt][n][3]);
                 *reinterpret_cast<__nv_bfloat162*>(out + (size_t)(tok + gid + 8) * DP + j) = v;
             }
         }
@@ -211,7 +236,7 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
     if (max_range <= 0) return cudaSuccess;
     const Geom& gm = c->geom;
     if (gm.dtype == TB_BF16) {
-        dim3 grid_mma((max_range + kPmTokens - 1) / kPmTokens, gm.Hkv, ut.layer_count * ut.n_seq);
+        dim3 grid_mma((max_range + kPmTokens - 1) / kPmTokens, gm.Hi, ut.layer_count * ut.n_seq);
         const __nv_bfloat16* kvp = (const __nv_bfloat16*)c->kv;
         const __nv_bfloat16* wp = (const __nv_bfloat16*)c->st.W;
         if (gm.dp == 32) {
@@ -233,7 +258,7 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
         }
         return cudaGetLastError();
     }
-    dim3 grid((max_range + kProjTokens - 1) / kProjTokens, gm.Hkv, ut.layer_count * ut.n_seq);
+    dim3 grid((max_range + kProjTokens - 1) / kProjTokens, gm.Hi, ut.layer_count * ut.n_seq);
 #define TB_PROJ(T, DP) \
     project_kernel<T, DP><<<grid, kProjThreads, 0, s>>>(gm, ut, pt, (const T*)c->kv, (const T*)c->st.W, (T*)c->kimp)
     if (gm.dp == 32) TB_PROJ(float, 32); else TB_PROJ(float, 16);

@@ -19,6 +19,12 @@ constexpr int kMaxGroup = 8;          // query heads per KV head
 // Geometry every kernel needs; passed by value.
 struct Geom {
     int n_layers, Hq, Hkv, g, D, dp;
+    // Selection scope (tb_list_scope): Hi key streams of the projected-key cache, Hl index lists and
+    // Ha attention units per (layer, sequence); gl importance queries are reduced into one list and
+    // ga query heads share an attention unit's gathered rows.
+    //   per KV head:    Hi = Hl = Ha = Hkv, gl = ga = g
+    //   per query head: Hi = Hkv, Hl = Ha = Hq, gl = ga = 1
+    int Hi, Hl, Ha, gl, ga;
     int max_batch, max_seq_len;
     int idx_cap;       // entries per index-list row
     int dtype;         // tb_dtype
@@ -67,19 +73,19 @@ struct AttnArgs {
 
 struct DevState {
     void* W;              // [n_layers][Hkv][D][dp] kv_dtype
-    int32_t* idx;         // [n_layers][max_batch][Hkv][idx_cap]
-    int32_t* cnt;         // [n_layers][max_batch][Hkv]
+    int32_t* idx;         // [n_layers][max_batch][Hl][idx_cap]
+    int32_t* cnt;         // [n_layers][max_batch][Hl]
     int32_t* status;      // device status word
-    uint32_t* attn_counter;  // [n_layers*max_batch*Hkv] split arrival counters (self-resetting)
+    uint32_t* attn_counter;  // [n_layers*max_batch*Ha] split arrival counters (self-resetting)
 };
 
 struct DevWork {
     float* part_o;        // [units_q][kMaxSplits][D]
     float* part_ml;       // [units_q][kMaxSplits][2]
-    int32_t* sel_idx;     // [n_layers*max_batch*Hkv][max_budget rounded]  pre-expansion selection
+    int32_t* sel_idx;     // [n_layers*max_batch*Hl][max_budget rounded]  pre-expansion selection
     int32_t* sel_cnt;
     int sel_stride;
-    uint32_t* sel_keys;   // [n_layers*max_batch*Hkv][max_seq_len rounded up to 256]  score keys of a many-problem selection launch
+    uint32_t* sel_keys;   // [n_layers*max_batch*Hl][max_seq_len rounded up to 256]  score keys of a many-problem selection launch
 };
 
 }  // namespace tb

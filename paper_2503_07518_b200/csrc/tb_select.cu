@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     const int hi = max(lo, L - a.recent);
     const int ncand = hi - lo;
     const int k = min(a.budget, ncand);
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t cu = list_unit(gm, ut, ll, s, h);
     const size_t dst_row = a.dst_is_state ? cu : (size_t)blockIdx.y;
     int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
     int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     const int my_tiles = max(0, min(tiles_per_cta, n_tiles - tile0));
     const int tok0 = lo + tile0 * kTileRows;           // token of local slot 0
     const int n_local = max(0, min(my_tiles * kTileRows, hi - tok0));
-    const long long row_base = (long long)cu * gm.max_seq_len + tok0;   // row of the 2-D view of the cache
+    const long long row_base = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len + tok0;   // row of the 2-D view of the cache
 
     if (tid == 0) {
         for (int i = 0; i < n_stages && i < my_tiles; ++i) {
@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         }
     }
     GroupScorer<T, DP, RED> scorer;
-    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    scorer.load(a.q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, sm->qs);
     if (RED != TB_GROUP_SUM) __syncthreads();
 
     // ---- stream + score + first digit histogram -------------------------------------------------
@@ -557,7 +557,7 @@ static int select_stage_count(int tiles_per_cta, int tile_bytes) {
 
 cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
     const Geom& gm = c->geom;
-    const int n_units = ut.layer_count * ut.n_seq * gm.Hkv;
+    const int n_units = ut.layer_count * ut.n_seq * gm.Hl;
     int max_cand = 0;
     for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) {
         int L = ut.len[i], lo = a.sinks < L ? a.sinks : L, hi = L - a.recent > lo ? L - a.recent : lo;

@@ -96,13 +96,24 @@ struct GroupScorer {
     }
 };
 
+// A selection unit is one index list: (layer, sequence, list head h < Hl).
 __device__ __forceinline__ void decode_unit(const Geom& gm, const UnitTable& ut, int u, int& ll, int& s, int& h) {
-    h = u % gm.Hkv;
-    s = (u / gm.Hkv) % ut.n_seq;
-    ll = u / (gm.Hkv * ut.n_seq);
+    h = u % gm.Hl;
+    s = (u / gm.Hl) % ut.n_seq;
+    ll = u / (gm.Hl * ut.n_seq);
 }
-__device__ __forceinline__ size_t cache_unit(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
-    return ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h;
+// Row of the unit in the context's lists, counts and parked-key workspace.
+__device__ __forceinline__ size_t list_unit(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
+    return ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hl + h;
+}
+// Key stream of the unit in the projected-key cache: its own (one list per KV head), its KV head's
+// (one list per query head) or the layer's only one.
+__device__ __forceinline__ size_t key_unit(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
+    return ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hi + (h * gm.Hi) / gm.Hl;
+}
+// The unit's importance queries: gl consecutive rows of q_imp [layer_count][n_seq][Hl * gl][d'].
+__device__ __forceinline__ size_t query_row(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
+    return ((size_t)(ll * ut.n_seq + s) * gm.Hl + h) * gm.gl;
 }
 
 }  // namespace tb

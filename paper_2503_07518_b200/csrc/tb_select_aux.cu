@@ -15,10 +15,10 @@ __global__ void __launch_bounds__(256) score_kernel(Geom gm, UnitTable ut, const
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
     const int L = ut.len[ll * ut.n_seq + s];
     GroupScorer<T, DP, RED> scorer;
-    scorer.load(q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, qs);
+    scorer.load(q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, qs);
     if (RED != TB_GROUP_SUM) __syncthreads();
-    const uint4* base = reinterpret_cast<const uint4*>(kimp + cache_unit(gm, ut, ll, s, h) * gm.max_seq_len * DP);
-    float* out = scores + ((size_t)(ll * ut.n_seq + s) * gm.Hkv + h) * gm.max_seq_len;
+    const uint4* base = reinterpret_cast<const uint4*>(kimp + key_unit(gm, ut, ll, s, h) * gm.max_seq_len * DP);
+    float* out = scores + ((size_t)(ll * ut.n_seq + s) * gm.Hl + h) * gm.max_seq_len;
     for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < L; t += gridDim.x * blockDim.x) {
         const uint4* row = base + (size_t)t * NCH;
         float sc = scorer.score([&](int c) { return __ldg(row + c); });
@@ -31,7 +31,7 @@ cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_im
     int maxL = 0;
     for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) maxL = ut.len[i] > maxL ? ut.len[i] : maxL;
     if (maxL == 0) return cudaSuccess;
-    dim3 grid((maxL + 255) / 256, ut.layer_count * ut.n_seq * gm.Hkv);
+    dim3 grid((maxL + 255) / 256, ut.layer_count * ut.n_seq * gm.Hl);
     if (grid.x > 64) grid.x = 64;
 #define TB_SCORE(T, DP)                                                                                                   \
     do {                                                                                                                  \
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kNbThreads) neighbor_kernel(Geom gm, UnitTable
     const int n_words = (span + 31) / 32;
     const int32_t* src = a.idx_src + (size_t)blockIdx.x * a.src_stride;
     const int cnt = a.cnt_src[blockIdx.x];
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t cu = list_unit(gm, ut, ll, s, h);
     int32_t* dst = state_idx + cu * gm.idx_cap;
 
     for (int i = tid; i < n_words; i += kNbThreads) mask[i] = 0;
@@ -134,7 +134,7 @@ cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const Neighbo
         if (e != cudaSuccess) return e;
     }
     if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
-    neighbor_kernel<<<ut.layer_count * ut.n_seq * gm.Hkv, kNbThreads, smem, s>>>(gm, ut, a, c->st.idx, c->st.cnt);
+    neighbor_kernel<<<ut.layer_count * ut.n_seq * gm.Hl, kNbThreads, smem, s>>>(gm, ut, a, c->st.idx, c->st.cnt);
     return cudaGetLastError();
 }
 
@@ -144,7 +144,7 @@ __global__ void copy_lists_kernel(Geom gm, UnitTable ut, const int32_t* __restri
                                   int32_t* __restrict__ idx_out, int32_t* __restrict__ cnt_out) {
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.x, ll, s, h);
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t cu = list_unit(gm, ut, ll, s, h);
     const int n = state_cnt[cu];
     if (idx_out)
         for (int i = threadIdx.x; i < n; i += blockDim.x) idx_out[(size_t)blockIdx.x * gm.idx_cap + i] = state_idx[cu * gm.idx_cap + i];
@@ -152,7 +152,7 @@ __global__ void copy_lists_kernel(Geom gm, UnitTable ut, const int32_t* __restri
 }
 
 cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s) {
-    copy_lists_kernel<<<ut.layer_count * ut.n_seq * c->geom.Hkv, 256, 0, s>>>(c->geom, ut, c->st.idx, c->st.cnt, idx_out, cnt_out);
+    copy_lists_kernel<<<ut.layer_count * ut.n_seq * c->geom.Hl, 256, 0, s>>>(c->geom, ut, c->st.idx, c->st.cnt, idx_out, cnt_out);
     return cudaGetLastError();
 }
 

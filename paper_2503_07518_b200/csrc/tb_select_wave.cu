@@ -459,15 +459,15 @@ __global__ void __launch_bounds__(kThreads, 4)
     const int cache_vecs = n_stages * (int)kTileBytes / 16;                      // 16-byte vectors of 4 keys
 
     const int tid = threadIdx.x, lane = tid & 31;
-    const int pair = order.pair[blockIdx.x / gm.Hkv], h = blockIdx.x % gm.Hkv;
+    const int pair = order.pair[blockIdx.x / gm.Hl], h = blockIdx.x % gm.Hl;
     const int ll = pair / ut.n_seq, s = pair % ut.n_seq;
     const int L = ut.len[pair];
     const int lo = min(a.sinks, L);
     const int hi = max(lo, L - a.recent);
     const int ncand = hi - lo;
     const int k = min(a.budget, ncand);
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
-    const size_t dst_row = a.dst_is_state ? cu : (size_t)pair * gm.Hkv + h;
+    const size_t cu = list_unit(gm, ut, ll, s, h);
+    const size_t dst_row = a.dst_is_state ? cu : (size_t)pair * gm.Hl + h;
     int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
     int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
 
@@ -492,7 +492,7 @@ __global__ void __launch_bounds__(kThreads, 4)
     __syncthreads();
 
     const int n_tiles = (ncand + kRows - 1) / kRows;
-    const long long row_base = (long long)cu * gm.max_seq_len + lo;              // row of candidate 0 in the 2-D view
+    const long long row_base = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len + lo;              // row of candidate 0 in the 2-D view
     uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255); // by candidate index, 16-byte aligned
     // The projected keys stream through L2 once; the score keys parked there must still be there when
     // the block comes back for them.
@@ -510,7 +510,7 @@ __global__ void __launch_bounds__(kThreads, 4)
         for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
     }
     GroupScorer<T, DP, RED> scorer;
-    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    scorer.load(a.q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, sm->qs);
     if (RED != TB_GROUP_SUM) __syncthreads();
     if (tid == 0)
         for (int i = 0; i < n_stages && i < n_tiles; ++i) {
@@ -604,7 +604,7 @@ extern "C" int tb_debug_wave_ns(unsigned long long* out) { return (int)cudaMemcp
 
 cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
     const Geom& gm = c->geom;
-    const int n_pairs = ut.layer_count * ut.n_seq, n_units = n_pairs * gm.Hkv;
+    const int n_pairs = ut.layer_count * ut.n_seq, n_units = n_pairs * gm.Hl;
     WaveOrder order;
     int cand[kMaxLaunchUnits];
     for (int i = 0; i < n_pairs; ++i) {
@@ -711,7 +711,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
     const int L = ut.len[ll * ut.n_seq + s];
     const int lo = min(a.sinks, L), ncand = max(lo, L - a.recent) - lo, k = min(a.budget, ncand);
-    const size_t cu = cache_unit(gm, ut, ll, s, h);
+    const size_t cu = list_unit(gm, ut, ll, s, h);
     const size_t dst_row = a.dst_is_state ? cu : (size_t)blockIdx.y;
     int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
     int32_t* cnt_dst = (a.dst_is_state ? state_cnt : a.cnt_dst) + dst_row;
@@ -747,7 +747,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     const int tile0 = rank * tiles_per_cta, my_tiles = max(0, min(tiles_per_cta, n_tiles - tile0));
     const int slot0 = tile0 * kRows;                   // candidate index of this block's first row
     const int n_local = max(0, min(my_tiles * kRows, ncand - slot0));
-    const long long row_base = (long long)cu * gm.max_seq_len + lo;              // row of candidate 0
+    const long long row_base = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len + lo;              // row of candidate 0
     uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255);
     const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
 
@@ -763,7 +763,7 @@ __global__ void __launch_bounds__(kThreads, 2)
         for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
     }
     GroupScorer<T, DP, RED> scorer;
-    scorer.load(a.q_imp + ((size_t)(ll * ut.n_seq + s) * gm.Hq + h * gm.g) * DP, gm.g, sm->qs);
+    scorer.load(a.q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, sm->qs);
     if (RED != TB_GROUP_SUM) __syncthreads();
     if (tid == 0)
         for (int i = 0; i < n_stages && i < my_tiles; ++i) {
@@ -1018,7 +1018,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 
 cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
     const Geom& gm = c->geom;
-    const int n_units = ut.layer_count * ut.n_seq * gm.Hkv;
+    const int n_units = ut.layer_count * ut.n_seq * gm.Hl;
     int max_cand = 0;
     for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) {
         const int L = ut.len[i], lo = a.sinks < L ? a.sinks : L, hi = L - a.recent > lo ? L - a.recent : lo;

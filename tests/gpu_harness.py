@@ -36,12 +36,20 @@ def to_host(t: torch.Tensor, dtype: int) -> np.ndarray:
 class Case:
     """A workload instantiated on the host (numpy) and on the device (tb.Context)."""
 
-    def __init__(self, w: wl.Workload, max_budget=None, max_radius=None, extra_len=0, project="device", kv_on_host=False):
+    def __init__(self, w: wl.Workload, max_budget=None, max_radius=None, extra_len=0, project="device", kv_on_host=False,
+                 list_scope=tb.TB_SCOPE_KV_HEAD):
         self.w = w
         self.lengths = list(w.lengths)
         self.cap = max(self.lengths) + extra_len
         self.ctx = tb.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, self.cap,
-                              max_budget or max(1, w.budget), w.radius if max_radius is None else max_radius, kv_on_host=kv_on_host)
+                              max_budget or max(1, w.budget), w.radius if max_radius is None else max_radius, kv_on_host=kv_on_host,
+                              list_scope=list_scope)
+        # Heads per (layer, sequence) under the selection scope: key streams of the projected-key cache,
+        # lists, attention units; importance queries per list and query heads per attention unit.
+        self.Hi, self.Hl = self.ctx.n_key_heads, self.ctx.n_lists
+        self.Ha = max(self.Hl, w.n_kv_heads)
+        self.gl = w.group if list_scope == tb.TB_SCOPE_KV_HEAD else 1
+        self.ga = w.n_q_heads // self.Ha
         self.K = [[None] * w.batch for _ in range(w.n_layers)]     # [layer][seq] -> [Hkv, cap, D] storage
         self.V = [[None] * w.batch for _ in range(w.n_layers)]
         self.Kimp = [[None] * w.batch for _ in range(w.n_layers)]  # oracle's projection, [Hkv, cap, d']
@@ -54,7 +62,7 @@ class Case:
                 K, V = wl.gen_KV(w, l, b)
                 self.K[l][b] = np.zeros((w.n_kv_heads, self.cap, w.head_dim), K.dtype)
                 self.V[l][b] = np.zeros_like(self.K[l][b])
-                self.Kimp[l][b] = np.zeros((w.n_kv_heads, self.cap, w.imp_dim), K.dtype)
+                self.Kimp[l][b] = np.zeros((self.Hi, self.cap, w.imp_dim), K.dtype)
                 self.K[l][b][:, :self.lengths[b]] = K
                 self.V[l][b][:, :self.lengths[b]] = V
             self._append_layer(l, [self.K[l][b][:, :self.lengths[b]] for b in range(w.batch)],
@@ -94,14 +102,18 @@ class Case:
             for b in range(w.batch):
                 if end[b] <= begin[b]:
                     continue
-                for h in range(w.n_kv_heads):
+                # one list per layer: the token's concatenated key [Hkv*D] times the stacked W_K [Hkv*D][d']
+                Ks = [self.K[l][b][h, begin[b]:end[b]] for h in range(w.n_kv_heads)] if self.Hi == w.n_kv_heads else \
+                    [np.concatenate([self.K[l][b][h, begin[b]:end[b]] for h in range(w.n_kv_heads)], axis=1)]
+                Ws = [self.W[l][h] for h in range(w.n_kv_heads)] if self.Hi == w.n_kv_heads else \
+                    [np.concatenate([self.W[l][h] for h in range(w.n_kv_heads)], axis=0)]
+                for h in range(self.Hi):
                     self.Kimp[l][b][h, begin[b]:end[b]] = orc.project_keys(
-                        np.ascontiguousarray(self.K[l][b][h, begin[b]:end[b]]), np.ascontiguousarray(self.W[l][h]), w.dtype)
+                        np.ascontiguousarray(Ks[h]), np.ascontiguousarray(Ws[h]), w.dtype)
                 if compare:
                     dev = to_host(self.ctx.kimp[l, b, :, begin[b]:end[b]], w.dtype)
-                    for h in range(w.n_kv_heads):
-                        worst = max(worst, projection_excess(dev[h], self.Kimp[l][b][h, begin[b]:end[b]],
-                                                             self.K[l][b][h, begin[b]:end[b]], self.W[l][h], w.dtype))
+                    for h in range(self.Hi):
+                        worst = max(worst, projection_excess(dev[h], self.Kimp[l][b][h, begin[b]:end[b]], Ks[h], Ws[h], w.dtype))
                 self.ctx.kimp[l, b, :, begin[b]:end[b]] = to_dev(self.Kimp[l][b][:, begin[b]:end[b]], w.dtype)
         for b in range(w.batch):
             self.proj[b] = max(self.proj[b], end[b])
@@ -114,9 +126,10 @@ class Case:
 
     # ---- oracle side --------------------------------------------------------------------------------
     def oracle_select(self, l, b, h, q_imp, p):
-        """Oracle list (after neighbours) and the fp64 scores, on the oracle's K_imp bytes."""
+        """Oracle list (after neighbours) and the fp64 scores, on the oracle's K_imp bytes.  h = list
+        head; q_imp = the (layer, sequence)'s importance queries [Hl * gl][d']."""
         w, L = self.w, self.cur[b]
-        s = orc.score(q_imp[h * w.group:(h + 1) * w.group], np.ascontiguousarray(self.Kimp[l][b][h, :L]), w.dtype,
+        s = orc.score(q_imp[h * self.gl:(h + 1) * self.gl], np.ascontiguousarray(self.Kimp[l][b][h * self.Hi // self.Hl, :L]), w.dtype,
                       reduce=getattr(p, "reduce", orc.GROUP_SUM))
         base = orc.select(s, p.sinks, p.recent, p.budget)
         lo, hi = orc.candidate_range(L, p.sinks, p.recent)
@@ -124,10 +137,12 @@ class Case:
         return base, full, s
 
     def oracle_attention(self, l, b, h, q, I, p, dense=False):
+        """h = attention unit (a KV head with its group, or one query head); I = the list it reads."""
         w, L = self.w, self.cur[b]
-        K = np.ascontiguousarray(self.K[l][b][h, :L])
-        V = np.ascontiguousarray(self.V[l][b][h, :L])
-        qh = np.ascontiguousarray(q[h * w.group:(h + 1) * w.group])
+        hk = h * w.n_kv_heads // self.Ha
+        K = np.ascontiguousarray(self.K[l][b][hk, :L])
+        V = np.ascontiguousarray(self.V[l][b][hk, :L])
+        qh = np.ascontiguousarray(q[h * self.ga:(h + 1) * self.ga])
         A = np.arange(L, dtype=np.int32) if dense else orc.attended_set(L, p.sinks, p.recent, I)
         return orc.attention(qh, K, V, A, w.dtype)
 
@@ -173,17 +188,17 @@ def check_selection(gpu_idx: np.ndarray, orc_idx: np.ndarray, scores: np.ndarray
 
 
 def gpu_select(case: Case, q_imp_all: np.ndarray, p, layer_begin=0, layer_count=None):
-    """q_imp_all [layer_count][B][Hq][d'] -> lists [layer_count][B][Hkv] of numpy arrays."""
+    """q_imp_all [layer_count][B][Hl * gl][d'] -> lists [layer_count][B][Hl] of numpy arrays."""
     w = case.w
     lc = w.n_layers - layer_begin if layer_count is None else layer_count
     cap = case.ctx.index_capacity
-    idx = torch.full((lc, w.batch, w.n_kv_heads, cap), -1, dtype=torch.int32, device="cuda")
-    cnt = torch.full((lc, w.batch, w.n_kv_heads), -1, dtype=torch.int32, device="cuda")
+    idx = torch.full((lc, w.batch, case.Hl, cap), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((lc, w.batch, case.Hl), -1, dtype=torch.int32, device="cuda")
     case.ctx.select_topk(layer_begin, lc, None, w.batch, torch.from_numpy(np.ascontiguousarray(q_imp_all, np.float32)).cuda(),
                          p, idx, cnt)
     torch.cuda.synchronize()
     idx, cnt = idx.cpu().numpy(), cnt.cpu().numpy()
-    return [[[idx[l, b, h, :cnt[l, b, h]].copy() for h in range(w.n_kv_heads)] for b in range(w.batch)] for l in range(lc)]
+    return [[[idx[l, b, h, :cnt[l, b, h]].copy() for h in range(case.Hl)] for b in range(w.batch)] for l in range(lc)]
 
 
 def gpu_attention(case: Case, q_all: np.ndarray, p, idx=None, cnt=None, layer_begin=0, layer_count=None, want_lse=True):

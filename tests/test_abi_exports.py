@@ -41,14 +41,14 @@ def test_binding_lists_the_same_names(libpath):
 def test_host_validation_needs_no_gpu(libpath):
     from paper_2503_07518_b200 import binding as b
     L = b.lib()
-    cfg = b.tb_config(2, 8, 8, 128, 32, b.TB_BF16, 1, 1024, 64, 1, 0)
+    cfg = b.tb_config(2, 8, 8, 128, 32, b.TB_BF16, 1, 1024, 64, 1, 0, 0)
     sizes = [ctypes.c_size_t() for _ in range(4)]
     assert L.tb_query_sizes(ctypes.byref(cfg), *[ctypes.byref(s) for s in sizes]) == b.TB_OK
     assert sizes[0].value == 2 * 1 * 8 * 1024 * 2 * 128 * 2            # interleaved K|V rows
     assert sizes[1].value == 2 * 1 * 8 * 1024 * 32 * 2                  # projected keys
-    bad = b.tb_config(2, 8, 8, 96, 32, b.TB_BF16, 1, 1024, 64, 1, 0)
+    bad = b.tb_config(2, 8, 8, 96, 32, b.TB_BF16, 1, 1024, 64, 1, 0, 0)
     assert L.tb_query_sizes(ctypes.byref(bad), *[ctypes.byref(s) for s in sizes]) == b.TB_ERR_UNSUPPORTED
-    bad = b.tb_config(2, 9, 8, 128, 32, b.TB_BF16, 1, 1024, 64, 1, 0)
+    bad = b.tb_config(2, 9, 8, 128, 32, b.TB_BF16, 1, 1024, 64, 1, 0, 0)
     assert L.tb_query_sizes(ctypes.byref(bad), *[ctypes.byref(s) for s in sizes]) == b.TB_ERR_INVALID_ARG
     assert L.tb_status_string(b.TB_ERR_UNPROJECTED) == b"candidate keys not projected"
 

@@ -28,18 +28,20 @@ def tb():
 
 def full_pipeline_check(H, case, p, step=0, dense_too=False):
     """select (vs oracle, with the near-tie rule) then attention from the stored lists (vs oracle on
-    the GPU's own list, and end to end when the sets agree)."""
+    the GPU's own list, and end to end when the sets agree).  Written over the case's lists and
+    attention units, so it serves every selection scope."""
     w = case.w
     q, qi = H.queries(w, step)
+    qi = qi[:, :, :case.Hl * case.gl]                     # one list per layer: a single importance query
     lists = H.gpu_select(case, qi, p)
     assert case.ctx.get_status() == 0
     swaps = 0
     for l in range(w.n_layers):
         for b in range(w.batch):
-            for h in range(w.n_kv_heads):
+            for h in range(case.Hl):
                 base, full, s = case.oracle_select(l, b, h, qi[l, b], p)
                 if p.radius == 0:
-                    swaps += H.check_selection(lists[l][b][h], full, s, "layer %d seq %d head %d" % (l, b, h))
+                    swaps += H.check_selection(lists[l][b][h], full, s, "layer %d seq %d list %d" % (l, b, h))
                 else:
                     # neighbour lists follow from the base selection; compare exactly when the base sets agree
                     if np.array_equal(lists[l][b][h], full):
@@ -52,20 +54,20 @@ def full_pipeline_check(H, case, p, step=0, dense_too=False):
     worst = 0.0
     for l in range(w.n_layers):
         for b in range(w.batch):
-            for h in range(w.n_kv_heads):
-                ref, ref_lse = case.oracle_attention(l, b, h, q[l, b], lists[l][b][h], p)
-                got = out[l, b, h * w.group:(h + 1) * w.group]
+            for h in range(case.Ha):
+                ref, ref_lse = case.oracle_attention(l, b, h, q[l, b], lists[l][b][h * case.Hl // case.Ha], p)
+                got = out[l, b, h * case.ga:(h + 1) * case.ga]
                 worst = max(worst, np.abs(got - ref).max())
-                assert np.allclose(lse[l, b, h * w.group:(h + 1) * w.group], ref_lse, atol=2e-3 if w.dtype == wl.BF16 else 1e-5, rtol=1e-5)
+                assert np.allclose(lse[l, b, h * case.ga:(h + 1) * case.ga], ref_lse, atol=2e-3 if w.dtype == wl.BF16 else 1e-5, rtol=1e-5)
     assert worst <= H.ATTN_TOL[w.dtype], worst
     if dense_too:
         pd = tb().select_params(-1)
         outd, _ = H.gpu_attention(case, q, pd)
         for l in range(w.n_layers):
             for b in range(w.batch):
-                for h in range(w.n_kv_heads):
+                for h in range(case.Ha):
                     ref, _ = case.oracle_attention(l, b, h, q[l, b], None, p, dense=True)
-                    assert np.abs(outd[l, b, h * w.group:(h + 1) * w.group] - ref).max() <= H.ATTN_TOL[w.dtype]
+                    assert np.abs(outd[l, b, h * case.ga:(h + 1) * case.ga] - ref).max() <= H.ATTN_TOL[w.dtype]
     return swaps, worst
 
 
@@ -493,7 +495,7 @@ def test_kv_cache_in_pinned_host_memory(H):
     assert np.array_equal(oa, ob) and np.array_equal(sa, sb) and np.array_equal(oa2, ob2) and np.array_equal(sa2, sb2)
     # pageable host memory is not addressable by the device: refused, nothing launched
     b = tb()
-    cfg = b.tb_config(1, 8, 8, 128, 32, b.TB_BF16, 1, 256, 16, 0, 0)
+    cfg = b.tb_config(1, 8, 8, 128, 32, b.TB_BF16, 1, 256, 16, 0, 0, 0)
     sizes = [ctypes.c_size_t() for _ in range(4)]
     assert b.lib().tb_query_sizes(ctypes.byref(cfg), *[ctypes.byref(s) for s in sizes]) == b.TB_OK
     dev = [torch.empty(s.value + 256, dtype=torch.uint8, device="cuda") for s in sizes]

@@ -419,3 +419,18 @@ def test_predictor_closed_forms(orc):
     qa = orc.predict_queries(H, one[0], b, W1, W2, F32, eps=0.0)
     qb = orc.predict_queries((4.0 * H).astype(np.float32), one[0], b, W1, W2, F32, eps=0.0)   # 4 h is exact in fp32
     assert np.allclose(qa, qb, rtol=1e-12, atol=1e-12)
+
+
+def test_per_layer_projection_is_the_sum_of_the_heads_projections(orc):
+    """One list per layer (App. "additional evaluation", head-less predictor): the projection of a token's
+    concatenated key [Hkv*D] by the stacked W_K [Hkv*D][d'] is the sum over heads of the per-head
+    projections; checked on integer-valued inputs, where both sides are exact."""
+    rng = np.random.default_rng(5)
+    Hkv, T, D, dp = 4, 9, 128, 16
+    K = rng.integers(-3, 4, size=(Hkv, T, D)).astype(np.float32)
+    W = rng.integers(-2, 3, size=(Hkv, D, dp)).astype(np.float32)
+    _, cat = orc.project_keys(np.ascontiguousarray(np.concatenate(list(K), axis=1)), np.ascontiguousarray(np.concatenate(list(W), axis=0)),
+                              orc.F32, want_f64=True)
+    per_head = sum(orc.project_keys(np.ascontiguousarray(K[h]), np.ascontiguousarray(W[h]), orc.F32, want_f64=True)[1] for h in range(Hkv))
+    assert np.array_equal(cat, per_head)
+    assert np.array_equal(cat, np.einsum("htc,hcj->tj", K.astype(np.float64), W.astype(np.float64)))

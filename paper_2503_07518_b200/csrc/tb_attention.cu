@@ -36,6 +36,16 @@ struct RowMap {
         }
         return w_begin + (r - n_list);
     }
+    // the same with a bad list entry reported as -1 (nothing else depends on the loaded value)
+    __device__ __forceinline__ int token_or_neg(int r) const {
+        if (dense || r < n_sink) return r;
+        r -= n_sink;
+        if (r < n_list) {
+            const int t = list[r];
+            return (t < 0 || t >= L) ? -1 : t;
+        }
+        return w_begin + (r - n_list);
+    }
 };
 
 // An attention unit is (layer, sequence, head h < Ha): one KV head with its group of query heads, or,
@@ -418,22 +428,24 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
         }
     };
     auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
-    auto issue = [&](int tile) {
-        bool bad;
-        const int t = lane < kTileTok ? rm.token(min(wb + tile * kTileTok + lane, we - 1), bad) : 0;
-        issue_token(tile, t);
-    };
     attn_stamp(1);
+    // Lane i < 16 keeps, one bit per tile from the current one on, whether its row of that tile is a
+    // bad list entry (outside the cached tokens): known when the tile's rows are issued, used when
+    // the tile is consumed.  (Reading the entry a second time at consumption, as an earlier version did,
+    // cost 5-8% of the kernel; fetching the entries one tile ahead of their issue cost 4% on
+    // bandwidth-saturated launches and is not done.)
+    uint32_t bad_bits = 0;
+    auto tokens_of = [&](int tile) {                // -1 = bad entry
+        return (tile < n_tiles && lane < kTileTok) ? rm.token_or_neg(min(wb + tile * kTileTok + lane, we - 1)) : 0;
+    };
     {   // the first tiles' list entries are fetched together (one memory round trip), then their rows
         int tok[kMmaStages];
 #pragma unroll
-        for (int t = 0; t < kMmaStages; ++t) {
-            bool bad;
-            tok[t] = (t < n_tiles && lane < kTileTok) ? rm.token(min(wb + t * kTileTok + lane, we - 1), bad) : 0;
-        }
+        for (int t = 0; t < kMmaStages; ++t) tok[t] = tokens_of(t);
 #pragma unroll
         for (int t = 0; t < kMmaStages; ++t) {
-            if (t < n_tiles) issue_token(t, tok[t]);
+            bad_bits |= (uint32_t)(tok[t] < 0) << t;
+            if (t < n_tiles) issue_token(t, max(tok[t], 0));
             commit();
         }
     }
@@ -471,14 +483,11 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
         const int st = tile % kMmaStages;
         const int r0 = wb + tile * kTileTok;
         // validity of the tile's 16 rows (past-the-end and out-of-range list entries are masked)
-        bool ok = false;
-        if (lane < kTileTok && r0 + lane < we) {
-            bool bad;
-            rm.token(r0 + lane, bad);
-            ok = !bad;
-            any_bad |= bad;
-        }
-        const unsigned vmask = __ballot_sync(0xffffffffu, ok);
+        const bool in_range = lane < kTileTok && r0 + lane < we;
+        const bool bad = in_range && (bad_bits & 1u);
+        any_bad |= bad;
+        bad_bits >>= 1;
+        const unsigned vmask = __ballot_sync(0xffffffffu, in_range && !bad);
         asm volatile("cp.async.wait_group %0;" ::"n"(kMmaStages - 1) : "memory");
         __syncwarp();                                  // every lane's copies of this tile are visible to the warp
         if (tile == 0) attn_stamp(3);
@@ -535,7 +544,11 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
             mma_bf16(o[mt], a0, a1, a2, a3, bl0, bl1);
         }
         __syncwarp();                                  // the warp is done reading this stage
-        if (tile + kMmaStages < n_tiles) issue(tile + kMmaStages);
+        if (tile + kMmaStages < n_tiles) {
+            const int t = tokens_of(tile + kMmaStages);
+            bad_bits |= (uint32_t)(t < 0) << (kMmaStages - 1);         // bit k is tile + 1 + k now
+            issue_token(tile + kMmaStages, max(t, 0));
+        }
         commit();
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");

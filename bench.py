@@ -37,6 +37,7 @@ NCU_TRAFFIC_BYTES = {
     ("cfg2_llama8b_32k", "select_kernel"): 67_198_720 + 815_872,   # profiles/select_kernel_cfg2_32k.md
     ("cfg2_llama8b_32k", "attn_kernel"): 13_579_264,               # profiles/attn_mma_kernel_cfg2_32k.md
     ("cfg3_batched_serving", "select_kernel"): 398_913_792 + 4_822_528,   # profiles/select_wave_kernel_cfg3_batched.md
+    ("cfg4_long_context_128k", "select_kernel"): 268_044_288 + 3_600_384,  # profiles/select_cw_kernel_cfg4_128k.md
 }
 
 

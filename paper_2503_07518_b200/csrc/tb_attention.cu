@@ -327,8 +327,14 @@ __device__ __forceinline__ void attn_stamp(int) {}
 #endif
 
 constexpr int kTileTok = 16;
-constexpr int kRowPitch = 528;                        // 512 B of K|V + 16 B pad
-constexpr int kStageBytes = kTileTok * kRowPitch;     // 8448
+// A stage holds 16 K|V rows at a pitch of 512 bytes; the 16-byte chunk c of row i sits at chunk
+// c ^ (i & 7), so the eight rows of an ldmatrix tile hit eight different bank groups without padding.
+// Every 128-byte line of a source row therefore lands in one 128-byte line of shared memory and the
+// copy of a row is four full-line requests.  (With a padded pitch of 528 a source line straddled two
+// destination lines and was split: invisible in HBM, but over the host link, where every request is
+// its own read transaction, it halved the throughput of a cache in page-locked host memory.)
+constexpr int kRowPitch = 512;
+constexpr int kStageBytes = kTileTok * kRowPitch;     // 8192
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -419,12 +425,13 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     // kMmaStages-1 groups are complete" always means "the tile about to be used has landed".
     const uint32_t stage_u32 = smem_u32(my_stage);
     auto issue_token = [&](int tile, int t) {     // t: lane i < 16 holds the token of row i
-        const uint32_t dst = stage_u32 + (tile % kMmaStages) * kStageBytes + lane * 16;
+        const uint32_t dst = stage_u32 + (tile % kMmaStages) * kStageBytes;
         const unsigned char* src = kv_unit + lane * 16;
 #pragma unroll
         for (int i = 0; i < kTileTok; ++i) {
             const int ti = __shfl_sync(0xffffffffu, t, i);
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * kRowPitch), "l"(src + (size_t)ti * 512) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * kRowPitch + ((lane ^ (i & 7)) << 4)),
+                         "l"(src + (size_t)ti * 512) : "memory");
         }
     };
     auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
@@ -476,8 +483,10 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
 
     // per-lane ldmatrix row addresses inside a stage
     const int mi = lane >> 3, r8 = lane & 7;
-    const uint32_t k_lane_off = ((mi & 1) * 8 + r8) * kRowPitch + (mi >> 1) * 16;          // + ks * 32   (A of S = K Q^T)
-    const uint32_t v_lane_off = ((mi >> 1) * 8 + r8) * kRowPitch + 256 + (mi & 1) * 16;    // + mt * 32   (A of O^T = V^T P^T)
+    // row offset + swizzled chunk: chunk 2 ks + (mi >> 1) of the K half, 16 + 2 mt + (mi & 1) of the V half,
+    // each xor (row & 7) = r8; the k-step / channel-tile part is xored in at the use
+    const uint32_t k_row_off = ((mi & 1) * 8 + r8) * kRowPitch, k_swz = (uint32_t)((mi >> 1) ^ r8) << 4;        // ^ ks * 32   (A of S = K Q^T)
+    const uint32_t v_row_off = ((mi >> 1) * 8 + r8) * kRowPitch + 256, v_swz = (uint32_t)((mi & 1) ^ r8) << 4;  // ^ mt * 32   (A of O^T = V^T P^T)
 
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int st = tile % kMmaStages;
@@ -498,7 +507,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t a0, a1, a2, a3;
-            ldmatrix_x4(sb + k_lane_off + ks * 32, a0, a1, a2, a3);
+            ldmatrix_x4(sb + k_row_off + ((ks * 32) ^ k_swz), a0, a1, a2, a3);
             mma_bf16(sc, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
         }
         const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
@@ -539,7 +548,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
             uint32_t a0, a1, a2, a3;
-            ldmatrix_x4_trans(sb + v_lane_off + mt * 32, a0, a1, a2, a3);
+            ldmatrix_x4_trans(sb + v_row_off + ((mt * 32) ^ v_swz), a0, a1, a2, a3);
             mma_bf16(o[mt], a0, a1, a2, a3, bh0, bh1);
             mma_bf16(o[mt], a0, a1, a2, a3, bl0, bl1);
         }

@@ -119,11 +119,12 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTabl
 
 // bf16 storage: the projection is the one dense contraction of the path ([tokens x 128] . [128 x d']
 // per KV head), so it runs on the tensor cores: 128 tokens per block, K rows and the W_K slice staged
-// in shared memory with 16-byte cp.async at conflict-free pitches, mma.sync m16n8k16 with fp32
+// in shared memory with 16-byte cp.async (K rows unpadded with an XOR swizzle of their 16-byte chunks, so
+// that a source line is one full-line request and ldmatrix still sees eight bank groups), mma.sync m16n8k16 with fp32
 // accumulation, one round-to-nearest-even to bf16.  HBM-bound: 256 B read + 2 d' B written per token.
 constexpr int kPmTokens = 128;
 constexpr int kPmThreads = 128;
-constexpr int kPmKPitch = 272;            // 256 B of K + 16 B pad
+constexpr int kPmKPitch = 256;            // 256 B of K per token, 16-byte chunk c of row t at chunk c ^ (t & 7)
 
 template <int DP>
 __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTable ut, ProjectTable pt,
@@ -133,7 +134,7 @@ __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTa
     constexpr int D = 128;
     constexpr int kWPitch = DP * 2 + 16;  // bytes per W row (one channel, d' outputs) + pad
     constexpr int NT = DP / 8;            // 8-wide output tiles
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* Ks = smem;                                  // [128 tokens][kPmKPitch]
     unsigned char* Ws = smem + kPmTokens * kPmKPitch;          // [128 channels][kWPitch]
 
@@ -167,7 +168,7 @@ __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTa
         for (int i = tid; i < kPmTokens * 16; i += kPmThreads) {          // 16 chunks of 16 B per K row
             const int t = i >> 4, ch = i & 15;
             const int tc = min(t, nt_valid - 1);                           // rows past the range repeat the last one
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ks_u32 + t * kPmKPitch + ch * 16),
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ks_u32 + t * kPmKPitch + ((ch ^ (t & 7)) << 4)),
                          "l"(kbase + (size_t)tc * 512 + ch * 16) : "memory");
         }
         for (int i = tid; i < D * (DP / 8); i += kPmThreads) {             // DP/8 chunks per W row
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTa
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 uint32_t a0, a1, a2, a3;
-                const uint32_t addr = ks_u32 + (tok + (mi & 1) * 8 + r8) * kPmKPitch + ks * 32 + (mi >> 1) * 16;
+                const uint32_t addr = ks_u32 + (tok + (mi & 1) * 8 + r8) * kPmKPitch + ((ks * 32) ^ (((mi >> 1) ^ r8) << 4));
                 asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
 #pragma unroll
                 for (int n = 0; n < NT; ++n)

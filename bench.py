@@ -35,9 +35,10 @@ UNIT = "tokens/s"
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
     ("cfg2_llama8b_32k", "select_kernel"): 67_198_720 + 815_872,   # profiles/select_kernel_cfg2_32k.md
-    ("cfg2_llama8b_32k", "attn_kernel"): 13_579_264,               # profiles/attn_mma_kernel_cfg2_32k.md
+    ("cfg2_llama8b_32k", "attn_kernel"): 13_582_080,               # profiles/attn_mma_kernel_cfg2_32k.md
     ("cfg3_batched_serving", "select_kernel"): 398_913_792 + 4_822_528,   # profiles/select_wave_kernel_cfg3_batched.md
     ("cfg4_long_context_128k", "select_kernel"): 268_044_288 + 3_600_384,  # profiles/select_cw_kernel_cfg4_128k.md
+    ("cfg5_interval_neighbors", "attn_kernel"): 309_482_496 + 3_839_488,   # profiles/attn_mma_kernel_cfg5_interval.md
 }
 
 
@@ -541,7 +542,8 @@ def run_trajectory(args, w):
                                     "gbs": att_bytes / (att_ms * 1e-3) / 1e9, "launches_per_step": w.n_layers}},
         "roofline": {"bound": "hbm", "kernel": "attn_mma_kernel", "achieved": att_bytes / (att_ms * 1e-3) / 1e9,
                      "peak": peak, "unit": "GB/s", "frac": att_bytes / (att_ms * 1e-3) / 1e9 / peak, "peak_kind": "of " + peak_kind,
-                     "traffic": None, "bytes_per_launch": att_bytes, "us_per_launch": att_ms * 1e3},
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, "attn_kernel")) if w.nmode == 0 else None,
+                     "bytes_per_launch": att_bytes, "us_per_launch": att_ms * 1e3},
         "clocks": sampler.summary(),
     }
     if rank == 0:

@@ -52,6 +52,8 @@ struct WaveOrder {
 #ifdef TB_PHASE_TIMING
 __device__ unsigned long long g_fin_ns[8];
 __device__ unsigned long long g_cw_ns[8];
+__device__ unsigned int g_wave_smid[1024];
+__device__ unsigned long long g_fin_blk[4][1024];
 __device__ unsigned long long g_wave_ns[4][1024];       // per block: start, first tile landed, rows streamed, end
 __device__ __forceinline__ unsigned long long wave_now() {
     unsigned long long t;
@@ -63,6 +65,11 @@ __device__ __forceinline__ void wave_stamp(int i) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         g_wave_ns[i][blockIdx.x] = t;
+        if (i == 0) {
+            unsigned smid;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            g_wave_smid[blockIdx.x] = smid;
+        }
     }
 }
 #else
@@ -167,7 +174,7 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
     const int tid = threadIdx.x, lane = tid & 31;
 #ifdef TB_PHASE_TIMING
     unsigned long long tf0 = wave_now();
-#define FIN_MARK(i) do { if (tid == 0) { unsigned long long tn = wave_now(); atomicAdd(&g_fin_ns[i], tn - tf0); tf0 = tn; } } while (0)
+#define FIN_MARK(i) do { if (tid == 0) { unsigned long long tn = wave_now(); atomicAdd(&g_fin_ns[i], tn - tf0); if (blockIdx.x < 1024 && (i) < 4) g_fin_blk[i][blockIdx.x] = tn - tf0; tf0 = tn; } } while (0)
 #else
 #define FIN_MARK(i) do {} while (0)
 #endif
@@ -194,7 +201,6 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
     // nibble, eight lanes' nibbles make a mask word.
     const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
     const int n_vec = (ncand + 3) / 4;
-    const uint32_t oct = 0xffu << (lane & 24);         // the eight lanes that share a mask word
     for (int v0 = tid; v0 < n_grp * (kRows / 4); v0 += kThreads * kBatch) {   // kBatch loads in flight, then their verdicts
         uint4 x[kBatch];
 #pragma unroll
@@ -216,7 +222,10 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
                 take |= (uint32_t)(valid && (c > bin || (c == bin && exact))) << e;
                 eqm |= (uint32_t)(valid && c == bin) << e;
             }
-            const uint32_t word = __reduce_or_sync(oct, take << (4 * (lane & 7)));
+            uint32_t word = take << (4 * (lane & 7));  // three shuffles: a reduction over a part of the warp was far slower
+            word |= __shfl_xor_sync(0xffffffffu, word, 1);
+            word |= __shfl_xor_sync(0xffffffffu, word, 2);
+            word |= __shfl_xor_sync(0xffffffffu, word, 4);
             if ((lane & 7) == 0) mask[v >> 3] = word;  // positions 32 (v / 8) .. + 31
             if (!exact && __any_sync(0xffffffffu, eqm != 0)) {
                 const int ne = __popc(eqm);
@@ -599,6 +608,8 @@ __global__ void __launch_bounds__(kThreads, 4)
 #ifdef TB_PHASE_TIMING
 extern "C" int tb_debug_cw_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_cw_ns, sizeof(g_cw_ns)); }
 extern "C" int tb_debug_fin_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_fin_ns, sizeof(g_fin_ns)); }
+extern "C" int tb_debug_wave_smid(unsigned int* out) { return (int)cudaMemcpyFromSymbol(out, g_wave_smid, sizeof(g_wave_smid)); }
+extern "C" int tb_debug_fin_blk(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_fin_blk, sizeof(g_fin_blk)); }
 extern "C" int tb_debug_wave_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_wave_ns, sizeof(g_wave_ns)); }
 #endif
 

@@ -33,7 +33,10 @@ constexpr int kBins = 2048;         // 11-bit digits (the last digit has 10 bits
 constexpr int kMaxCluster = 8;
 constexpr int kMaxKeysPerBlock = 32768;   // 128 KB of on-chip keys per block at most
 constexpr int kListCap = 256;       // non-empty first-digit bins a block may publish on the fast path
-constexpr int kCwFrom = 48 * 1024;   // candidates from which the parked-key cluster kernel takes over
+#ifndef TB_CW_FROM
+#define TB_CW_FROM (48 * 1024)
+#endif
+constexpr int kCwFrom = TB_CW_FROM;   // candidates from which the parked-key cluster kernel takes over (macro: tuning builds)
 constexpr int kCwLimit = 8 * 32768;  // ... and up to which it can (8 blocks x 64 KB of first digits)
 constexpr int kCandCap = 4096;      // keys of the threshold bin gathered at rank 0 (aliases merged[1..2])
 

@@ -978,16 +978,22 @@ __global__ void __launch_bounds__(kThreads, 2)
 
     // ---- every block ranks the list itself ------------------------------------------------------------
     if (!exact) {
-        int r_of = 0, i_of = tid;                      // thread t takes entry t of the concatenated regions
+        // the regions' entries side by side first (one entry per thread), so that the ranking loop runs
+        // over one short array with a single bound
+        uint2* all = list + C * kCwListCap;
+        int r_of = 0, i_of = tid, n_all = 0;
+        for (unsigned r = 0; r < C; ++r) n_all += cs->n_in[r];
         while (r_of < (int)C && i_of >= cs->n_in[r_of]) i_of -= cs->n_in[r_of], ++r_of;
+        uint2 it = make_uint2(0u, 0u);
+        if (r_of < (int)C) it = list[r_of * kCwListCap + i_of], all[tid] = it;
+        __syncthreads();
         if (r_of < (int)C) {
-            const uint2 it = list[r_of * kCwListCap + i_of];
             int before = 0;                            // larger key, or equal key at a lower position
-            for (unsigned r = 0; r < C; ++r)
-                for (int j = 0; j < cs->n_in[r]; ++j) {
-                    const uint2 o = list[r * kCwListCap + j];
-                    before += (o.x > it.x) | ((o.x == it.x) & (o.y < it.y));
-                }
+#pragma unroll 4
+            for (int j = 0; j < n_all; ++j) {
+                const uint2 o = all[j];
+                before += (o.x > it.x) | ((o.x == it.x) & (o.y < it.y));
+            }
             if (before < krem) {
                 atomicAdd(&cs->winners[r_of], 1);
                 if (r_of == (int)rank) {
@@ -1045,7 +1051,7 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
     const int tile_bytes = kRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
     const size_t fixed = 1024 + kDigitBins * sizeof(int) + (size_t)tiles_per_cta * kRows * 2 + (size_t)tiles_per_cta * (kRows / 32) * 4 +
                          sizeof(CwSmem);
-    const size_t ring_min = (size_t)C * kCwListCap * sizeof(uint2);   // list regions
+    const size_t ring_min = (size_t)(C + 1) * kCwListCap * sizeof(uint2);   // list regions + the entries side by side
     const size_t budget = (size_t)(C * n_units > c->sm_count ? 113 : 224) * 1024;
     if (fixed + ring_min > 224 * 1024) return cudaErrorInvalidConfiguration;
     int n_stages = fixed < budget ? (int)((budget - fixed) / tile_bytes) : 0;

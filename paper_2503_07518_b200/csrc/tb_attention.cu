@@ -668,6 +668,9 @@ static int pick_nsplit(const tb_ctx* c, int units, int max_rows) {
     // (256 blocks) ran at 58.5 us, 5 at 63.6, 6 at 61.5, 7 (448 blocks, four more than fit at once) at 75.7,
     // 10 at 65.0
     int n = 2 * c->sm_count / units;
+#ifdef TB_FORCE_NSPLIT
+    n = TB_FORCE_NSPLIT;
+#endif
     int by_rows = max_rows / 64;
     if (n > by_rows) n = by_rows;
     if (n > kMaxSplits) n = kMaxSplits;

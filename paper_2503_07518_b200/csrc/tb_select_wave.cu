@@ -191,6 +191,11 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
     if (mask_bytes > scratch_bytes || (!exact && (bc > (scratch_bytes - mask_bytes) / 8 || bin == 0))) return false;
     const uint32_t bin_base = dg.base + ((uint32_t)(bin - 1) << dg.shift);       // lowest key of the threshold bin
     const int bin_bits = bin == 2047 ? 32 : dg.shift;  // bits of (key - bin_base) inside the bin; the top bin is open-ended
+    // Keys of the threshold bin: [bin_from, above_from); keys of the bins above it: [above_from, 2^32), if any.
+    // Bin 0 holds the keys below the digit's base, bin 2047 is open-ended.
+    const uint64_t above64 = bin == 0 ? (uint64_t)dg.base : bin == 2047 ? (1ull << 32) : (uint64_t)dg.base + ((uint64_t)bin << dg.shift);
+    const uint32_t above_mask = above64 <= 0xffffffffull ? 0xfu : 0u;
+    const uint32_t above_from = (uint32_t)above64, bin_from = bin == 0 ? 0u : bin_base;
     if (tid == 0) sm->n_list = 0;
     __syncthreads();
 #ifdef TB_PHASE_TIMING
@@ -214,14 +219,19 @@ __device__ __forceinline__ bool wave_finish_mask(int* hist, WaveSmem* sm, const 
             const int v = v0 + u * kThreads;
             if (v - lane >= n_grp * (kRows / 4)) break;    // warp-uniform: whole warps leave together
             const uint32_t kk[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
-            uint32_t take = 0, eqm = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int c = dg.bin(kk[e]);
-                const bool valid = v * 4 + e < ncand;
-                take |= (uint32_t)(valid && (c > bin || (c == bin && exact))) << e;
-                eqm |= (uint32_t)(valid && c == bin) << e;
+            // the keys' digits against the threshold bin, as compares with the bin's two bounds (the pass
+            // is bound by instruction issue: a digit per key, with a validity test per key, cost 2.5 x as much)
+            uint32_t ab = (uint32_t)(kk[0] >= above_from) | (uint32_t)(kk[1] >= above_from) << 1 | (uint32_t)(kk[2] >= above_from) << 2 |
+                          (uint32_t)(kk[3] >= above_from) << 3;
+            uint32_t ge = (uint32_t)(kk[0] >= bin_from) | (uint32_t)(kk[1] >= bin_from) << 1 | (uint32_t)(kk[2] >= bin_from) << 2 |
+                          (uint32_t)(kk[3] >= bin_from) << 3;
+            ab &= above_mask;
+            if (v * 4 + 3 >= ncand) {                  // the problem's last vector (and the padding after it)
+                const uint32_t vm = v * 4 < ncand ? (1u << (ncand - v * 4)) - 1u : 0u;
+                ab &= vm, ge &= vm;
             }
+            const uint32_t eqm = ge & ~ab;
+            const uint32_t take = exact ? ge : ab;
             uint32_t word = take << (4 * (lane & 7));  // three shuffles: a reduction over a part of the warp was far slower
             word |= __shfl_xor_sync(0xffffffffu, word, 1);
             word |= __shfl_xor_sync(0xffffffffu, word, 2);

@@ -19,6 +19,11 @@ __global__ void append_kernel(Geom gm, UnitTable ut, AppendTable at, int total_n
     const int chunks_per_pair = 2 * chunks_per_row;
     const int ll = blockIdx.y;
     const long long work = (long long)total_new * gm.Hkv * chunks_per_pair;
+    // Launched as a programmatic dependent (a decode step appends right after the previous layer's
+    // attention): resident early, but the new rows may come from the predecessor and the cache rows
+    // written here may still be read by it, so wait first; the successor may then get ready.
+    pdl_wait();
+    pdl_launch_dependents();
     for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < work; w += (long long)gridDim.x * blockDim.x) {
         int chunk = (int)(w % chunks_per_pair);
         long long th = w / chunks_per_pair;
@@ -47,13 +52,16 @@ cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new
     int threads = 256;
     long long blocks = (work + threads - 1) / threads;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    dim3 grid((unsigned)blocks, ut.layer_count);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, ut.layer_count, 1), cfg.blockDim = dim3(threads, 1, 1), cfg.dynamicSmemBytes = 0, cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see pdl_wait()
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
     if (gm.dtype == TB_BF16)
-        append_kernel<__nv_bfloat16><<<grid, threads, 0, s>>>(gm, ut, at, total_new, (const __nv_bfloat16*)k,
-                                                            (const __nv_bfloat16*)v, (__nv_bfloat16*)c->kv);
-    else
-        append_kernel<float><<<grid, threads, 0, s>>>(gm, ut, at, total_new, (const float*)k, (const float*)v, (float*)c->kv);
-    return cudaGetLastError();
+        return cudaLaunchKernelEx(&cfg, append_kernel<__nv_bfloat16>, gm, ut, at, total_new, (const __nv_bfloat16*)k,
+                                  (const __nv_bfloat16*)v, (__nv_bfloat16*)c->kv);
+    return cudaLaunchKernelEx(&cfg, append_kernel<float>, gm, ut, at, total_new, (const float*)k, (const float*)v, (float*)c->kv);
 }
 
 // ---------------------------------------------------------------------------------------------

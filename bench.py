@@ -225,14 +225,17 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode)
+    scope = {"kv_head": tbh.TB_SCOPE_KV_HEAD, "q_head": tbh.TB_SCOPE_Q_HEAD, "layer": tbh.TB_SCOPE_LAYER}[args.list_scope]
     ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + 8,
-                      w.budget, w.radius, device=local, kv_on_host=args.offload_kv)
+                      w.budget, w.radius, device=local, kv_on_host=args.offload_kv, list_scope=scope)
     proj_info = fill_caches(ctx, w, torch, tbh)
     dt = tbh.torch_dtype(w.dtype)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(wl.seed_for(w.cfg_id, 0, 0, wl.TAG_Q))
     q = torch.randn(w.n_layers, w.batch, w.n_q_heads, w.head_dim, generator=gen, device="cuda").to(dt)
     qi = torch.randn(w.n_layers, w.batch, w.n_q_heads, w.imp_dim, generator=gen, device="cuda")
+    if scope == tbh.TB_SCOPE_LAYER:                          # the head-less predictor: one importance query per layer
+        qi = qi[:, :, :1].contiguous()
     out = torch.empty(w.n_layers, w.batch, w.n_q_heads, w.head_dim, device="cuda")
     q_host, qi_host = q.cpu().pin_memory(), qi.cpu().pin_memory()
     out_host = torch.empty_like(out, device="cpu").pin_memory()
@@ -357,7 +360,8 @@ def run_ours(args, w):
         "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name + ("+offloaded_kv" if args.offload_kv else ""), "layers": w.n_layers, "batch_per_gpu": w.batch,
+        "config": {"workload": w.name + ("+offloaded_kv" if args.offload_kv else "") +
+                   ("+lists_per_" + args.list_scope if args.list_scope != "kv_head" else ""), "layers": w.n_layers, "batch_per_gpu": w.batch,
                    "q_heads": w.n_q_heads,
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "imp_dim": w.imp_dim,
                    "kv_storage": "bf16" if w.dtype == wl.BF16 else "f32", "context": w.lengths if len(set(w.lengths)) > 1 else w.lengths[0],
@@ -390,7 +394,7 @@ def run_ours(args, w):
         "clocks": sampler.summary(),
     }
     if rank == 0:
-        if world == 1 and not args.no_cpu:
+        if world == 1 and not args.no_cpu and args.list_scope == "kv_head":   # the oracle sample below is per KV head
             leg = cpu_leg(w, args.cpu_layers, 3)
             best = min(leg["times"])
             line["cpu_baseline"] = {"value": w.batch / best, "unit": UNIT, "cores": leg["threads"], "kind": "oracle",
@@ -565,6 +569,8 @@ def main():
     ap.add_argument("--profile", action="store_true", help="only warm-up + steps of plain launches (for ncu)")
     ap.add_argument("--offload-kv", action="store_true",
                     help="K|V cache in page-locked host memory (selected rows cross the host link); also times the dense step")
+    ap.add_argument("--list-scope", default="kv_head", choices=["kv_head", "q_head", "layer"],
+                    help="which heads share an index list (configs 1-4; default: one list per KV head)")
     ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
                     help="neighbour rule of the interval workload (default: its own, +-r dilation)")
     args = ap.parse_args()

@@ -367,7 +367,7 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                 int lo, hi;
                 cand_range(c->len[u], p->sinks, p->recent, &lo, &hi);
                 if (c->len_proj[u] < hi) return TB_ERR_UNPROJECTED;
-                bytes += (uint64_t)(hi - lo) * c->geom.Hl * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);   // every list streams its keys
+                bytes += (uint64_t)(hi - lo) * c->geom.Hi * c->cfg.imp_dim * elem_size(c->cfg.kv_dtype);   // every key stream once (lists that share one re-read it from L2)
             }
     } else {
         for (int l = lb; l < lb + lc; ++l)

@@ -17,7 +17,7 @@ int elem_size(int dtype) { return dtype == TB_BF16 ? 2 : 4; }
 struct Layout {
     size_t kv_bytes, kimp_bytes;
     size_t off_W, off_idx, off_cnt, off_status, off_counter, state_bytes;
-    size_t off_part_o, off_part_ml, off_sel_idx, off_sel_cnt, off_sel_keys, work_bytes;
+    size_t off_part_o, off_part_ml, off_sel_idx, off_sel_cnt, off_sel_keys, off_sel_bins, work_bytes;
     int idx_cap, sel_stride;
 };
 
@@ -72,6 +72,7 @@ void compute_layout(const tb_config* c, Layout* l) {
     l->off_sel_cnt = o, o = align_up(o + units * 4, 256);
     const size_t row = align_up((size_t)c->max_seq_len, 256);
     l->off_sel_keys = o, o = align_up(o + units * row * 4, 256);       // one 32-bit key per token
+    l->off_sel_bins = o, o = align_up(o + units * row * 2, 256);       // one 16-bit first digit per token
     l->work_bytes = o;
 }
 
@@ -203,6 +204,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->wk.sel_cnt = (int32_t*)(wp + l.off_sel_cnt);
     c->wk.sel_stride = l.sel_stride;
     c->wk.sel_keys = (uint32_t*)(wp + l.off_sel_keys);
+    c->wk.sel_bins = (uint16_t*)(wp + l.off_sel_bins);
     Geom& g = c->geom;
     g.n_layers = cfg->n_layers, g.Hq = cfg->n_q_heads, g.Hkv = cfg->n_kv_heads, g.g = cfg->n_q_heads / cfg->n_kv_heads;
     scope_heads(cfg, &g.Hi, &g.Hl, &g.Ha);

@@ -86,6 +86,7 @@ struct DevWork {
     int32_t* sel_cnt;
     int sel_stride;
     uint32_t* sel_keys;   // [n_layers*max_batch*Hl][max_seq_len rounded up to 256]  score keys of a many-problem selection launch
+    uint16_t* sel_bins;   // same shape, 2 bytes per token: first digits of a very long problem's rows, when they do not fit on chip
 };
 
 }  // namespace tb

@@ -37,7 +37,8 @@ constexpr int kListCap = 256;       // non-empty first-digit bins a block may pu
 #define TB_CW_FROM (48 * 1024)
 #endif
 constexpr int kCwFrom = TB_CW_FROM;   // candidates from which the parked-key cluster kernel takes over (macro: tuning builds)
-constexpr int kCwLimit = 8 * 32768;  // ... and up to which it can (8 blocks x 64 KB of first digits)
+constexpr int kCwLimit = 8 * 262144; // ... and up to which it can (8 blocks x 32 KB of bitmask; the rows' first digits move to the workspace when
+                                     // they no longer fit on chip)
 constexpr int kCandCap = 4096;      // keys of the threshold bin gathered at rank 0 (aliases merged[1..2])
 
 // Optional per-phase timestamps of the first and last block of unit 0, for tuning builds only
@@ -567,9 +568,9 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
         if (hi - lo > max_cand) max_cand = hi - lo;
     }
     // Many problems (one and a half per SM or more; measured crossover between 32 and 256 on 148 SMs)
-    // fill the GPU by themselves: one block each, no clusters.  So do problems too long for a cluster's
-    // on-chip key arrays.
-    if (2 * n_units >= 3 * c->sm_count || max_cand > kMaxCluster * kMaxKeysPerBlock) return launch_select_wave(c, ut, a, s);
+    // fill the GPU by themselves: one block each, no clusters.  So do problems beyond what the parked-key
+    // cluster kernel takes.
+    if (2 * n_units >= 3 * c->sm_count || max_cand > kCwLimit) return launch_select_wave(c, ut, a, s);
     // Long problems (beyond ~48K candidates) go to the cluster kernel that parks the keys in memory and
     // keeps 2 bytes per row on chip: two blocks per SM where this one, with 4 bytes per row, has room for
     // one (128K tokens: 70.1 -> 59.1 us per launch; at 32K the two are level, below that this one wins).

@@ -709,7 +709,7 @@ template <typename T, int DP, int RED>
 __global__ void __launch_bounds__(kThreads, 2)
     select_cw_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut, SelectArgs a,
                      int tiles_per_cta, int n_stages, int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt,
-                     int32_t* __restrict__ status, uint32_t* __restrict__ keys_g) {
+                     int32_t* __restrict__ status, uint32_t* __restrict__ keys_g, uint16_t* bins_g) {
     constexpr int RB = DP * Elem<T>::kBytes;
     constexpr int NCH = RB / 16;
     constexpr uint32_t kTileBytes = kRows * RB;
@@ -717,8 +717,10 @@ __global__ void __launch_bounds__(kThreads, 2)
     unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     const int ring_bytes = n_stages * (int)kTileBytes;
     int* hist = reinterpret_cast<int*>(stage_base + ring_bytes);                 // this block's first-digit histogram
-    uint16_t* bins = reinterpret_cast<uint16_t*>(hist + kDigitBins);             // first digit of every row of this block
-    uint32_t* mask = reinterpret_cast<uint32_t*>(bins + (size_t)tiles_per_cta * kRows);   // tiles_per_cta * 8 words
+    // first digit of every row of this block: on chip, or (bins_g: problems of several hundred thousand
+    // rows per block) in the workspace row, through the same pointer
+    uint16_t* bins_sm = reinterpret_cast<uint16_t*>(hist + kDigitBins);
+    uint32_t* mask = reinterpret_cast<uint32_t*>(bins_sm + (bins_g ? 0 : (size_t)tiles_per_cta * kRows));   // tiles_per_cta * 8 words
     CwSmem* cs = reinterpret_cast<CwSmem*>(mask + tiles_per_cta * (kRows / 32));
     WaveSmem* sm = &cs->w;
     // after the stream the ring holds the list (one region per rank)
@@ -770,6 +772,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     const int n_local = max(0, min(my_tiles * kRows, ncand - slot0));
     const long long row_base = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len + lo;              // row of candidate 0
     uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255);
+    uint16_t* bins = bins_g ? bins_g + cu * (size_t)((gm.max_seq_len + 255) & ~255) + slot0 : bins_sm;
     const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
 
     // sample row and query first, then the ring's opening requests (see the kernel above)
@@ -1059,11 +1062,16 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
     if (C < 1) C = 1;
     const int tiles_per_cta = (n_tiles + C - 1) / C > 0 ? (n_tiles + C - 1) / C : 1;
     const int tile_bytes = kRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
-    const size_t fixed = 1024 + kDigitBins * sizeof(int) + (size_t)tiles_per_cta * kRows * 2 + (size_t)tiles_per_cta * (kRows / 32) * 4 +
-                         sizeof(CwSmem);
     const size_t ring_min = (size_t)(C + 1) * kCwListCap * sizeof(uint2);   // list regions + the entries side by side
     const size_t budget = (size_t)(C * n_units > c->sm_count ? 113 : 224) * 1024;
-    if (fixed + ring_min > 224 * 1024) return cudaErrorInvalidConfiguration;
+    const size_t fixed_off = 1024 + kDigitBins * sizeof(int) + (size_t)tiles_per_cta * (kRows / 32) * 4 + sizeof(CwSmem);
+    const size_t bins_bytes = (size_t)tiles_per_cta * kRows * 2;
+    const size_t ring_least = ring_min > 2 * (size_t)tile_bytes ? ring_min : 2 * (size_t)tile_bytes;
+    // the rows' first digits stay on chip while they leave the block's share of the SM room for a ring; beyond that they
+    // live in the workspace
+    const bool digits_on_chip = fixed_off + bins_bytes + ring_least <= budget;
+    const size_t fixed = fixed_off + (digits_on_chip ? bins_bytes : 0);
+    if (fixed + ring_least > 224 * 1024) return cudaErrorInvalidConfiguration;
     int n_stages = fixed < budget ? (int)((budget - fixed) / tile_bytes) : 0;
     if (n_stages > kStagesMax) n_stages = kStagesMax;
     if (n_stages < 2) n_stages = 2;
@@ -1086,7 +1094,8 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
             if (e != cudaSuccess) return e;                                                                              \
         }                                                                                                                \
         return cudaLaunchKernelEx(&cfg, select_cw_kernel<T, DP, RED>, c->kimp_map, (const unsigned char*)c->kimp, gm, ut, a, \
-                                  tiles_per_cta, n_stages, c->st.idx, c->st.cnt, c->st.status, c->wk.sel_keys);          \
+                                  tiles_per_cta, n_stages, c->st.idx, c->st.cnt, c->st.status, c->wk.sel_keys,           \
+                                  digits_on_chip ? (uint16_t*)nullptr : c->wk.sel_bins);                                \
     } while (0)
 #define TB_CW(T, DP)                                                \
     do {                                                            \

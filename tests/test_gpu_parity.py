@@ -415,11 +415,15 @@ def test_many_problem_selection_kernel(H):
     _crafted_batch_case(H, _bf16_exact(r.standard_normal((n_seq, n_heads, 300))), budget=10, sinks=100, recent=200)
 
 
-def test_selection_beyond_cluster_capacity(H):
-    """A single problem with more candidates than a cluster keeps on chip (8 x 32768) goes to the
-    one-block-per-problem kernel, whose bitmask does not fit its scratch either: the general path."""
+def test_selection_of_very_long_problems(H):
+    """A single problem of 270K candidates: the parked-key cluster kernel with its rows' first digits on
+    chip.  One of 700K: more rows per block than shared memory holds digits for, so they live in the
+    workspace; ordinary scores, and a few distinct values (crowded threshold bins: the bin is cut again from
+    the parked keys, then the general path)."""
     r = np.random.Generator(np.random.PCG64(79))
     _crafted_scores_case(H, _bf16_exact(r.standard_normal((1, 270001))), budget=5000, sinks=4, recent=64)
+    _crafted_scores_case(H, _bf16_exact(r.standard_normal((1, 700001))), budget=9000, sinks=4, recent=64)
+    _crafted_scores_case(H, r.integers(0, 40, size=(1, 700001)).astype(np.float32), budget=30000)
 
 
 @pytest.mark.parametrize("act", [0, 1, 2])

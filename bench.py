@@ -571,12 +571,16 @@ def main():
                     help="K|V cache in page-locked host memory (selected rows cross the host link); also times the dense step")
     ap.add_argument("--list-scope", default="kv_head", choices=["kv_head", "q_head", "layer"],
                     help="which heads share an index list (configs 1-4; default: one list per KV head)")
+    ap.add_argument("--context", type=int, default=0,
+                    help="override every sequence's context length (e.g. --config 4 --context 1048576 --layers 8)")
     ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
                     help="neighbour rule of the interval workload (default: its own, +-r dilation)")
     args = ap.parse_args()
     w = wl.workload(args.config)
     if args.layers:
         w = w.scaled(n_layers=args.layers)
+    if args.context:
+        w = w.scaled(lengths=[args.context] * w.batch, name="%s@%d" % (w.name, args.context))
     if args.neighbors:
         w = w.scaled(nmode=0 if args.neighbors == "dilate" else 1)
     if args.impl == "reference":

@@ -709,7 +709,7 @@ template <typename T, int DP, int RED>
 __global__ void __launch_bounds__(kThreads, 2)
     select_cw_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut, SelectArgs a,
                      int tiles_per_cta, int n_stages, int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt,
-                     int32_t* __restrict__ status, uint32_t* __restrict__ keys_g, uint16_t* bins_g) {
+                     int32_t* __restrict__ status, uint32_t* __restrict__ keys_g, uint16_t* bins_g, int keep_in_l2) {
     constexpr int RB = DP * Elem<T>::kBytes;
     constexpr int NCH = RB / 16;
     constexpr uint32_t kTileBytes = kRows * RB;
@@ -773,7 +773,8 @@ __global__ void __launch_bounds__(kThreads, 2)
     const long long row_base = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len + lo;              // row of candidate 0
     uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255);
     uint16_t* bins = bins_g ? bins_g + cu * (size_t)((gm.max_seq_len + 255) & ~255) + slot0 : bins_sm;
-    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
+    // parked keys are kept in L2 for the block's return to them, unless the launch parks more than L2 can hold
+    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = keep_in_l2 ? l2_policy_evict_last() : stream_policy;
 
     // sample row and query first, then the ring's opening requests (see the kernel above)
     const bool sampled = ncand >= kMinSampled;
@@ -1072,6 +1073,8 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
     const bool digits_on_chip = fixed_off + bins_bytes + ring_least <= budget;
     const size_t fixed = fixed_off + (digits_on_chip ? bins_bytes : 0);
     if (fixed + ring_least > 224 * 1024) return cudaErrorInvalidConfiguration;
+    // 4 bytes of key (+ 2 of digit) per candidate: ask L2 to keep them only while a launch's worth fits comfortably
+    const int keep_in_l2 = (double)n_units * max_cand * (digits_on_chip ? 4 : 6) <= 64e6;
     int n_stages = fixed < budget ? (int)((budget - fixed) / tile_bytes) : 0;
     if (n_stages > kStagesMax) n_stages = kStagesMax;
     if (n_stages < 2) n_stages = 2;
@@ -1095,7 +1098,7 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
         }                                                                                                                \
         return cudaLaunchKernelEx(&cfg, select_cw_kernel<T, DP, RED>, c->kimp_map, (const unsigned char*)c->kimp, gm, ut, a, \
                                   tiles_per_cta, n_stages, c->st.idx, c->st.cnt, c->st.status, c->wk.sel_keys,           \
-                                  digits_on_chip ? (uint16_t*)nullptr : c->wk.sel_bins);                                \
+                                  digits_on_chip ? (uint16_t*)nullptr : c->wk.sel_bins, keep_in_l2);                    \
     } while (0)
 #define TB_CW(T, DP)                                                \
     do {                                                            \

@@ -461,7 +461,7 @@ __device__ __forceinline__ void wave_general(int* hist, WaveSmem* sm, const uint
 template <typename T, int DP, int RED>
 __global__ void __launch_bounds__(kThreads, 4)
     select_wave_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp, Geom gm, UnitTable ut,
-                       WaveOrder order, SelectArgs a, int n_stages,
+                       WaveOrder order, SelectArgs a, int n_stages, int keep_in_l2,
                        int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt, int32_t* __restrict__ status,
                        uint32_t* __restrict__ keys_g) {
     constexpr int RB = DP * Elem<T>::kBytes;          // bytes per projected-key row: 32, 64 or 128
@@ -515,7 +515,7 @@ __global__ void __launch_bounds__(kThreads, 4)
     uint32_t* keys_unit = keys_g + cu * (size_t)((gm.max_seq_len + 255) & ~255); // by candidate index, 16-byte aligned
     // The projected keys stream through L2 once; the score keys parked there must still be there when
     // the block comes back for them.
-    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = l2_policy_evict_last();
+    const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = keep_in_l2 ? l2_policy_evict_last() : stream_policy;
     // The sample row and the query are requested before the ring's first tiles: behind the whole
     // grid's opening burst of bulk copies they would wait for microseconds.
     const bool sampled = ncand >= kMinSampled;
@@ -643,6 +643,13 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
     if (n_stages > kStagesMax) n_stages = kStagesMax;
     if (n_stages < 2) n_stages = 2;
     const size_t smem = fixed + (size_t)n_stages * tile_bytes;
+    // 4 bytes of key per candidate: ask L2 to keep them only while a launch's worth fits comfortably
+    double parked = 0;
+    for (int i = 0; i < n_pairs; ++i) parked += 4.0 * cand[i] * gm.Hl;
+#ifndef TB_KEEP_BYTES
+#define TB_KEEP_BYTES 96e6
+#endif
+    const int keep_in_l2 = parked <= TB_KEEP_BYTES;
 
 #define TB_SEL_R(T, DP, RED)                                                                                                   \
     do {                                                                                                                \
@@ -652,7 +659,7 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
                                                  226 * 1024);                                                            \
             if (e != cudaSuccess) return e;                                                                             \
         }                                                                                                               \
-        select_wave_kernel<T, DP, RED><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, c->st.idx, c->st.cnt, \
+        select_wave_kernel<T, DP, RED><<<n_units, kThreads, smem, s>>>(c->kimp_map, (const unsigned char*)c->kimp, gm, ut, order, a, n_stages, keep_in_l2, c->st.idx, c->st.cnt, \
                                                                   c->st.status, c->wk.sel_keys);                        \
         return cudaGetLastError();                                                                                      \
     } while (0)

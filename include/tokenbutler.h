@@ -204,11 +204,14 @@ tb_status tb_sparse_decode_attention(tb_ctx* ctx, int32_t layer_begin, int32_t l
  *   seq_slots  (host, NULL = 0..n_seq-1) cache slot of each listed sequence; seq_lens (host) tokens cached
  *   q_dev      [n_seq][Hq][D] kv_dtype;  out_dev [n_seq][Hq][D] fp32;  lse_dev optional [n_seq][Hq]
  *   idx_dev / cnt_dev  caller lists [n_seq][Hkv][idx_stride] / [n_seq][Hkv] (ascending positions inside the
- *              candidate range), or both NULL for dense attention; entries outside [0, len) are skipped
+ *              candidate range), or both NULL for dense attention; entries outside [0, len) are skipped and
+ *              recorded as TB_ERR_BAD_INDEX in a status word inside the same array, which tb_static_get_status
+ *              returns and clears
  *   sinks, recent, sm_scale  as in tb_sparse_decode_attention
  *
  * Limits: n_seq * Hq <= TB_STATIC_MAX_QHEADS and n_seq <= 64, otherwise TB_ERR_CAPACITY and nothing is
- * launched.  The first call on each device looks up the array's device address (that device must be
+ * launched.  kv_dev must be memory of the current device (or page-locked host memory the device can
+ * address), else TB_ERR_INVALID_ARG.  The first call on each device looks up the array's device address (that device must be
  * current) and configures the kernel; make that first call outside any stream capture.  All calls in
  * the process share the one array: the counters are cleared on `stream` at the start of every call, and
  * two calls whose kernels overlap on the GPU (different streams, no ordering) race on the partials. */
@@ -219,6 +222,9 @@ tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32_t kv_dtype
                                             const int32_t* idx_dev, const int32_t* cnt_dev, int32_t idx_stride,
                                             int32_t sinks, int32_t recent, float sm_scale, float* out_dev,
                                             float* lse_dev, void* stream);
+/* Synchronise `stream` and return, then clear, the status word of the allocation-free entry point on
+ * the current device (TB_OK or TB_ERR_BAD_INDEX).  Allocates nothing. */
+tb_status tb_static_get_status(void* stream, int32_t* device_status);
 
 /* Importance-query predictor forward (paper Sec. 3.1 "Query prediction"; App. A: a two-layer MLP with
  * hidden size 512 at every producer layer; Table 6's parameter counts fix bias-free linears and a layer

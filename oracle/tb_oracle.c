@@ -19,6 +19,7 @@
  *   orc_neighbors      neighbour fetching                   Sec. 3.4 "Neighbor fetching"
  *   orc_attended_set   Sink | Important | Local-Window      Sec. 3.3 (three buffers)
  *   orc_attention      softmax(q K^T / sqrt(D)) V           Sec. 3.3 ("standard attention kernel")
+ *   orc_is_prediction_step  which decode steps re-select    Sec. 3.4 "Prediction interval"
  *   orc_step_units     the steps above chained per unit     Sec. 3.3 / 3.4
  *   orc_predict_queries  Q_imp = f(LN(H)), two-layer MLP    Sec. 3.1 "Query prediction", App. A (hidden
  *                                                           size 512), Table 6 (bias-free linears, LN
@@ -297,6 +298,16 @@ typedef struct {
     int32_t budget, sinks, recent, radius, nmode, reduce;
     double score_scale, sm_scale;
 } orc_params;
+
+/* Sec. 3.4 "Prediction interval": with interval P the prediction pipeline (scores, top-B, neighbours)
+ * runs once every P decode steps and the P-1 steps in between reuse the stored selection; the local
+ * window moves every step regardless.  Steps are counted from the first sparse decode step, which
+ * predicts (there is no selection to reuse yet): step t predicts iff t is a multiple of P.  Over T
+ * steps that is ceil(T / P) predictions -- the paper's "T to about T/N". */
+int orc_is_prediction_step(int step, int interval) {
+    if (interval < 1 || step < 0) return -1;
+    return step % interval == 0 ? 1 : 0;
+}
 
 void orc_step_units(orc_unit* units, int n_units, const orc_params* p, int n_threads) {
 #ifdef _OPENMP

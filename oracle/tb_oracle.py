@@ -163,6 +163,13 @@ def dense_attention(q, K, V, dtype, sm_scale=None):
     return attention(q, K, V, np.arange(K.shape[0], dtype=np.int32), dtype, sm_scale)
 
 
+def is_prediction_step(step: int, interval: int) -> bool:
+    """Sec. 3.4 prediction interval: does decode step `step` (0 = first sparse step) re-select?"""
+    v = lib().orc_is_prediction_step(C.c_int(step), C.c_int(interval))
+    assert v >= 0, "step >= 0 and interval >= 1"
+    return bool(v)
+
+
 class Unit:
     """One (sequence, layer, KV head): its caches and the stale selection (Sec. 3.4 interval)."""
 

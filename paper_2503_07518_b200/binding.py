@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libtokenbutler.so")
 
 EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb_set_projection", "tb_reset_sequence",
            "tb_get_length", "tb_append_kv", "tb_project_keys", "tb_score_tokens", "tb_select_topk",
-           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_predict_importance_queries", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
+           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
 
 
 class tb_config(C.Structure):
@@ -80,6 +80,7 @@ def lib():
                                                  vp, vp, vp]
         L.tb_sparse_decode_attention_static.argtypes = [vp, i32, i32, i32, i32, i32, ip, ip, i32, vp, vp, vp, i32, i32, i32,
                                                         C.c_float, vp, vp, vp]
+        L.tb_static_get_status.argtypes = [vp, ip]
         L.tb_predict_importance_queries.argtypes = [vp, vp, i32, vp, vp, vp]
         L.tb_get_status.argtypes = [vp, vp, ip]
         L.tb_last_step_bytes.argtypes = [vp]
@@ -125,6 +126,15 @@ def sparse_decode_attention_static(kv, kv_dtype, n_q_heads, n_kv_heads, head_dim
                                                    _ints(seq_slots), _ints(seq_lens), len(seq_lens), _ptr(q), _ptr(idx),
                                                    _ptr(cnt), idx_stride, sinks, recent, sm_scale, _ptr(out), _ptr(lse),
                                                    _stream(stream))
+
+
+def static_get_status(stream=None):
+    """Status word of the allocation-free entry point on the current device (read and cleared)."""
+    v = C.c_int32()
+    st = lib().tb_static_get_status(_stream(stream), C.byref(v))
+    if st != TB_OK:
+        raise TBError(st, "tb_static_get_status")
+    return v.value
 
 
 def predict_importance_queries(hidden, ln_weight, ln_bias, w1, w2, dtype, n_q_heads, n_slots, imp_dim, scratch, q_imp,

@@ -880,6 +880,18 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     int sm_count = 0;
     tb_status st = static_scratch_for_current_device(&scratch, &sm_count);
     if (st != TB_OK) return st;
+    {
+        // The scratch address belongs to the current device; a cache that lives on another GPU would be
+        // read by kernels launched here.  (Page-locked host memory has no owning device and is accepted.)
+        cudaPointerAttributes pa;
+        int dev = -1;
+        if (cudaPointerGetAttributes(&pa, kv_dev) != cudaSuccess || cudaGetDevice(&dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return TB_ERR_INVALID_ARG;
+        }
+        if ((pa.type == cudaMemoryTypeDevice || pa.type == cudaMemoryTypeManaged) && pa.device != dev) return TB_ERR_INVALID_ARG;
+        if (pa.type == cudaMemoryTypeUnregistered) return TB_ERR_INVALID_ARG;
+    }
     float* part_o = reinterpret_cast<float*>(scratch);
     float* part_ml = reinterpret_cast<float*>(scratch + kStaticPartO);
     uint32_t* counters = reinterpret_cast<uint32_t*>(scratch + kStaticPartO + kStaticPartMl);
@@ -912,7 +924,8 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     a.early_ok = 0;
     for (int i = 0; i < n_seq; ++i) a.known_cnt[i] = -1;
     a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)head_dim);
-    {   // same split rule as the context path
+    {   // about four 4-warp blocks per SM, at least 64 rows per split; no clusters here: the splits
+        // always merge through the scratch array (last block to arrive, fixed order)
         int units = n_seq * n_kv_heads, target = 4 * sm_count;
         int n = (target + units - 1) / units, by_rows = max_rows / 64;
         if (n > by_rows) n = by_rows;
@@ -921,8 +934,9 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
         a.nsplit = n;
     }
     cudaStream_t s = (cudaStream_t)stream;
-    // the array keeps whatever the previous call left: the arrival counters and the status word must start at zero
-    if (cudaMemsetAsync(counters, 0, kStaticCounters + kStaticStatus, s) != cudaSuccess) return TB_ERR_CUDA;
+    // the array keeps whatever the previous call left: the arrival counters must start at zero.  The status
+    // word is left alone: it collects errors until tb_static_get_status reads and clears it.
+    if (cudaMemsetAsync(counters, 0, kStaticCounters, s) != cudaSuccess) return TB_ERR_CUDA;
     dim3 grid(a.nsplit, n_kv_heads, n_seq);
     // the stored-list arguments of the kernels are never read here (caller lists or dense)
     if (kv_dtype == TB_BF16) {
@@ -936,3 +950,18 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     return cudaGetLastError() == cudaSuccess ? TB_OK : TB_ERR_CUDA;
 }
 
+extern "C" tb_status tb_static_get_status(void* stream, int32_t* device_status) {
+    if (!device_status) return TB_ERR_INVALID_ARG;
+    unsigned char* scratch = nullptr;
+    int sm_count = 0;
+    tb_status st = static_scratch_for_current_device(&scratch, &sm_count);
+    if (st != TB_OK) return st;
+    int32_t* status = reinterpret_cast<int32_t*>(scratch + kStaticPartO + kStaticPartMl + kStaticCounters);
+    int32_t v = 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&v, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return TB_ERR_CUDA;
+    if (cudaMemsetAsync(status, 0, 4, s) != cudaSuccess) return TB_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return TB_ERR_CUDA;
+    *device_status = v;
+    return TB_OK;
+}

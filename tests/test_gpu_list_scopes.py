@@ -36,7 +36,8 @@ def test_scope_pipeline_matches_oracle(H, scope, ci):
     p = b_.select_params(w.budget, w.sinks, w.recent)
     full_pipeline_check(H, case, p, dense_too=True)
     pn = b_.select_params(w.budget, w.sinks, w.recent, radius=2, nmode=b_.TB_NEIGHBOR_DILATE)
-    full_pipeline_check(H, case, pn, step=1)
+    full_pipeline_check(H, case, b_.select_params(w.budget, w.sinks, w.recent, radius=1, nmode=b_.TB_NEIGHBOR_CLUSTER), step=3)
+    full_pipeline_check(H, case, pn, step=1)                               # leaves the DILATE lists stored for the reuse step below
     # a decode step that appends and reuses the stored lists (interval 4, step 1)
     case.append_step(0)
     case.project_range(list(case.proj), list(case.cur))

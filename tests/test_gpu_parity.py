@@ -33,22 +33,29 @@ def full_pipeline_check(H, case, p, step=0, dense_too=False):
     w = case.w
     q, qi = H.queries(w, step)
     qi = qi[:, :, :case.Hl * case.gl]                     # one list per layer: a single importance query
+    base_lists = None
+    if p.radius > 0:
+        # The GPU's own pre-expansion selection: the same launch with radius 0 (selection is bit-reproducible).
+        # It is held to the oracle's with the near-tie rule; the expanded list must then be EXACTLY the
+        # oracle's neighbour rule applied to it.  Taken first, so the lists left in the context are the expanded ones.
+        assert p.step % p.interval == 0
+        p0 = tb().select_params(p.budget, p.sinks, p.recent, 0, p.nmode, p.interval, p.step, p.reduce, p.score_scale)
+        base_lists = H.gpu_select(case, qi, p0)
     lists = H.gpu_select(case, qi, p)
     assert case.ctx.get_status() == 0
     swaps = 0
     for l in range(w.n_layers):
         for b in range(w.batch):
             for h in range(case.Hl):
+                what = "layer %d seq %d list %d" % (l, b, h)
                 base, full, s = case.oracle_select(l, b, h, qi[l, b], p)
                 if p.radius == 0:
-                    swaps += H.check_selection(lists[l][b][h], full, s, "layer %d seq %d list %d" % (l, b, h))
+                    swaps += H.check_selection(lists[l][b][h], full, s, what)
                 else:
-                    # neighbour lists follow from the base selection; compare exactly when the base sets agree
-                    if np.array_equal(lists[l][b][h], full):
-                        continue
+                    swaps += H.check_selection(base_lists[l][b][h], base, s, what)
                     lo, hi = H.orc.candidate_range(case.cur[b], p.sinks, p.recent)
-                    assert np.all((lists[l][b][h] >= lo) & (lists[l][b][h] < hi))
-                    swaps += 1
+                    want = H.orc.neighbors(base_lists[l][b][h], p.radius, p.nmode, lo, hi)
+                    assert np.array_equal(lists[l][b][h], want), "%s: expanded list is not the neighbour rule of the GPU's selection" % what
     out, lse = H.gpu_attention(case, q, p)
     assert case.ctx.get_status() == 0
     worst = 0.0

@@ -275,7 +275,8 @@ def test_interval_reuses_stale_list_and_window_slides(orc):
     prev = None
     for t in range(steps):
         L = L0 + t
-        refresh = int(t % P == 0)
+        refresh = int(orc.is_prediction_step(t, P))
+        assert refresh == int(t in (0, 4, 8))
         qi = [r.standard_normal((g, dp)).astype(np.float32) for _ in units]
         qs = [rand_storage(r, (g, D), BF16) for _ in units]
         out = orc.step_units(units, [L] * 2, qi, qs, [refresh] * 2, g=g, D=D, dp=dp, dtype=BF16, budget=Bud, sinks=S,
@@ -300,18 +301,32 @@ def test_interval_reuses_stale_list_and_window_slides(orc):
 
 
 def test_interval_one_is_per_step_selection(orc):
+    # P = 1: every step predicts, and each step's stored list is the plain definition (numpy float64
+    # scores, lexsort) at that step's length and with that step's importance query -- not a stale one
     r = rng(17)
-    L, D, dp, g = 128, 128, 16, 1
-    ua = make_units(orc, rng(18), 1, L, L + 3, D, dp, F32, 10)
-    ub = make_units(orc, rng(18), 1, L, L + 3, D, dp, F32, 10)
+    L0, D, dp, g, S, Wn, Bud = 128, 128, 16, 2, 2, 4, 10
+    units = make_units(orc, rng(18), 1, L0, L0 + 3, D, dp, F32, Bud)
     for t in range(3):
+        assert orc.is_prediction_step(t, 1)
+        L = L0 + t
         qi = [r.standard_normal((g, dp)).astype(np.float32)]
         qs = [rand_storage(r, (g, D), F32)]
-        kw = dict(g=g, D=D, dp=dp, dtype=F32, budget=10, sinks=2, recent=4)
-        oa = orc.step_units(ua, [L + t], qi, qs, [1], **kw)              # P = 1: refresh every step
-        ub[0].cnt[0] = 0
-        ob = orc.step_units(ub, [L + t], qi, qs, [1], **kw)
-        assert np.array_equal(oa, ob)
+        orc.step_units(units, [L], qi, qs, [int(orc.is_prediction_step(t, 1))], g=g, D=D, dp=dp, dtype=F32, budget=Bud, sinks=S,
+                       recent=Wn)
+        s = f64(units[0].Kimp[:L], F32) @ qi[0].astype(np.float64).sum(0)
+        assert np.array_equal(units[0].idx[:units[0].cnt[0]], lexsort_select(s, S, Wn, Bud))
+
+
+def test_prediction_steps_are_the_multiples_of_the_interval(orc):
+    # Sec. 3.4: the pipeline runs once every N steps, starting with the first sparse step (nothing to
+    # reuse before it); T steps cost ceil(T / N) predictions ("T to about T/N"), 16 at N = 16 over 256 steps
+    for P in (1, 2, 4, 16):
+        steps = [t for t in range(256) if orc.is_prediction_step(t, P)]
+        assert steps == list(range(0, 256, P)) and len(steps) == -(-256 // P)
+        gaps = np.diff(steps)
+        assert len(gaps) == 0 or np.all(gaps == P)                   # exactly P - 1 reuse steps between two predictions
+    assert sum(orc.is_prediction_step(t, 16) for t in range(256)) == 16
+    assert sum(orc.is_prediction_step(t, 4) for t in range(9)) == 3  # steps 0, 4, 8
 
 
 # ------------------------------------------------------------------ values the paper prints

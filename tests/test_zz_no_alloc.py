@@ -63,12 +63,53 @@ def test_static_entry_matches_context_entry_twice(H, cfg):
         assert st == tb.TB_OK
         torch.cuda.synchronize()
         assert (out - dense_ref).abs().max().item() <= tol
-        # and against the oracle, on the GPU's own list
-        o = out.cpu().numpy()
+        # the sparse result against the oracle on the caller's lists, every sequence and KV head; one dense unit
+        sparse = torch.full_like(ref, float("nan"))
+        st = tb.sparse_decode_attention_static(case.ctx.kv[layer], w.dtype, w.n_q_heads, w.n_kv_heads, w.head_dim, case.cap,
+                                               None, case.cur, q_dev, sparse, idx=idx, cnt=cnt, idx_stride=cap, sinks=w.sinks,
+                                               recent=w.recent)
+        assert st == tb.TB_OK
+        torch.cuda.synchronize()
+        sp, o = sparse.cpu().numpy(), out.cpu().numpy()
         got_idx, got_cnt = idx.cpu().numpy(), cnt.cpu().numpy()
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                refo, _ = case.oracle_attention(layer, b, h, q[layer, b], got_idx[0, b, h, :got_cnt[0, b, h]], p)
+                assert np.abs(sp[b, h * w.group:(h + 1) * w.group] - refo).max() <= tol
         refo, _ = case.oracle_attention(layer, 1, 0, q[layer, 1], None, p, dense=True)
         assert np.abs(o[1, :w.group] - refo).max() <= tol
+        assert tb.static_get_status() == 0
     assert case.ctx.get_status() == 0
+
+
+def test_static_entry_reports_an_out_of_range_list_entry(H):
+    """A caller list entry equal to the sequence length is skipped (no access outside the cache) and
+    shows up once in the entry point's own status word; the rest of the list is attended as usual."""
+    from paper_2503_07518_b200 import binding as tb
+    w = wl.workload(2, n_layers=1, n_q_heads=8, n_kv_heads=2, lengths=[600], budget=32)
+    case = H.Case(w, project="oracle-only")
+    q, _ = H.queries(w)
+    r = np.random.Generator(np.random.PCG64(6))
+    mine = [np.sort(r.choice(np.arange(5, 590), 20, replace=False)).astype(np.int32) for _ in range(2)]
+    idx = np.zeros((1, 2, 24), np.int32)
+    for h in range(2):
+        idx[0, h, :20] = mine[h]
+    idx[0, 1, 7] = 600                                                    # one past the end
+    cnt = np.full((1, 2), 20, np.int32)
+    q_dev = H.to_dev(q[0], w.dtype)
+    out = torch.full((1, w.n_q_heads, w.head_dim), float("nan"), device="cuda")
+    assert tb.static_get_status() == 0
+    st = tb.sparse_decode_attention_static(case.ctx.kv[0], w.dtype, w.n_q_heads, w.n_kv_heads, w.head_dim, case.cap, None,
+                                           case.cur, q_dev, out, idx=torch.from_numpy(idx).cuda(), cnt=torch.from_numpy(cnt).cuda(),
+                                           idx_stride=24, sinks=5, recent=10)
+    assert st == tb.TB_OK
+    assert tb.static_get_status() == tb.TB_ERR_BAD_INDEX
+    assert tb.static_get_status() == 0                                    # reading clears it
+    p = tb.select_params(32, 5, 10)
+    o = out.cpu().numpy()
+    for h, lst in enumerate([mine[0], np.delete(mine[1], 7)]):
+        refo, _ = case.oracle_attention(0, 0, h, q[0, 0], lst, p)
+        assert np.abs(o[0, h * 4:(h + 1) * 4] - refo).max() <= 2e-3
 
 
 def test_static_entry_rejects_what_its_scratch_cannot_hold(H):
@@ -84,3 +125,7 @@ def test_static_entry_rejects_what_its_scratch_cannot_hold(H):
     assert st == tb.TB_ERR_INVALID_ARG
     st = tb.sparse_decode_attention_static(kv, tb.TB_BF16, 32, 8, 96, 64, None, [64], q, out)
     assert st == tb.TB_ERR_UNSUPPORTED
+    # a cache the device cannot address (pageable host memory) is refused, not handed to a kernel
+    st = tb.sparse_decode_attention_static(torch.zeros(8 * 64 * 2 * 128, dtype=torch.bfloat16), tb.TB_BF16, 32, 8, 128, 64,
+                                           None, [64], q, out)
+    assert st == tb.TB_ERR_INVALID_ARG

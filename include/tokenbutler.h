@@ -16,8 +16,11 @@
  *     allocates the four regions sized by tb_query_sizes() (256-byte aligned) and binds them with
  *     tb_create().  `stream` is a cudaStream_t passed as void*; all work is enqueued on it and the
  *     call returns without synchronising (tb_get_status is the one exception).
- *   - Errors are return codes only.  A call that returns anything but TB_OK has changed no state and
- *     launched nothing.  Problems only the device can see (an out-of-range entry in a caller-supplied
+ *   - Errors are return codes only.  Every error but TB_ERR_CUDA is found on the host before the call's
+ *     first launch (for all of the call's layers): such a call has changed no state and launched nothing.
+ *     TB_ERR_CUDA means that the CUDA runtime refused a launch or a copy in mid-call: earlier launches of
+ *     that call may have run, and the sequences it named must be reset (tb_reset_sequence) before they
+ *     are used again.  Problems only the device can see (an out-of-range entry in a caller-supplied
  *     index list, an internal wait that ran out) set a device status word, skip the offending access
  *     and let the kernel finish; tb_get_status() reads and clears that word.
  *   - Shapes: B sequences, Hq query heads, Hkv KV heads, g = Hq/Hkv, D = head_dim (128),
@@ -260,6 +263,17 @@ tb_status tb_predict_importance_queries(const tb_predictor* p, const void* hidde
 /* Synchronise `stream`, return the device status word (TB_OK, TB_ERR_TIMEOUT or TB_ERR_BAD_INDEX)
  * in *device_status and clear it. */
 tb_status tb_get_status(tb_ctx* ctx, void* stream, int32_t* device_status);
+
+/* Diagnostics of the bounded device waits (every wait of a kernel on a copy it requested polls at most
+ * a fixed number of times -- seconds -- then the kernel records TB_ERR_TIMEOUT in the status word, stops
+ * requesting copies, finishes normally and leaves nothing in flight; the lists of that call are void).
+ * poll_limit > 0 sets the number of polls for this context's selection launches (0 restores the
+ * default).  drop_tile >= 0 makes the NEXT selection launch arm the barrier of its drop_tile-th tile of
+ * 256 rows without requesting the copy, so that this wait runs out: the way to exercise the path without
+ * a fault, a trap or an unbounded wait.  It is honoured only by a launch of one block (one sequence, one
+ * list, at most 1023 candidates: nothing else is in flight and no other block waits); any other selection
+ * call then returns TB_ERR_UNSUPPORTED and launches nothing.  One-shot; -1 = none. */
+tb_status tb_set_wait_diagnostics(tb_ctx* ctx, int32_t poll_limit, int32_t drop_tile);
 
 /* Algorithmic bytes (projected keys scanned + K/V rows gathered, upper bound from host-known sizes)
  * of the most recent select or attention call. */

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libtokenbutler.so")
 
 EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb_set_projection", "tb_reset_sequence",
            "tb_get_length", "tb_append_kv", "tb_project_keys", "tb_score_tokens", "tb_select_topk",
-           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
+           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_set_wait_diagnostics", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
 
 
 class tb_config(C.Structure):
@@ -83,6 +83,7 @@ def lib():
         L.tb_static_get_status.argtypes = [vp, ip]
         L.tb_predict_importance_queries.argtypes = [vp, vp, i32, vp, vp, vp]
         L.tb_get_status.argtypes = [vp, vp, ip]
+        L.tb_set_wait_diagnostics.argtypes = [vp, i32, i32]
         L.tb_last_step_bytes.argtypes = [vp]
         L.tb_launch_count.argtypes = [vp]
         L.tb_status_string.argtypes = [i32]
@@ -237,6 +238,9 @@ class Context:
         v = C.c_int32()
         self._chk(lib().tb_get_status(self.h, _stream(stream), C.byref(v)), "tb_get_status")
         return v.value
+
+    def set_wait_diagnostics(self, poll_limit=0, drop_tile=-1):
+        self._chk(lib().tb_set_wait_diagnostics(self.h, poll_limit, drop_tile), "tb_set_wait_diagnostics")
 
     def last_step_bytes(self):
         return lib().tb_last_step_bytes(self.h)

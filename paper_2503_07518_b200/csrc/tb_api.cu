@@ -214,6 +214,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     const size_t n = (size_t)cfg->n_layers * cfg->max_batch;
     c->len.assign(n, 0), c->len_proj.assign(n, 0), c->has_sel.assign(n, 0), c->sel_cnt.assign(n, -1);
     c->last_bytes = 0, c->launches = 0;
+    c->wait_poll_limit = 0, c->drop_tile = -1;
     c->last_cache_write = c->last_list_write = -4;
     c->tile_rows = 256;
     for (int i = 0; i < 17; ++i) c->attn_max_active[i] = 0;
@@ -377,37 +378,43 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                 if (!c->has_sel[(size_t)l * mb + seqs[i]]) return TB_ERR_STATE;
     }
     const int step = layers_per_launch(n_seq);
-    for (int l0 = lb; l0 < lb + lc; l0 += step) {
-        const int n = l0 + step <= lb + lc ? step : lb + lc - l0;
-        UnitTable ut;
-        fill_table(c, &ut, l0, n, seqs, n_seq);
-        const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->geom.Hl;
-        if (refresh) {
-            SelectArgs a;
-            a.q_imp = q_imp + (size_t)(l0 - lb) * n_seq * c->geom.Hl * c->geom.gl * c->cfg.imp_dim;
-            a.budget = p->budget, a.sinks = p->sinks, a.recent = p->recent, a.reduce = reduce;
-            if (p->radius == 0) {
-                a.idx_dst = nullptr, a.cnt_dst = nullptr, a.dst_is_state = 1, a.idx_stride = c->geom.idx_cap;
-            } else {
-                a.idx_dst = c->wk.sel_idx, a.cnt_dst = c->wk.sel_cnt, a.dst_is_state = 0, a.idx_stride = c->wk.sel_stride;
+    // Two passes over the call's chunks: the first only checks that every launch has a configuration
+    // (sizes beyond what a kernel takes are refused before anything runs), the second launches.
+    for (int pass = 0; pass < 2; ++pass) {
+        const bool dry = pass == 0;
+        if (dry && !refresh) continue;
+        for (int l0 = lb; l0 < lb + lc; l0 += step) {
+            const int n = l0 + step <= lb + lc ? step : lb + lc - l0;
+            UnitTable ut;
+            fill_table(c, &ut, l0, n, seqs, n_seq);
+            const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->geom.Hl;
+            if (refresh) {
+                SelectArgs a;
+                a.q_imp = q_imp + (size_t)(l0 - lb) * n_seq * c->geom.Hl * c->geom.gl * c->cfg.imp_dim;
+                a.budget = p->budget, a.sinks = p->sinks, a.recent = p->recent, a.reduce = reduce;
+                if (p->radius == 0) {
+                    a.idx_dst = nullptr, a.cnt_dst = nullptr, a.dst_is_state = 1, a.idx_stride = c->geom.idx_cap;
+                } else {
+                    a.idx_dst = c->wk.sel_idx, a.cnt_dst = c->wk.sel_cnt, a.dst_is_state = 0, a.idx_stride = c->wk.sel_stride;
+                }
+                cudaError_t e = launch_select(c, ut, a, (cudaStream_t)stream, dry);
+                if (e != cudaSuccess) return dry ? TB_ERR_UNSUPPORTED : TB_ERR_CUDA;
+                if (!dry) c->last_list_write = (long long)c->launches, c->launches++;
+                if (p->radius > 0) {
+                    NeighborArgs na;
+                    na.idx_src = c->wk.sel_idx, na.cnt_src = c->wk.sel_cnt, na.src_stride = c->wk.sel_stride;
+                    na.radius = p->radius, na.nmode = p->nmode, na.sinks = p->sinks, na.recent = p->recent;
+                    e = launch_neighbors(c, ut, na, (cudaStream_t)stream, dry);
+                    if (e != cudaSuccess) return dry ? TB_ERR_UNSUPPORTED : TB_ERR_CUDA;
+                    if (!dry) c->last_list_write = (long long)c->launches, c->launches++;
+                }
             }
-            if (launch_select(c, ut, a, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
-            c->last_list_write = (long long)c->launches;
-            c->launches++;
-            if (p->radius > 0) {
-                NeighborArgs na;
-                na.idx_src = c->wk.sel_idx, na.cnt_src = c->wk.sel_cnt, na.src_stride = c->wk.sel_stride;
-                na.radius = p->radius, na.nmode = p->nmode, na.sinks = p->sinks, na.recent = p->recent;
-                if (launch_neighbors(c, ut, na, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
-                c->last_list_write = (long long)c->launches;
+            if (!dry && (idx_out || cnt_out)) {
+                if (launch_copy_lists(c, ut, idx_out ? idx_out + unit_off * c->geom.idx_cap : nullptr,
+                                      cnt_out ? cnt_out + unit_off : nullptr, (cudaStream_t)stream) != cudaSuccess)
+                    return TB_ERR_CUDA;
                 c->launches++;
             }
-        }
-        if (idx_out || cnt_out) {
-            if (launch_copy_lists(c, ut, idx_out ? idx_out + unit_off * c->geom.idx_cap : nullptr,
-                                  cnt_out ? cnt_out + unit_off : nullptr, (cudaStream_t)stream) != cudaSuccess)
-                return TB_ERR_CUDA;
-            c->launches++;
         }
     }
     if (refresh) {
@@ -492,6 +499,13 @@ tb_status tb_get_status(tb_ctx* c, void* stream, int32_t* device_status) {
     if (cudaMemsetAsync(c->st.status, 0, 4, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     *device_status = v;
+    return TB_OK;
+}
+
+tb_status tb_set_wait_diagnostics(tb_ctx* c, int32_t poll_limit, int32_t drop_tile) {
+    if (!c || poll_limit < 0) return TB_ERR_INVALID_ARG;
+    c->wait_poll_limit = poll_limit;
+    c->drop_tile = drop_tile < 0 ? -1 : drop_tile;
     return TB_OK;
 }
 

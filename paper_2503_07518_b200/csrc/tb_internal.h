@@ -106,6 +106,8 @@ struct tb_ctx {
     int tile_rows;                        // rows per TMA box of the score pass
     int sm_count;
     int attn_max_active[17];              // co-resident attention clusters per cluster size (0 = not asked yet)
+    int wait_poll_limit;                  // polls per bounded wait of the selection kernels; 0 = the default (seconds)
+    int drop_tile;                        // diagnostics: tile whose copy the next single-block selection leaves out, -1 = none
     uint64_t last_bytes, launches;
     // index (value of `launches` at launch time) of the last kernel that wrote the caches / the stored
     // lists; a kernel may read them before its dependency wait only if that writer is not its predecessor
@@ -132,12 +134,14 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
 // tb_select.cu
 cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, int reduce, float scale, float* scores,
                          cudaStream_t s);
-cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
+// `dry`: work out the launch configuration and report whether it exists, launch nothing, change nothing
+// (the entry points check every chunk of a call this way before the first real launch)
+cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry = false);
 // one block per problem; launch_select hands over to it when a launch holds at least two problems per SM
-cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
+cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry = false);
 // few, long problems: a cluster per problem on parked keys
-cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s);
-cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s);
+cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry = false);
+cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s, bool dry = false);
 cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s);
 
 // tb_attention.cu

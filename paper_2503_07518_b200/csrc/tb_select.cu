@@ -4,17 +4,25 @@
 // One thread-block cluster (1..8 blocks) per (layer, sequence, KV head).  Each block streams its share
 // of the candidate rows of the projected-key cache through shared memory with 2-D TMA tiles, scores
 // every row, and keeps the scores on chip as order-preserving 32-bit keys (scores never go to HBM).
-// The exact top-B is a radix select on those keys:
-//   digit 1 (top 11 bits)  histogrammed while streaming; the blocks publish their non-empty bins to
-//                          each other through distributed shared memory, one cluster barrier, and
-//                          every block finds the threshold bin itself;
-//   digits 2, 3            only the keys of the threshold bin matter (a few per cent): they are
-//                          gathered at rank 0, which finishes alone and hands every rank the
-//                          threshold and its output offsets;
-//   compaction             ordered (warp ballots), ties taken in position order, ascending list
-//                          written straight to its destination.
-// Unusual inputs (more non-empty bins than a list holds, a crowded threshold bin) and single-block
-// launches take the general path: every digit through cluster-merged histograms.
+// The exact top-B is a radix select on those keys whose first digit is placed by a look at the data:
+//   sample      every block of the cluster scores the same 64 rows spread over the problem and
+//               brackets, generously, where the B-th largest score will fall.  The first digit has
+//               1024 bins: 1022 equal slices of key space across the bracket, one open bin below, one
+//               above.  It is monotone in the key whatever the sample says, so the result never
+//               depends on the sample; only how few keys share the threshold's bin does (a handful).
+//   stream      score, key, first-digit histogram.
+//   exchange    every block sends its histogram (16-bit counts) to every peer through distributed shared
+//               memory, one cluster barrier; every block then finds the threshold bin and every rank's
+//               counts above and inside it from its own copy -- no remote read, no serial section.
+//   candidates  one pass over the block's keys turns "above the threshold bin" into a bitmask and sends
+//               the few keys inside the bin, with their positions, to every peer; second barrier; every
+//               block ranks that short list itself (equal keys by position), sets its winners' bits and
+//               writes its part of the ascending list.
+// A distributed-memory round trip costs 0.3-0.7 us on this part and a cluster barrier 0.2 us, so the
+// finish is built from two one-way exchanges instead of request/response steps.
+// Unusual inputs (a crowded threshold bin: massive ties, a threshold outside the bracket) and problems
+// too small to sample take the general path: the key's own digits (11 + 11 + 10 bits) through
+// cluster-merged histograms, then an ordered compaction.
 #include <cooperative_groups.h>
 
 #include <cstddef>
@@ -29,17 +37,19 @@ constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kTileRows = 256;      // rows per TMA box = one row per thread
 constexpr int kMaxStages = 12;      // depth of the TMA ring is chosen per launch (bytes in flight vs. blocks per SM)
-constexpr int kBins = 2048;         // 11-bit digits (the last digit has 10 bits)
+constexpr int kBins = 2048;         // 11-bit digits of the general path (the last digit has 10 bits)
 constexpr int kMaxCluster = 8;
-constexpr int kMaxKeysPerBlock = 32768;   // 128 KB of on-chip keys per block at most
-constexpr int kListCap = 256;       // non-empty first-digit bins a block may publish on the fast path
+constexpr int kMaxKeysPerBlock = 32768;   // 128 KB of on-chip keys per block at most (and 16-bit histogram counts)
+constexpr int kFastBins = 1024;     // bins of the sampled first digit
+constexpr int kFastCand = 256;      // keys of the threshold bin that every block ranks itself
+constexpr int kSampleRows = 64;     // rows scored up front to place the first digit's bins
+constexpr int kMinSampled = 2048;   // smaller problems use the key's top bits as first digit
 #ifndef TB_CW_FROM
 #define TB_CW_FROM (48 * 1024)
 #endif
 constexpr int kCwFrom = TB_CW_FROM;   // candidates from which the parked-key cluster kernel takes over (macro: tuning builds)
 constexpr int kCwLimit = 8 * 262144; // ... and up to which it can (8 blocks x 32 KB of bitmask; the rows' first digits move to the workspace when
                                      // they no longer fit on chip)
-constexpr int kCandCap = 4096;      // keys of the threshold bin gathered at rank 0 (aliases merged[1..2])
 
 // Optional per-phase timestamps of the first and last block of unit 0, for tuning builds only
 // (-DTB_PHASE_TIMING); the product build compiles these away.
@@ -55,31 +65,50 @@ __device__ __forceinline__ void phase_stamp(int i) {
 extern "C" int tb_debug_phase_ns(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, g_phase_ns, sizeof(g_phase_ns));
 }
+__device__ unsigned int g_sel_fallbacks[2];
+extern "C" int tb_debug_sel_fallbacks(unsigned int* out) { return (int)cudaMemcpyFromSymbol(out, g_sel_fallbacks, sizeof(g_sel_fallbacks)); }
+__device__ __forceinline__ void phase_value(int i, unsigned long long v) {
+    if (threadIdx.x == 0 && blockIdx.y == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) g_phase_ns[blockIdx.x == 0 ? 0 : 1][i] = v;
+}
 #else
 __device__ __forceinline__ void phase_stamp(int) {}
+__device__ __forceinline__ void phase_value(int, unsigned long long) {}
 #endif
 
 struct __align__(16) SelSmem {
-    int res[8];                         // rank 0's verdict: prefix, low_bits, krem, gt_base, eq_base (16-byte stores)
+    uint32_t peer_hi[kBins];            // directly behind `merged`: together the peers' 16-bit histograms, [8][1024]
+    uint32_t sample[kSampleRows];       // read with 16-byte loads
     uint64_t full[kMaxStages];
     int warp_a[kSelWarps];
     int warp_b[kSelWarps];
     int tot[kMaxCluster][2];
-    int bc_bin, bc_krem, bc_count, pad0;
-    int list_len[kMaxCluster];          // per rank: entries in lists[rank]
-    int above[kMaxCluster];             // per rank: keys in bins above the threshold bin
+    int bc_bin, bc_krem, bc_count, n_cand;
+    uint32_t s_lo, s_hi;                // sample keys bracketing the expected threshold
+    int pad1[2];
     int inbin[kMaxCluster];             // per rank: keys in the threshold bin
-    uint32_t lists[kMaxCluster][kListCap];   // (bin << 16 | count) of every rank's non-empty bins
+    int winners[kMaxCluster];           // per rank: keys of the threshold bin that made it
     alignas(16) float qs[kMaxGroup * 32];           // TB_GROUP_MAX: the group's importance queries
 };
 
-static_assert(offsetof(SelSmem, qs) % 16 == 0, "qs is read with 16-byte loads");
+static_assert(offsetof(SelSmem, peer_hi) == 0, "the peers' histograms continue from `merged` into peer_hi");
+static_assert(offsetof(SelSmem, qs) % 16 == 0 && offsetof(SelSmem, sample) % 16 == 0, "read with 16-byte loads");
+static_assert(kMaxCluster * kFastBins * 2 <= 2 * kBins * 4, "peers' histograms fit merged + peer_hi");
 
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ void smem_add(int* p, int v) {
     asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
 }
+
+// First digit of the fast path: 1024 bins, monotone in the key.  Bin 0 = below `base`, bins 1..1022 =
+// equal slices of 2^shift keys from `base` up, bin 1023 = everything above.
+struct SampledDigit {
+    uint32_t base;
+    int shift;
+    __device__ __forceinline__ int bin(uint32_t key) const {
+        return key < base ? 0 : (int)min((key - base) >> shift, (uint32_t)(kFastBins - 2)) + 1;
+    }
+};
 
 // PER consecutive counters of thread `tid` (16-byte loads, at most 2-way bank conflicts).
 template <int PER>
@@ -110,15 +139,14 @@ __device__ __forceinline__ int block_excl_scan(int v, int* slots, int& total) {
     return before + incl - v;
 }
 
-// Finds, over PER*256 counters ordered by digit value, the digit b with
-//   count(digits > b) < k <= count(digits >= b)
-// and returns it with k' = k - count(digits > b) and the population of b.  All threads call it and
+// Finds, over PER*256 counters ordered by digit value (thread `tid` holds counters tid*PER .. +PER-1 in
+// `b`), the digit d with
+//   count(digits > d) < k <= count(digits >= d)
+// and returns it with k' = k - count(digits > d) and the population of d.  All threads call it and
 // all receive the same answer.  Preconditions: 1 <= k <= total count.
 template <int PER>
-__device__ __forceinline__ void find_digit(const int* hist, int k, SelSmem* sm, int& bin, int& krem, int& bcount) {
+__device__ __forceinline__ void find_digit_regs(const int (&b)[PER], int k, SelSmem* sm, int& bin, int& krem, int& bcount) {
     const int tid = threadIdx.x;
-    int b[PER];
-    load_bins<PER>(hist, tid, b);
     int mine = 0;
 #pragma unroll
     for (int i = 0; i < PER; ++i) mine += b[i];
@@ -141,10 +169,17 @@ __device__ __forceinline__ void find_digit(const int* hist, int k, SelSmem* sm, 
     bin = sm->bc_bin, krem = sm->bc_krem, bcount = sm->bc_count;
     __syncthreads();                                  // bc_* and warp_a may be reused right away
 }
+template <int PER>
+__device__ __forceinline__ void find_digit(const int* hist, int k, SelSmem* sm, int& bin, int& krem, int& bcount) {
+    int b[PER];
+    load_bins<PER>(hist, threadIdx.x, b);
+    find_digit_regs<PER>(b, k, sm, bin, krem, bcount);
+}
 
 template <typename T, int DP, int RED>
-__global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_constant__ CUtensorMap tmap, Geom gm, UnitTable ut,
-                                                             SelectArgs a, int tiles_per_cta, int n_stages,
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_constant__ CUtensorMap tmap, const unsigned char* __restrict__ kimp,
+                                                             Geom gm, UnitTable ut, SelectArgs a, int tiles_per_cta, int n_stages,
+                                                             uint32_t wait_limit, int drop_tile,
                                                              int32_t* __restrict__ state_idx, int32_t* __restrict__ state_cnt,
                                                              int32_t* __restrict__ status) {
     constexpr int RB = DP * Elem<T>::kBytes;          // bytes per projected-key row: 32, 64 or 128
@@ -155,13 +190,18 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     // swizzled TMA boxes need their shared-memory base on the swizzle period (up to 1024 bytes)
     unsigned char* stage_base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // n_stages * kTileBytes
     int* hist = reinterpret_cast<int*>(stage_base + n_stages * kTileBytes);       // local histogram
-    int* merged = hist + kBins;                                                   // cluster-merged first-digit histogram
+    int* merged = hist + kBins;                                                   // general path: cluster-merged first-digit histogram
     SelSmem* sm = reinterpret_cast<SelSmem*>(merged + kBins);
     uint32_t* keys = reinterpret_cast<uint32_t*>(sm + 1);                         // tiles_per_cta * kTileRows
-    // The ring is idle once the block has streamed its rows; its first 16 KB then serve as the merged
-    // histograms of digits 2 and 3 (general path) or as rank 0's candidate buffer (fast path).  Peers
+    unsigned char* sample_rows = reinterpret_cast<unsigned char*>(keys + tiles_per_cta * kTileRows);   // kSampleRows * RB
+    // fast path: every rank's first-digit histogram, 16-bit counts, written by the peers (merged + sm->peer_hi)
+    uint16_t* peer_hist = reinterpret_cast<uint16_t*>(merged);                    // [kMaxCluster][kFastBins]
+    // The ring is idle once the block has streamed its rows.  Its first 16 KB then serve as the merged
+    // histograms of digits 2 and 3 (general path) or as bitmask and candidate list (fast path).  Peers
     // write there only after a cluster barrier that every block reaches after its streaming loop.
     int* merged_late = reinterpret_cast<int*>(stage_base);                        // 2 * kBins ints
+    uint32_t* mask = reinterpret_cast<uint32_t*>(stage_base);                     // one bit per local slot: up to 4 KB
+    uint2* cand = reinterpret_cast<uint2*>(stage_base + kMaxKeysPerBlock / 8);    // kFastCand (key, candidate index) pairs
 
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
@@ -194,231 +234,329 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
 
     // ---- set-up -------------------------------------------------------------------------------
     phase_stamp(0);
-    for (int i = tid; i < 2 * kBins; i += kSelThreads) hist[i] = 0;               // local + merged first digit
+    const int n_tiles = (ncand + kTileRows - 1) / kTileRows;
+    const int tile0 = rank * tiles_per_cta;
+    const int my_tiles = max(0, min(tiles_per_cta, n_tiles - tile0));
+    const int slot0 = tile0 * kTileRows;               // candidate index of local slot 0
+    const int tok0 = lo + slot0;                       // its token
+    const int n_local = max(0, min(my_tiles * kTileRows, ncand - slot0));
+    const long long unit_row = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len;   // row of token 0 in the 2-D view of the cache
+    const long long row_base = unit_row + tok0;
+
+    const bool sampled = ncand >= kMinSampled;
+    // What everything else waits for is requested first, straight into shared memory with asynchronous
+    // copies: the unit's importance queries, then the sample rows.  Requested behind the grid's opening
+    // burst of bulk copies they would queue for microseconds (measured: 5 us for the queries, with the
+    // ring full and idle meanwhile).  Every block of the cluster reads the same sample rows (L2 hits for
+    // all but one); nothing waits for them here: the digit is placed a few tiles into the stream (below).
+    {
+        const float* q_unit = a.q_imp + query_row(gm, ut, ll, s, h) * DP;
+        if (tid < gm.gl * DP)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(sm->qs + tid)), "l"(q_unit + tid) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (sampled) {
+            for (int c = tid; c < kSampleRows * NCH; c += kSelThreads) {
+                const int row = c / NCH, ch = c % NCH;
+                const int slot = (int)(((long long)row * ncand) / kSampleRows);
+                const unsigned char* src = kimp + (size_t)(unit_row + lo + slot) * RB + ch * 16;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(sample_rows + c * 16)), "l"(src) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    // `issued`: tiles whose copy has been requested.  A wait that runs out (wait_limit polls; a correct
+    // run never gets there) makes the block give up streaming: it requests nothing further, still
+    // waits -- bounded -- for what it had in flight, scores the rows it never received as the lowest key
+    // and goes through every later phase and barrier, so the cluster stays in step and nothing is left
+    // in flight at exit.  The caller learns of it from the status word; that call's lists are then
+    // unspecified (valid positions, wrong choice).
+    int issued = min(n_stages, my_tiles);
     if (tid == 0) {
         prefetch_tmap(&tmap);
         for (int i = 0; i < n_stages; ++i) mbar_init(&sm->full[i], 1);
         fence_mbar_init();
-    }
-    __syncthreads();
-    // Split cluster barrier: arrive now, wait only before the first access to a peer's shared memory
-    // (after the streaming phase), so its latency hides behind the loads.
-    if (C > 1) cluster_arrive();
-
-    phase_stamp(1);
-    const int n_tiles = (ncand + kTileRows - 1) / kTileRows;
-    const int tile0 = rank * tiles_per_cta;
-    const int my_tiles = max(0, min(tiles_per_cta, n_tiles - tile0));
-    const int tok0 = lo + tile0 * kTileRows;           // token of local slot 0
-    const int n_local = max(0, min(my_tiles * kTileRows, hi - tok0));
-    const long long row_base = (long long)key_unit(gm, ut, ll, s, h) * gm.max_seq_len + tok0;   // row of the 2-D view of the cache
-
-    if (tid == 0) {
-        for (int i = 0; i < n_stages && i < my_tiles; ++i) {
+        for (int i = 0; i < issued; ++i) {
             mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
-            tma_load_2d(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kTileRows), &sm->full[i]);
-        }
-    }
-    GroupScorer<T, DP, RED> scorer;
-    scorer.load(a.q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, sm->qs);
-    if (RED != TB_GROUP_SUM) __syncthreads();
-
-    // ---- stream + score + first digit histogram -------------------------------------------------
-    bool timed_out = false;
-    int st = 0;
-    uint32_t phase = 0;
-    for (int i = 0; i < my_tiles; ++i) {
-        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;   // keep going: control flow stays uniform
-        const unsigned char* tile = stage_base + st * kTileBytes;
-        const int slot = i * kTileRows + tid;
-        if (slot < n_local) {
-            const uint32_t off = tid * RB;
-            float sc = scorer.score([&](int c) {
-                uint32_t o = off + c * 16;
-                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
-                return *reinterpret_cast<const uint4*>(tile + o);
-            });
-            uint32_t key = order_key(sc);
-            keys[slot] = key;
-            smem_add(&hist[key >> 21], 1);
-        }
-        __syncthreads();                               // all reads of this stage are done
-        if (tid == 0 && i + n_stages < my_tiles) {
-            fence_proxy_async();
-            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
-            tma_load_2d(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kTileRows),
-                        &sm->full[st]);
-        }
-        if (++st == n_stages) st = 0, phase ^= 1u;
-    }
-    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
-    // the ring is idle now: clear the part that later serves as merged histograms (see merged_late)
-    for (int i = tid; i < 2 * kBins; i += kSelThreads) merged_late[i] = 0;
-    __syncthreads();
-    phase_stamp(2);
-
-    uint32_t prefix = 0;          // digits fixed so far (value of key >> low_bits)
-    int low_bits = 32;            // bits of the key not yet fixed
-    int krem = k;
-    bool exact = false;           // the class {key >> low_bits == prefix} is taken whole
-    int start_pass = 0;
-    bool have_bases = false;      // fast path: taken / class counts of the lower ranks are already known
-    int gt_base = 0, eq_base = 0;
-
-    // ---- fast path over a cluster ----------------------------------------------------------------
-    if (C > 1) {
-        // my non-empty first-digit bins -> lists[rank] (own copy), then the same entries to every peer
-        int b[8];
-        load_bins<8>(hist, tid, b);
-        int nz = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) nz += b[i] != 0;
-        int total;
-        int off = block_excl_scan(nz, sm->warp_b, total);
-        if (total <= kListCap) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (b[i]) sm->lists[rank][off++] = ((uint32_t)(tid * 8 + i) << 16) | (uint32_t)b[i];
-        }
-        if (tid == 0) sm->list_len[rank] = total;
-        __syncthreads();
-        cluster_wait();                                // all peers run and have zeroed their histograms
-        if (total <= kListCap) {
-            for (int r = 1; r < C; ++r) {              // one remote store per thread and peer
-                const int peer = (rank + r) % C;
-                if (tid < total) *cluster.map_shared_rank(&sm->lists[rank][tid], peer) = sm->lists[rank][tid];
-            }
-        }
-        if (tid < C && tid != rank) *cluster.map_shared_rank(&sm->list_len[rank], tid) = total;
-        phase_stamp(8);
-        cluster.sync();                                // barrier 1
-        phase_stamp(9);
-        bool fast = true;
-        for (int r = 0; r < C; ++r) fast = fast && sm->list_len[r] <= kListCap;
-        if (fast) {
-            // warp w merges rank w's list into merged[0] (still zero)
-            if (warp < C)
-                for (int i = lane; i < sm->list_len[warp]; i += 32) {
-                    const uint32_t e = sm->lists[warp][i];
-                    smem_add(&merged[e >> 16], (int)(e & 0xFFFFu));
-                }
-            __syncthreads();
-            int bin, kr, bc;
-            find_digit<8>(merged, k, sm, bin, kr, bc);
-            prefix = (uint32_t)bin, low_bits = 21, krem = kr, start_pass = 1;
-            if (warp < C) {                            // warp w sums rank w's list around the threshold bin
-                int ab = 0, ib = 0;
-                for (int i = lane; i < sm->list_len[warp]; i += 32) {
-                    const uint32_t e = sm->lists[warp][i];
-                    const int eb = (int)(e >> 16), ec = (int)(e & 0xFFFFu);
-                    ab += eb > bin ? ec : 0;
-                    ib += eb == bin ? ec : 0;
-                }
-                ab = warp_sum_int(ab), ib = warp_sum_int(ib);
-                if (lane == 0) sm->above[warp] = ab, sm->inbin[warp] = ib;
-            }
-            for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
-            __syncthreads();
-            phase_stamp(10);
-            if (bc == kr) {                            // the whole threshold bin is taken: nothing to refine
-                exact = true, have_bases = true, start_pass = 3;
-                for (int r = 0; r < rank; ++r) gt_base += sm->above[r], eq_base += sm->inbin[r];
-            } else if (bc <= kCandCap) {
-                // my keys of the threshold bin -> rank 0 (any order inside my region)
-                const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
-                const int n_vec = (n_local + 3) / 4;
-                int mine = 0;
-                for (int v = tid; v < n_vec; v += kSelThreads) {
-                    const uint4 x = keys4[v];
-                    const int base = v * 4;
-                    mine += (base < n_local && (x.x >> 21) == (uint32_t)bin) + (base + 1 < n_local && (x.y >> 21) == (uint32_t)bin) +
-                            (base + 2 < n_local && (x.z >> 21) == (uint32_t)bin) + (base + 3 < n_local && (x.w >> 21) == (uint32_t)bin);
-                }
-                int tot_mine;
-                int pos = block_excl_scan(mine, sm->warp_b, tot_mine);
-                for (int r = 0; r < rank; ++r) pos += sm->inbin[r];
-                uint32_t* cand_local = reinterpret_cast<uint32_t*>(merged_late);
-                uint32_t* cand0 = cluster.map_shared_rank(cand_local, 0);
-                if (mine) {
-                    for (int v = tid; v < n_vec; v += kSelThreads) {
-                        const uint4 x = keys4[v];
-                        const int base = v * 4;
-                        if (base < n_local && (x.x >> 21) == (uint32_t)bin) cand0[pos++] = x.x;
-                        if (base + 1 < n_local && (x.y >> 21) == (uint32_t)bin) cand0[pos++] = x.y;
-                        if (base + 2 < n_local && (x.z >> 21) == (uint32_t)bin) cand0[pos++] = x.z;
-                        if (base + 3 < n_local && (x.w >> 21) == (uint32_t)bin) cand0[pos++] = x.w;
-                    }
-                }
-                phase_stamp(11);
-                cluster.sync();                        // barrier 2
-                phase_stamp(12);
-                if (rank == 0) {
-                    uint32_t pf = (uint32_t)bin;
-                    int lb = 21, kk = kr;
-                    bool ex = false;
-#pragma unroll 1
-                    for (int pass = 1; pass < 3 && !ex; ++pass) {
-                        const int bits = pass == 2 ? 10 : 11, nb = 1 << bits, shift = lb - bits;
-#pragma unroll 4
-                        for (int i = tid; i < bc; i += kSelThreads) {
-                            const uint32_t key = cand_local[i];
-                            if ((key >> lb) == pf) smem_add(&hist[(key >> shift) & (nb - 1)], 1);
-                        }
-                        __syncthreads();
-                        int d, kr2, c2;
-                        if (pass == 1) find_digit<8>(hist, kk, sm, d, kr2, c2);
-                        else find_digit<4>(hist, kk, sm, d, kr2, c2);
-                        pf = (pf << bits) | (uint32_t)d, lb = shift, kk = kr2;
-                        ex = c2 == kr2;
-                        if (!ex) {
-                            for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
-                            __syncthreads();
-                        }
-                    }
-                    if (warp < C) {                    // warp w counts rank w's candidates against the threshold
-                        int base_w = 0;
-                        for (int r = 0; r < warp; ++r) base_w += sm->inbin[r];
-                        const int n_w = sm->inbin[warp];
-                        int gt = 0, eq = 0;
-#pragma unroll 4
-                        for (int i = lane; i < n_w; i += 32) {
-                            const uint32_t kk2 = cand_local[base_w + i] >> lb;
-                            gt += kk2 > pf, eq += kk2 == pf;
-                        }
-                        gt = warp_sum_int(gt), eq = warp_sum_int(eq);
-                        if (lane == 0) sm->warp_a[warp] = gt, sm->warp_b[warp] = eq;
-                    }
-                    __syncthreads();
-                    if (tid < C) {
-                        int gb = 0, eb = 0;
-                        for (int r = 0; r < tid; ++r) gb += sm->above[r] + sm->warp_a[r], eb += sm->warp_b[r];
-                        int4* dst = reinterpret_cast<int4*>(cluster.map_shared_rank(&sm->res[0], tid));
-                        dst[0] = make_int4((int)pf, lb, kk, gb);
-                        dst[1] = make_int4(eb, 0, 0, 0);
-                    }
-                }
-                phase_stamp(13);
-                cluster.sync();                        // barrier 3
-                phase_stamp(14);
-                prefix = (uint32_t)sm->res[0], low_bits = sm->res[1], krem = sm->res[2];
-                gt_base = sm->res[3], eq_base = sm->res[4];
-                exact = true, have_bases = true, start_pass = 3;   // nothing left for the general passes
-            }
+            // drop_tile: diagnostics only (see tb_set_wait_diagnostics): the barrier is armed and the copy left out
+            if (i != drop_tile) tma_load_2d(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + (long long)i * kTileRows), &sm->full[i]);
         }
     }
     phase_stamp(3);
+    // local first-digit histogram; the general path's merged one too when the problem starts there (the
+    // fast path never reads `merged` as such: the peers overwrite their slots of it, and a fall-back zeroes it)
+    for (int i = tid; i < (sampled ? kBins : 2 * kBins); i += kSelThreads) hist[i] = 0;
+    if (tid < kMaxCluster) sm->winners[tid] = 0;
+    if (tid == 0) sm->n_cand = 0;
+    asm volatile("cp.async.wait_group 1;" ::: "memory");                          // this thread's part of the queries
+    __syncthreads();
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load_staged(sm->qs, gm.gl);
+    phase_stamp(6);
+    // Split cluster barrier: arrive now, wait only before the first access to a peer's shared memory
+    // (after the streaming phase), so its latency hides behind the loads.
+    // (Sampled problems have written nothing yet that a peer will touch, so their arrival carries no
+    // release: a releasing arrival would first wait for the sample rows still in flight.)
+    if (C > 1) {
+        if (sampled) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+        else cluster_arrive();
+    }
 
-    // ---- general path: digits not yet fixed are found with cluster-merged histograms ----------------
+    // ---- where to put the first digit's bins ---------------------------------------------------------
+    // Identical in every block of the cluster: same rows, same arithmetic.  Only the bins' resolution
+    // depends on the sample, never the result.  Called by all threads, once, when the sample rows have
+    // had time to arrive: the keys scored before that are counted then (`done_tiles` of them per thread).
+    SampledDigit dg = {0u, 22};
+    auto place_digit = [&](int done_tiles) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+        if (tid < kSampleRows) {
+            const unsigned char* row = sample_rows + tid * RB;
+            sm->sample[tid] = order_key(scorer.score([&](int c) { return *reinterpret_cast<const uint4*>(row + c * 16); }));
+        }
+        __syncthreads();
+        if (tid < kSampleRows) {   // descending rank of this thread's sample key (equal keys by index)
+            const uint32_t mine = sm->sample[tid];
+            const uint4* s4 = reinterpret_cast<const uint4*>(sm->sample);
+            int r = 0;
+#pragma unroll 8
+            for (int j4 = 0; j4 < kSampleRows / 4; ++j4) {
+                const uint4 x = s4[j4];
+                const int j = j4 * 4;
+                r += (x.x > mine) | ((x.x == mine) & (j < tid));
+                r += (x.y > mine) | ((x.y == mine) & (j + 1 < tid));
+                r += (x.z > mine) | ((x.z == mine) & (j + 2 < tid));
+                r += (x.w > mine) | ((x.w == mine) & (j + 3 < tid));
+            }
+            // about p * kSampleRows sample keys lie above the threshold (p = k / candidates); bracket it widely
+            const float p = (float)k / (float)ncand, mean = p * kSampleRows, sd = sqrtf(mean * (1.f - p));
+            // (+- 4 standard deviations of the sample rank: the threshold falls outside about once in 10^4
+            // problems, which then take the general path; a tighter bracket means fewer keys per bin)
+            const int r_hi = max(0, (int)floorf(mean - 4.f * sd) - 1), r_lo = min(kSampleRows - 1, (int)ceilf(mean + 4.f * sd) + 1);
+            if (r == r_hi) sm->s_hi = mine;
+            if (r == r_lo) sm->s_lo = mine;
+        }
+        __syncthreads();
+        const uint32_t s_lo = sm->s_lo, s_hi = sm->s_hi;
+        uint32_t range = s_hi - s_lo;
+        const uint64_t wide = (uint64_t)range + (range >> 1);   // half as much again above the highest bracketing sample
+        range = wide > 0xffffffffull ? 0xffffffffu : (uint32_t)wide;
+        dg.base = s_lo, dg.shift = 0;
+        while ((range >> dg.shift) >= (uint32_t)(kFastBins - 2)) ++dg.shift;
+        for (int i = 0; i < done_tiles; ++i) {
+            const int slot = i * kTileRows + tid;
+            if (slot < n_local) smem_add(&hist[dg.bin(keys[slot])], 1);   // this thread's own earlier keys
+        }
+    };
+    // the tile before which the digit is placed: late enough for the sample to have landed without a wait
+    const int place_at = sampled ? min(my_tiles, 6) : -1;
+    phase_stamp(1);
+
+    // ---- stream + score + first digit histogram -------------------------------------------------
+    bool dead = false;
+    int st = 0;
+    uint32_t phase = 0;
+    for (int i = 0; i < my_tiles; ++i) {
+        if (i == place_at) place_digit(i);
+        const bool ok = i < issued && mbar_wait(&sm->full[st], phase, wait_limit);
+        const unsigned char* tile = stage_base + st * kTileBytes;
+        const int slot = i * kTileRows + tid;
+        if (slot < n_local) {
+            uint32_t key = 0u;
+            if (ok) {
+                const uint32_t off = tid * RB;
+                const float sc = scorer.score([&](int c) {
+                    uint32_t o = off + c * 16;
+                    o ^= ((o >> 7) & (NCH - 1)) << 4;  // TMA swizzle of 16-byte chunks (mode = row size)
+                    return *reinterpret_cast<const uint4*>(tile + o);
+                });
+                key = order_key(sc);
+            }
+            keys[slot] = key;
+            if (!sampled) smem_add(&hist[key >> 21], 1);
+            else if (i >= place_at) smem_add(&hist[dg.bin(key)], 1);
+        }
+        if (__syncthreads_or(!ok)) dead = true;        // all reads of this stage are done; uniform verdict on the wait
+        if (!dead && i + n_stages < my_tiles) {
+            if (tid == 0) {
+                fence_proxy_async();
+                mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+                if (i + n_stages != drop_tile)
+                    tma_load_2d(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kTileRows),
+                                &sm->full[st]);
+            }
+            issued = i + n_stages + 1;
+        }
+        if (++st == n_stages) st = 0, phase ^= 1u;
+    }
+    if (dead && tid == 0) atomicExch(status, kStatusTimeout);
+    if (place_at == my_tiles) {                        // a short share: the digit is placed after its last tile
+        place_digit(my_tiles);
+        __syncthreads();                               // the histogram is read next
+    }
+    phase_stamp(2);
+
+    uint32_t prefix = 0;          // general path: digits fixed so far (value of key >> low_bits)
+    int low_bits = 32;            // bits of the key not yet fixed
+    int krem = k;
+    bool exact = false;           // the class {key >> low_bits == prefix} is taken whole
+    bool rebuild_first = false;   // general path after a fast-path attempt: the first digit's histogram comes from the keys
+
+    // ---- fast path --------------------------------------------------------------------------------------
+    if (sampled) {
+        // my histogram, 16-bit counts, into slot `rank` of every block's copy (4 bins = 8 bytes per thread and peer)
+        {
+            const int4 x = reinterpret_cast<const int4*>(hist)[tid];
+            const uint2 packed = make_uint2((uint32_t)x.x | ((uint32_t)x.y << 16), (uint32_t)x.z | ((uint32_t)x.w << 16));
+            uint2* mine = reinterpret_cast<uint2*>(peer_hist + rank * kFastBins) + tid;
+            if (C > 1) cluster_wait();                 // every peer runs (its shared memory exists) and is past zeroing it
+            for (int r = 0; r < C; ++r) *cluster.map_shared_rank(mine, (rank + r) % C) = packed;
+        }
+        phase_stamp(8);
+        if (C > 1) cluster.sync(); else __syncthreads();   // barrier 1: every block's histogram is everywhere, every ring idle
+        phase_stamp(9);
+        // threshold bin from the cluster's histogram; with it, the keys that the lower ranks hold above the bin
+        // (where this block's part of the list starts) and every rank's keys inside it
+        int b[4] = {0, 0, 0, 0}, low[4] = {0, 0, 0, 0};
+        for (int r = 0; r < C; ++r) {
+            const uint2 x = reinterpret_cast<const uint2*>(peer_hist + r * kFastBins)[tid];
+            const int c0 = (int)(x.x & 0xffffu), c1 = (int)(x.x >> 16), c2 = (int)(x.y & 0xffffu), c3 = (int)(x.y >> 16);
+            b[0] += c0, b[1] += c1, b[2] += c2, b[3] += c3;
+            if (r < rank) low[0] += c0, low[1] += c1, low[2] += c2, low[3] += c3;
+        }
+        int bin, kr, bc;
+        find_digit_regs<4>(b, k, sm, bin, kr, bc);
+        {
+            int la = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) la += tid * 4 + i > bin ? low[i] : 0;
+            la = warp_sum_int(la);
+            if (lane == 0) sm->warp_b[warp] = la;
+            if (tid < C) sm->inbin[tid] = (int)peer_hist[tid * kFastBins + bin];
+        }
+        __syncthreads();
+        int lower_above = 0;
+#pragma unroll
+        for (int w = 0; w < kSelWarps; ++w) lower_above += sm->warp_b[w];
+        phase_stamp(10);
+        phase_value(4, (unsigned long long)bin), phase_value(5, (unsigned long long)bc), phase_value(14, (unsigned long long)kr);
+        phase_value(15, ((unsigned long long)dg.base << 8) | (unsigned)dg.shift);
+        const bool whole = bc == kr;                   // the whole threshold bin is taken: nothing to rank
+#ifdef TB_PHASE_TIMING
+        if (rank == 0 && tid == 0) atomicAdd(&g_sel_fallbacks[whole || bc <= kFastCand ? 0 : 1], 1u);
+#endif
+        if (whole || bc <= kFastCand) {
+            // Keys of the threshold bin: [bin_from, above_from); keys of the bins above it: [above_from, 2^32), if any.
+            const uint64_t above64 = bin == 0 ? (uint64_t)dg.base : bin == kFastBins - 1 ? (1ull << 32) : (uint64_t)dg.base + ((uint64_t)bin << dg.shift);
+            const uint64_t from64 = bin == 0 ? 0ull : (uint64_t)dg.base + ((uint64_t)(bin - 1) << dg.shift);
+            const uint32_t above_ok = above64 <= 0xffffffffull ? 0xfu : 0u, above_from = (uint32_t)above64;
+            const uint32_t from_ok = from64 <= 0xffffffffull ? 0xfu : 0u, bin_from = (uint32_t)from64;
+            int cand_base = 0;
+            for (int r = 0; r < rank; ++r) cand_base += sm->inbin[r];
+            // own keys -> bitmask (lane l of a warp holds slots 128 g + 4 l .. + 3: its four verdicts are a
+            // nibble, eight lanes' nibbles make a mask word); own keys of the threshold bin -> every block's list
+            const uint4* keys4 = reinterpret_cast<const uint4*>(keys);
+            const int n_grp = (n_local + kTileRows - 1) / kTileRows;
+#pragma unroll 4
+            for (int v = tid; v < n_grp * (kTileRows / 4); v += kSelThreads) {
+                const uint4 x = keys4[v];
+                const uint32_t kk[4] = {x.x, x.y, x.z, x.w};
+                uint32_t ab = (uint32_t)(kk[0] >= above_from) | (uint32_t)(kk[1] >= above_from) << 1 | (uint32_t)(kk[2] >= above_from) << 2 |
+                              (uint32_t)(kk[3] >= above_from) << 3;
+                uint32_t ge = (uint32_t)(kk[0] >= bin_from) | (uint32_t)(kk[1] >= bin_from) << 1 | (uint32_t)(kk[2] >= bin_from) << 2 |
+                              (uint32_t)(kk[3] >= bin_from) << 3;
+                ab &= above_ok, ge &= from_ok;
+                const uint32_t vm = v * 4 + 3 < n_local ? 0xfu : v * 4 < n_local ? (1u << (n_local - v * 4)) - 1u : 0u;   // slots past the end hold stale keys
+                ab &= vm, ge &= vm;
+                uint32_t eqm = whole ? 0u : ge & ~ab;
+                uint32_t word = (whole ? ge : ab) << (4 * (lane & 7));
+                word |= __shfl_xor_sync(0xffffffffu, word, 1);
+                word |= __shfl_xor_sync(0xffffffffu, word, 2);
+                word |= __shfl_xor_sync(0xffffffffu, word, 4);
+                if ((lane & 7) == 0) mask[v >> 3] = word;
+                while (eqm) {                          // rare: a handful of keys per block
+                    const int e = __ffs(eqm) - 1;
+                    eqm &= eqm - 1;
+                    const int i = cand_base + atomicAdd(&sm->n_cand, 1);
+                    const uint2 ent = make_uint2(kk[e], (uint32_t)(slot0 + v * 4 + e));
+                    for (int r = 0; r < C; ++r) *cluster.map_shared_rank(&cand[i], (rank + r) % C) = ent;
+                }
+            }
+            phase_stamp(11);
+            if (C > 1) cluster.sync(); else __syncthreads();   // barrier 2: the list is complete everywhere
+            phase_stamp(12);
+            if (!whole) {
+                // every block ranks the list itself: an entry counts the entries ranked before it (larger key, or
+                // equal key at a lower position) and knows at once whether it is among the `kr` winners
+                if (tid < bc) {
+                    const uint2 it = cand[tid];
+                    int before = 0;
+#pragma unroll 4
+                    for (int j = 0; j < bc; ++j) {
+                        const uint2 o = cand[j];
+                        before += (o.x > it.x) | ((o.x == it.x) & (o.y < it.y));
+                    }
+                    if (before < kr) {
+                        int r_of = 0, i_of = tid;
+                        while (i_of >= sm->inbin[r_of]) i_of -= sm->inbin[r_of], ++r_of;
+                        atomicAdd(&sm->winners[r_of], 1);
+                        if (r_of == rank) {
+                            const int ls = (int)it.y - slot0;
+                            atomicOr(&mask[ls >> 5], 1u << (ls & 31));
+                        }
+                    }
+                }
+                __syncthreads();
+            }
+            phase_stamp(13);
+            // ascending list from the mask: each thread owns a run of 16-bit half words
+            int out_base = lower_above;
+            for (int r = 0; r < rank; ++r) out_base += whole ? sm->inbin[r] : sm->winners[r];
+            const uint16_t* mask16 = reinterpret_cast<const uint16_t*>(mask);
+            const int n_half = n_grp * (kTileRows / 16);
+            const int per = (n_half + kSelThreads - 1) / kSelThreads;
+            const int w0 = min(n_half, tid * per), w1 = min(n_half, w0 + per);
+            int cnt = 0;
+            for (int w = w0; w < w1; ++w) cnt += __popc((uint32_t)mask16[w]);
+            int total;
+            int o = out_base + block_excl_scan(cnt, sm->warp_b, total);
+            for (int w = w0; w < w1; ++w) {
+                uint32_t bits = mask16[w];
+                while (bits) {
+                    const int bpos = __ffs(bits) - 1;
+                    bits &= bits - 1;
+                    if (o < k) idx_dst[o] = tok0 + w * 16 + bpos;
+                    ++o;
+                }
+            }
+            if (rank == 0 && tid == 0) *cnt_dst = k;
+            phase_stamp(7);
+            return;
+        }
+        // A crowded threshold bin (massive ties, a threshold outside the bracket).  The decision is the same
+        // in every block.  The general path needs the merged histograms zero before any peer adds to them.
+        for (int i = tid; i < 2 * kBins; i += kSelThreads) hist[i] = 0;
+        for (int i = tid; i < 2 * kBins; i += kSelThreads) merged_late[i] = 0;
+        rebuild_first = true;
+        if (C > 1) cluster.sync(); else __syncthreads();
+    } else {
+        // the ring is idle now: clear the part that later serves as merged histograms (see merged_late)
+        for (int i = tid; i < 2 * kBins; i += kSelThreads) merged_late[i] = 0;
+        __syncthreads();
+        if (C > 1) cluster_wait();                     // every peer runs and has zeroed its histograms
+    }
+    phase_stamp(3);
+
+    // ---- general path: the key's own digits through cluster-merged histograms -----------------------------
 #pragma unroll 1
-    for (int pass = start_pass; pass < 3; ++pass) {
+    for (int pass = 0; pass < 3; ++pass) {
         const int bits = pass == 2 ? 10 : 11;
         const int nbins = 1 << bits;
         const int shift = low_bits - bits;
-        if (pass > 0) {
+        if (pass > 0 || rebuild_first) {
             if (!exact) {
                 for (int i = tid; i < n_local; i += kSelThreads) {
                     uint32_t key = keys[i];
-                    if ((key >> low_bits) == prefix) smem_add(&hist[(key >> shift) & (nbins - 1)], 1);
+                    if (pass == 0 || (key >> low_bits) == prefix) smem_add(&hist[(key >> shift) & (nbins - 1)], 1);
                 }
             }
             __syncthreads();
@@ -488,9 +626,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
         gt_before += w < warp ? x : 0, eq_before += w < warp ? y : 0;
         gt_cta += x, eq_cta += y;
     }
-    if (have_bases) {
-        gt_before += gt_base, eq_before += eq_base;
-    } else if (C > 1) {
+    if (C > 1) {
         if (tid < C) {
             int* dst = cluster.map_shared_rank(&sm->tot[rank][0], tid);
             dst[0] = gt_cta, dst[1] = eq_cta;
@@ -539,16 +675,16 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     phase_stamp(7);
 }
 
-// Shared memory of one block without its TMA ring: alignment slack, two histograms, control block, keys.
-static size_t select_fixed_smem(int tiles_per_cta) {
-    return 1024 + 2 * kBins * sizeof(int) + sizeof(SelSmem) + (size_t)tiles_per_cta * kTileRows * 4;
+// Shared memory of one block without its TMA ring: alignment slack, two histograms, control block, keys, sample rows.
+static size_t select_fixed_smem(int tiles_per_cta, int tile_bytes) {
+    return 1024 + 2 * kBins * sizeof(int) + sizeof(SelSmem) + (size_t)tiles_per_cta * kTileRows * 4 + (size_t)kSampleRows * (tile_bytes / kTileRows);
 }
 
 // Ring depth: the score pass is bound by bytes in flight (bandwidth x loaded latency is about 90 KB
 // per SM), so take as many stages as fit while keeping two blocks per SM when the keys leave room
 // for that, one block per SM otherwise.  At least 16 KB of ring (reused after streaming).
 static int select_stage_count(int tiles_per_cta, int tile_bytes) {
-    const size_t fixed = select_fixed_smem(tiles_per_cta);
+    const size_t fixed = select_fixed_smem(tiles_per_cta, tile_bytes);
     const size_t two_per_sm = 113 * 1024, one_per_sm = 226 * 1024;
     const int min_stages = tile_bytes >= 16384 ? 2 : 16384 / tile_bytes + 1;
     int n = fixed + (size_t)3 * tile_bytes <= two_per_sm ? (int)((two_per_sm - fixed) / tile_bytes)
@@ -559,7 +695,7 @@ static int select_stage_count(int tiles_per_cta, int tile_bytes) {
     return n;
 }
 
-cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
+cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry) {
     const Geom& gm = c->geom;
     const int n_units = ut.layer_count * ut.n_seq * gm.Hl;
     int max_cand = 0;
@@ -570,11 +706,13 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     // Many problems (one and a half per SM or more; measured crossover between 32 and 256 on 148 SMs)
     // fill the GPU by themselves: one block each, no clusters.  So do problems beyond what the parked-key
     // cluster kernel takes.
-    if (2 * n_units >= 3 * c->sm_count || max_cand > kCwLimit) return launch_select_wave(c, ut, a, s);
+    const bool to_wave = 2 * n_units >= 3 * c->sm_count || max_cand > kCwLimit, to_cw = max_cand > kCwFrom && max_cand <= kCwLimit;
+    if (c->drop_tile >= 0 && (to_wave || to_cw)) return cudaErrorInvalidConfiguration;   // wait diagnostics: single-block launches of this kernel only
+    if (to_wave) return launch_select_wave(c, ut, a, s, dry);
     // Long problems (beyond ~48K candidates) go to the cluster kernel that parks the keys in memory and
     // keeps 2 bytes per row on chip: two blocks per SM where this one, with 4 bytes per row, has room for
     // one (128K tokens: 70.1 -> 59.1 us per launch; at 32K the two are level, below that this one wins).
-    if (max_cand > kCwFrom && max_cand <= kCwLimit) return launch_select_cw(c, ut, a, s);
+    if (to_cw) return launch_select_cw(c, ut, a, s, dry);
     const int n_tiles = (max_cand + kTileRows - 1) / kTileRows;
     // Cluster size: enough blocks to cover the GPU about twice, at least 4 tiles per block, and a
     // key array per block of at most 32 KB where the cluster limit allows (64 KB otherwise).
@@ -591,7 +729,7 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
         if (C > kMaxCluster) C = kMaxCluster;
         while (C > 1 && n_tiles / C < 4) --C;
         const int tpc = (n_tiles + C - 1) / C;
-        if (1024 + 2 * kBins * 4 + sizeof(SelSmem) + (size_t)tpc * kTileRows * 4 + 3 * (size_t)tile_b > 113 * 1024) {
+        if (select_fixed_smem(tpc, tile_b) + 3 * (size_t)tile_b > 113 * 1024) {
             C = c->sm_count / n_units;
             if (C > kMaxCluster) C = kMaxCluster;
             while (C > 1 && n_tiles / C < 4) --C;
@@ -603,7 +741,14 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
     if (tiles_per_cta * kTileRows > kMaxKeysPerBlock) return cudaErrorInvalidConfiguration;
     const int tile_bytes = kTileRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
     const int n_stages = select_stage_count(tiles_per_cta, tile_bytes);
-    size_t smem = select_fixed_smem(tiles_per_cta) + (size_t)n_stages * tile_bytes;
+    size_t smem = select_fixed_smem(tiles_per_cta, tile_bytes) + (size_t)n_stages * tile_bytes;
+
+    // diagnostics of the bounded waits (tb_set_wait_diagnostics): one-shot, single-block launches only
+    const uint32_t wait_limit = c->wait_poll_limit > 0 ? (uint32_t)c->wait_poll_limit : kWaitPollLimit;
+    const int drop_tile = C == 1 && n_units == 1 ? c->drop_tile : -1;
+    if (c->drop_tile >= 0 && drop_tile < 0) return cudaErrorInvalidConfiguration;
+    if (dry) return cudaSuccess;
+    const_cast<tb_ctx*>(c)->drop_tile = -1;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(C, n_units, 1);
@@ -628,8 +773,8 @@ cudaError_t launch_select(const tb_ctx* c, const UnitTable& ut, const SelectArgs
                                                  227 * 1024);                                                      \
             if (e != cudaSuccess) return e;                                                                        \
         }                                                                                                          \
-        return cudaLaunchKernelEx(&cfg, select_kernel<T, DP, RED>, c->kimp_map, gm, ut, a, tiles_per_cta, n_stages, c->st.idx, \
-                                  c->st.cnt, c->st.status);                                                        \
+        return cudaLaunchKernelEx(&cfg, select_kernel<T, DP, RED>, c->kimp_map, (const unsigned char*)c->kimp, gm, ut, a, \
+                                  tiles_per_cta, n_stages, wait_limit, drop_tile, c->st.idx, c->st.cnt, c->st.status); \
     } while (0)
 #define TB_SEL(T, DP)                                            \
     do {                                                         \

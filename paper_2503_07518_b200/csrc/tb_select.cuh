@@ -89,6 +89,12 @@ struct GroupScorer {
             for (int i = threadIdx.x; i < g_ * DP; i += blockDim.x) qs_smem[i] = q_unit[i];
         }
     }
+    // The same from queries that already sit in shared memory ([g][DP] floats, visible to the thread):
+    // the summed query is built in the same order, so the scores are the same bits.
+    __device__ __forceinline__ void load_staged(const float* qs_smem, int g_) {
+        g = g_, qs = qs_smem;
+        if constexpr (RED == TB_GROUP_SUM) load_group_query<DP>(qs_smem, g_, qr);
+    }
     template <typename LoadChunk>
     __device__ __forceinline__ float score(LoadChunk ld) const {
         if constexpr (RED == TB_GROUP_SUM) return row_score<T, DP>(qr, ld);

@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(kNbThreads) neighbor_kernel(Geom gm, UnitTable
     if (tid == 0) state_cnt[cu] = all;
 }
 
-cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s) {
+cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s, bool dry) {
     const Geom& gm = c->geom;
     int max_span = 0;
     for (int i = 0; i < ut.layer_count * ut.n_seq; ++i) {
@@ -128,12 +128,13 @@ cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const Neighbo
         if (hi - lo > max_span) max_span = hi - lo;
     }
     size_t smem = (size_t)((max_span + 31) / 32) * 4 + 16;
+    if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;   // one bit per candidate on chip: up to 1,638,272 candidates
+    if (dry) return cudaSuccess;
     static unsigned char seen[64];
     if (first_use_on_this_device(seen)) {
         cudaError_t e = cudaFuncSetAttribute(neighbor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
     }
-    if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
     neighbor_kernel<<<ut.layer_count * ut.n_seq * gm.Hl, kNbThreads, smem, s>>>(gm, ut, a, c->st.idx, c->st.cnt);
     return cudaGetLastError();
 }

@@ -574,35 +574,45 @@ __global__ void __launch_bounds__(kThreads, 4)
     }
 
     // ---- stream + score + first digit histogram -------------------------------------------------
-    bool timed_out = false;
+    // A wait that runs out (never in a correct run) makes the block give up streaming: it requests no
+    // further tile, still waits -- bounded -- for those in flight, gives the rows it never received the
+    // lowest key and finishes normally; the status word tells the caller that this call's lists are void.
+    bool dead = false;
+    int issued = min(n_stages, n_tiles);               // tiles whose copy has been requested
     int st = 0;
     uint32_t phase = 0;
     for (int i = 0; i < n_tiles; ++i) {
-        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;   // keep going: control flow stays uniform
+        const bool ok = i < issued && mbar_wait(&sm->full[st], phase);
         const unsigned char* tile = stage_base + st * kTileBytes;
         const int slot = i * kRows + tid;
         if (i == 0) wave_stamp(1);
         if (slot < ncand) {
-            const uint32_t off = tid * RB;
-            const float sc = scorer.score([&](int c) {
-                uint32_t o = off + c * 16;
-                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
-                return *reinterpret_cast<const uint4*>(tile + o);
-            });
-            const uint32_t key = order_key(sc);
+            uint32_t key = 0u;
+            if (ok) {
+                const uint32_t off = tid * RB;
+                const float sc = scorer.score([&](int c) {
+                    uint32_t o = off + c * 16;
+                    o ^= ((o >> 7) & (NCH - 1)) << 4;  // TMA swizzle of 16-byte chunks (mode = row size)
+                    return *reinterpret_cast<const uint4*>(tile + o);
+                });
+                key = order_key(sc);
+            }
             st_global_hint(keys_unit + slot, key, keep_policy);
             hist_add(&hist[dg.bin(key)]);
         }
-        __syncthreads();                               // all reads of this stage are done
-        if (tid == 0 && i + n_stages < n_tiles) {
-            fence_proxy_async();
-            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
-            tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kRows), &sm->full[st],
-                             stream_policy);
+        if (__syncthreads_or(!ok)) dead = true;        // all reads of this stage are done; uniform verdict on the wait
+        if (!dead && i + n_stages < n_tiles) {
+            if (tid == 0) {
+                fence_proxy_async();
+                mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+                tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + (long long)(i + n_stages) * kRows), &sm->full[st],
+                                 stream_policy);
+            }
+            issued = i + n_stages + 1;
         }
         if (++st == n_stages) st = 0, phase ^= 1u;
     }
-    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    if (dead && tid == 0) atomicExch(status, kStatusTimeout);
     __syncthreads();                                   // histogram complete, own keys visible to the block
     wave_stamp(2);
 
@@ -623,7 +633,7 @@ extern "C" int tb_debug_fin_blk(unsigned long long* out) { return (int)cudaMemcp
 extern "C" int tb_debug_wave_ns(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_wave_ns, sizeof(g_wave_ns)); }
 #endif
 
-cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
+cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry) {
     const Geom& gm = c->geom;
     const int n_pairs = ut.layer_count * ut.n_seq, n_units = n_pairs * gm.Hl;
     WaveOrder order;
@@ -650,6 +660,7 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
 #define TB_KEEP_BYTES 96e6
 #endif
     const int keep_in_l2 = parked <= TB_KEEP_BYTES;
+    if (dry) return cudaSuccess;
 
 #define TB_SEL_R(T, DP, RED)                                                                                                   \
     do {                                                                                                                \
@@ -839,22 +850,26 @@ __global__ void __launch_bounds__(kThreads, 2)
 
     CW_MARK(1);
     // ---- stream: score, park the key, keep the first digit ---------------------------------------------
-    bool timed_out = false;
+    bool dead = false;                                 // a wait ran out: see the kernel above
+    int issued = min(n_stages, my_tiles);
     int st = 0;
     uint32_t phase = 0;
     for (int i = 0; i < my_tiles; ++i) {
-        if (!mbar_wait(&sm->full[st], phase)) timed_out = true;
+        const bool ok = i < issued && mbar_wait(&sm->full[st], phase);
         const unsigned char* tile = stage_base + st * kTileBytes;
         const int slot = i * kRows + tid;
         uint16_t b = 0;                                // rows past the end: below everything
         if (slot < n_local) {
-            const uint32_t off = tid * RB;
-            const float sc = scorer.score([&](int c) {
-                uint32_t o = off + c * 16;
-                o ^= ((o >> 7) & (NCH - 1)) << 4;      // TMA swizzle of 16-byte chunks (mode = row size)
-                return *reinterpret_cast<const uint4*>(tile + o);
-            });
-            const uint32_t key = order_key(sc);
+            uint32_t key = 0u;
+            if (ok) {
+                const uint32_t off = tid * RB;
+                const float sc = scorer.score([&](int c) {
+                    uint32_t o = off + c * 16;
+                    o ^= ((o >> 7) & (NCH - 1)) << 4;  // TMA swizzle of 16-byte chunks (mode = row size)
+                    return *reinterpret_cast<const uint4*>(tile + o);
+                });
+                key = order_key(sc);
+            }
 #ifdef TB_NOHINT
             keys_unit[slot0 + slot] = key;
 #else
@@ -864,16 +879,19 @@ __global__ void __launch_bounds__(kThreads, 2)
             hist_add(&hist[b]);
         }
         bins[slot] = b;
-        __syncthreads();
-        if (tid == 0 && i + n_stages < my_tiles) {
-            fence_proxy_async();
-            mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
-            tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + slot0 + (long long)(i + n_stages) * kRows),
-                             &sm->full[st], stream_policy);
+        if (__syncthreads_or(!ok)) dead = true;
+        if (!dead && i + n_stages < my_tiles) {
+            if (tid == 0) {
+                fence_proxy_async();
+                mbar_arrive_expect_tx(&sm->full[st], kTileBytes);
+                tma_load_2d_hint(stage_base + st * kTileBytes, &tmap, 0, (int)(row_base + slot0 + (long long)(i + n_stages) * kRows),
+                                 &sm->full[st], stream_policy);
+            }
+            issued = i + n_stages + 1;
         }
         if (++st == n_stages) st = 0, phase ^= 1u;
     }
-    if (timed_out && lane == 0) atomicExch(status, kStatusTimeout);
+    if (dead && tid == 0) atomicExch(status, kStatusTimeout);
     __syncthreads();
     CW_MARK(2);
 #ifdef TB_PHASE_TIMING
@@ -1054,7 +1072,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     CW_MARK(3);
 }
 
-cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s) {
+cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry) {
     const Geom& gm = c->geom;
     const int n_units = ut.layer_count * ut.n_seq * gm.Hl;
     int max_cand = 0;
@@ -1088,6 +1106,7 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
     while ((size_t)n_stages * tile_bytes < ring_min) ++n_stages;
     const size_t smem = fixed + (size_t)n_stages * tile_bytes;
     if (smem > 226 * 1024 || n_stages > kStagesMax) return cudaErrorInvalidConfiguration;
+    if (dry) return cudaSuccess;
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(C, n_units, 1), cfg.blockDim = dim3(kThreads, 1, 1), cfg.dynamicSmemBytes = smem, cfg.stream = s;

@@ -1,0 +1,111 @@
+"""Boundary behaviour of the C ABI on the GPU: errors found before the first launch, the bounded-wait
+path of the selection kernel in its safe form, and the analytic byte counter behind every roofline
+figure."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2503_07518_b200 import workloads as wl  # noqa: E402
+from test_gpu_parity import H, tb  # noqa: E402,F401
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable(H):
+    """One tile's barrier is armed without its copy being requested (diagnostic hook, single-block launch
+    only, so nothing else is in flight and no other block waits).  The wait gives up after its poll
+    limit, the kernel finishes normally, the status word says TB_ERR_TIMEOUT, and the next ordinary call
+    on the same context is clean and exact."""
+    b_ = tb()
+    w = wl.workload(2, n_layers=1, n_q_heads=4, n_kv_heads=1, lengths=[900], budget=50)     # 4 tiles, one block
+    case = H.Case(w)
+    q, qi = H.queries(w)
+    p = b_.select_params(w.budget, 0, 0)
+    clean = H.gpu_select(case, qi, p)
+    assert case.ctx.get_status() == 0
+    case.ctx.set_wait_diagnostics(poll_limit=2000, drop_tile=1)
+    n0 = case.ctx.launch_count()
+    lost = H.gpu_select(case, qi, p)
+    assert case.ctx.launch_count() > n0                                  # the kernel ran and returned
+    assert case.ctx.get_status() == b_.TB_ERR_TIMEOUT
+    assert case.ctx.get_status() == 0                                    # reading clears it
+    assert len(lost[0][0][0]) == w.budget and np.all((lost[0][0][0] >= 0) & (lost[0][0][0] < 900))   # void, but in range
+    case.ctx.set_wait_diagnostics(0, -1)
+    again = H.gpu_select(case, qi, p)
+    assert case.ctx.get_status() == 0
+    _, full, _ = case.oracle_select(0, 0, 0, qi[0, 0], p)
+    assert np.array_equal(again[0][0][0], clean[0][0][0]) and np.array_equal(again[0][0][0], full)
+    out, _ = H.gpu_attention(case, q, p)                                 # and attention from the stored list still matches
+    ref, _ = case.oracle_attention(0, 0, 0, q[0, 0], full, p)
+    assert np.abs(out[0, 0] - ref).max() <= 2e-3
+
+
+def test_wait_diagnostics_are_refused_by_multi_block_launches(H):
+    """The hook never reaches a launch in which another block could be left waiting: such a call returns
+    TB_ERR_UNSUPPORTED and launches nothing."""
+    b_ = tb()
+    w = wl.workload(2, n_layers=1, n_q_heads=8, n_kv_heads=2, lengths=[5000], budget=50)    # two lists, clusters
+    case = H.Case(w)
+    _, qi = H.queries(w)
+    case.ctx.set_wait_diagnostics(poll_limit=2000, drop_tile=0)
+    n0 = case.ctx.launch_count()
+    with pytest.raises(b_.TBError) as e:
+        H.gpu_select(case, qi, b_.select_params(w.budget))
+    assert e.value.status == b_.TB_ERR_UNSUPPORTED and case.ctx.launch_count() == n0
+    case.ctx.set_wait_diagnostics(0, -1)
+    H.gpu_select(case, qi, b_.select_params(w.budget))
+    assert case.ctx.get_status() == 0
+
+
+def test_oversized_neighbour_span_is_refused_before_anything_runs(H):
+    """Neighbour expansion keeps one bit per candidate on chip (up to 1,638,272 candidates).  A longer
+    sequence is selected from without neighbours, and refused with them -- before the selection kernel of
+    the same call is launched, not after it."""
+    b_ = tb()
+    L = 1_700_000
+    ctx = b_.Context(1, 1, 1, 128, 32, b_.TB_BF16, 1, L + 8, 64, max_radius=1)
+    ctx.set_projection(0, torch.zeros(1, 128, 32, dtype=torch.bfloat16, device="cuda"))
+    k = torch.zeros(L, 1, 128, dtype=torch.bfloat16, device="cuda")
+    k[::1000, 0, 0] = 1.0
+    ctx.append_kv(0, 1, None, [L], k, k)
+    ctx.project_keys(0, 1, None, [0], [L])
+    qi = torch.ones(1, 1, 1, 32, device="cuda")
+    idx = torch.zeros(1, 1, 1, ctx.index_capacity, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, 1, 1, dtype=torch.int32, device="cuda")
+    ctx.select_topk(0, 1, None, 1, qi, b_.select_params(64), idx, cnt)           # all scores equal: the first 64 positions
+    torch.cuda.synchronize()
+    assert cnt.item() == 64 and np.array_equal(idx[0, 0, 0, :64].cpu().numpy(), np.arange(64))
+    n0 = ctx.launch_count()
+    with pytest.raises(b_.TBError) as e:
+        ctx.select_topk(0, 1, None, 1, qi, b_.select_params(64, radius=1), idx, cnt)
+    assert e.value.status == b_.TB_ERR_UNSUPPORTED
+    assert ctx.launch_count() == n0 and ctx.get_length(0, 0) == (L, L)
+    out = torch.empty(1, 1, 128, device="cuda")
+    ctx.sparse_decode_attention(0, 1, None, 1, k[:1, 0], b_.select_params(64), out)   # the stored list is still the first call's
+    assert ctx.get_status() == 0
+
+
+def test_byte_counter_reproduces_the_papers_bandwidth_reduction(H):
+    """tb_last_step_bytes is the numerator of every roofline figure.  At 64K tokens with about 8K
+    accessed (128 sinks + 7808 selected + 256 recent) the K/V bytes of a sparse step are 1/8.00 of the
+    dense step's (Sec. 4.2: "8x" KV-access reduction); the selection reads d' elements per candidate
+    and key stream."""
+    b_ = tb()
+    L, S, W, B = 65536, 128, 256, 7808
+    ctx = b_.Context(1, 32, 8, 128, 32, b_.TB_BF16, 1, L + 8, B)
+    ctx.set_projection(0, torch.zeros(8, 128, 32, dtype=torch.bfloat16, device="cuda"))
+    k = torch.zeros(L, 8, 128, dtype=torch.bfloat16, device="cuda")
+    ctx.append_kv(0, 1, None, [L], k, k)
+    ctx.project_keys(0, 1, None, [0], [L])
+    p = b_.select_params(B, S, W)
+    ctx.select_topk(0, 1, None, 1, torch.ones(1, 1, 32, 32, device="cuda"), p)
+    assert ctx.last_step_bytes() == (L - S - W) * 8 * 32 * 2
+    q = torch.zeros(1, 32, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.empty(1, 32, 128, device="cuda")
+    ctx.sparse_decode_attention(0, 1, None, 1, q, p, out)
+    sparse = ctx.last_step_bytes()
+    ctx.sparse_decode_attention(0, 1, None, 1, q, b_.select_params(-1), out)
+    dense = ctx.last_step_bytes()
+    assert sparse == (S + B + W) * 8 * 2 * 128 * 2 == 8192 * 8 * 512
+    assert dense == L * 8 * 512 and dense / sparse == 8.0
+    assert ctx.get_status() == 0

@@ -10,6 +10,10 @@ layers.  Default workload: the Llama-3-8B-shaped decode at 32K context (32 layer
 The printed JSON line carries the device-timed throughput (inputs resident in HBM), the same metric
 end to end through the public API with pinned host buffers, the roofline of the dominant kernel
 measured live with CUDA events, and the CPU oracle timed on a bounded sample of the same workload.
+Run without --config, the line also carries a `workloads` block with the same measurements, in brief, for
+the batched-serving, long-context and prediction-interval workloads (configs 3, 4, 5) at their full sizes.
+Every timed region is K steps between device events; it is repeated until at least 0.3 s have been timed
+and the median repeat is reported (min and max beside it).
 """
 from __future__ import annotations
 
@@ -85,8 +89,8 @@ def oracle_sample(w: wl.Workload, n_layers: int, passes: int, threads: int, max_
     return times, len(units)
 
 
-def cpu_leg(w: wl.Workload, sample_layers: int, passes: int, max_units: int = 0):
-    threads = len(os.sched_getaffinity(0))
+def cpu_leg(w: wl.Workload, sample_layers: int, passes: int, max_units: int = 0, threads: int = 0):
+    threads = threads or len(os.sched_getaffinity(0))
     times, n_units = oracle_sample(w, sample_layers, passes, threads, max_units)
     total_units = w.n_layers * w.batch * w.n_kv_heads
     step_s = [t * total_units / n_units for t in times]          # units are independent: linear scaling
@@ -210,19 +214,31 @@ def fill_caches(ctx, w, torch, tbh):
     return {"us_per_layer": ms * 1e3, "bytes_per_layer": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9}
 
 
-def run_ours(args, w):
+def dist_env(torch, dist):
+    """(world, rank, local) of this process; the NCCL group (barrier + max-over-ranks only) is set up once."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+def storage_name(w):
+    return "bf16" if w.dtype == wl.BF16 else "f32"
+
+
+def measure_static(args, w, brief=False):
+    """Workloads whose lengths do not change (configs 1-4): the step is captured once in a CUDA graph and
+    replayed.  Returns the JSON line as a dict (without the CPU baseline).  `brief`: the step, its two
+    kernels and the end-to-end figure only (the entries of the default run's `workloads` block)."""
     import torch
     import torch.distributed as dist
     from paper_2503_07518_b200 import binding as tbh
     from paper_2503_07518_b200 import build
     build.build()
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    world, rank, local = dist_env(torch, dist)
 
     p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode)
     scope = {"kv_head": tbh.TB_SCOPE_KV_HEAD, "q_head": tbh.TB_SCOPE_Q_HEAD, "layer": tbh.TB_SCOPE_LAYER}[args.list_scope]
@@ -237,21 +253,24 @@ def run_ours(args, w):
     if scope == tbh.TB_SCOPE_LAYER:                          # the head-less predictor: one importance query per layer
         qi = qi[:, :, :1].contiguous()
     out = torch.empty(w.n_layers, w.batch, w.n_q_heads, w.head_dim, device="cuda")
+    # end-to-end leg: two sets of device buffers, so that a step's inputs arrive while the step before it computes
+    bufs = [(q, qi, out), (q.clone(), qi.clone(), torch.empty_like(out))]
     q_host, qi_host = q.cpu().pin_memory(), qi.cpu().pin_memory()
     out_host = torch.empty_like(out, device="cpu").pin_memory()
 
     groups = [(l, min(GROUP_LAYERS, w.n_layers - l)) for l in range(0, w.n_layers, GROUP_LAYERS)]
     sel_bytes, att_bytes = [], []
 
-    def step_launches(record=False):
+    def step_launches(record=False, b=0):
         # model-faithful schedule: at each producer the selections of its consumer layers, then
         # attention layer by layer
+        q_, qi_, out_ = bufs[b]
         for (l0, n) in groups:
-            ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p)
+            ctx.select_topk(l0, n, None, w.batch, qi_[l0:l0 + n], p)
             if record:
                 sel_bytes.append(ctx.last_step_bytes())
             for l in range(l0, l0 + n):
-                ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l])
+                ctx.sparse_decode_attention(l, 1, None, w.batch, q_[l], p, out_[l])
                 if record:
                     att_bytes.append(ctx.last_step_bytes())
 
@@ -267,8 +286,7 @@ def run_ours(args, w):
             for _ in range(args.warmup + args.steps):
                 step_launches()
             torch.cuda.synchronize()
-            print(json.dumps({"profile_run": w.name, "layers": w.n_layers, "launches_per_step": int(launches_per_step)}))
-            return
+            return {"profile_run": w.name, "layers": w.n_layers, "launches_per_step": int(launches_per_step)}
 
         def capture(fn):
             g = torch.cuda.CUDAGraph()
@@ -276,78 +294,123 @@ def run_ours(args, w):
                 fn()
             return g
 
-        g_step = capture(step_launches)
+        g_step = [capture(lambda: step_launches(b=0)), capture(lambda: step_launches(b=1))]
         g_sel = capture(lambda: [ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p) for (l0, n) in groups])
         g_att = capture(lambda: [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)])
 
-        def timed(fn, steps, warmup, sampler=None):
+        def timed(fn, steps, warmup, sampler=None, min_ms=300.0, stats=None, tail=None):
+            """K steps between two events on the launching stream (barrier + synchronise on both sides),
+            max over ranks; repeated until min_ms of device time have been timed.  Returns the median
+            repeat in ms per step; `stats` receives min / max / repeats."""
             for _ in range(warmup):
                 fn()
-            stream.synchronize()
-            if world > 1:
-                dist.barrier()
             torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             if sampler:
                 sampler.start()
-            e0.record(stream)
-            for _ in range(steps):
-                fn()
-            e1.record(stream)
-            if sampler:
-                while not e1.query():
-                    time.sleep(0.002)
-            torch.cuda.synchronize()
+            reps, total = [], 0.0
+            while True:
+                if world > 1:
+                    dist.barrier()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(steps):
+                    fn()
+                if tail:
+                    tail()                                  # joins work on other streams to the launching stream
+                e1.record(stream)
+                if sampler:
+                    while not e1.query():
+                        time.sleep(0.002)
+                torch.cuda.synchronize()
+                if world > 1:
+                    dist.barrier()
+                ms = max_over_ranks(e0.elapsed_time(e1), "cuda")       # the same number on every rank: a common exit
+                reps.append(ms / steps)
+                total += ms
+                if total >= min_ms or len(reps) >= 400:
+                    break
             if sampler:
                 sampler.sample()
                 sampler.stop_flag = True
-            if world > 1:
-                dist.barrier()
-            return max_over_ranks(e0.elapsed_time(e1), "cuda") / steps
+            if stats is not None:
+                stats.update({"min": float(np.min(reps)), "max": float(np.max(reps)), "repeats": len(reps)})
+            return float(np.median(reps))
 
         sampler = ClockSampler(local)
-        ms_step = timed(g_step.replay, args.steps, args.warmup, sampler)
+        step_stats = {}
+        ms_step = timed(g_step[0].replay, args.steps, args.warmup, sampler, stats=step_stats)
+
+        # End to end through the public API: every step copies its queries and importance queries in from
+        # page-locked host memory and its outputs back.  The copies run on two copy streams and the steps
+        # alternate between two sets of device buffers, so step i+1's inputs cross the link while step i
+        # computes and step i's outputs go back while step i+1 computes; events keep every buffer's
+        # producer and consumer in order.
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_done = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+        counter = [0]
 
         def e2e_step():
-            q.copy_(q_host, non_blocking=True)
-            qi.copy_(qi_host, non_blocking=True)
-            g_step.replay()
-            out_host.copy_(out, non_blocking=True)
+            b = counter[0] & 1
+            counter[0] += 1
+            q_, qi_, out_ = bufs[b]
+            s_in.wait_event(ev_done[b])                     # the step that last read this set is through
+            with torch.cuda.stream(s_in):
+                q_.copy_(q_host, non_blocking=True)
+                qi_.copy_(qi_host, non_blocking=True)
+                ev_in[b].record(s_in)
+            stream.wait_event(ev_in[b])
+            stream.wait_event(ev_out[b])                    # this set's previous outputs have left
+            g_step[b].replay()
+            ev_done[b].record(stream)
+            s_out.wait_event(ev_done[b])
+            with torch.cuda.stream(s_out):
+                out_host.copy_(out_, non_blocking=True)
+                ev_out[b].record(s_out)
 
-        ms_e2e = timed(e2e_step, args.steps, args.warmup)
-        ms_sel = timed(g_sel.replay, max(20, args.steps // 4), 3) / len(groups)
-        ms_att = timed(g_att.replay, max(20, args.steps // 4), 3) / w.n_layers
-        # Upper bound, not the method's schedule: the importance queries of all layers at once, so the
-        # selection runs as one call over every layer (many problems per launch) before the attentions.
+        def e2e_region_end():
+            stream.wait_event(ev_out[0])
+            stream.wait_event(ev_out[1])
+
+        ms_e2e = timed(e2e_step, args.steps, args.warmup, tail=e2e_region_end)
+        kstats_s, kstats_a = {}, {}
+        ms_sel = timed(g_sel.replay, max(20, args.steps // 4), 3, min_ms=100.0, stats=kstats_s) / len(groups)
+        ms_att = timed(g_att.replay, max(20, args.steps // 4), 3, min_ms=100.0, stats=kstats_a) / w.n_layers
         offload_info = None
         if args.offload_kv:
             # the comparison the paper draws for offloaded KV: the same step attending to every cached token
             p_dense = tbh.select_params(-1)
             g_dense = capture(lambda: [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p_dense, out[l]) for l in range(w.n_layers)])
-            ms_dense = timed(g_dense.replay, 3, 1)
+            ms_dense = timed(g_dense.replay, 3, 1, min_ms=0.0)
             dense_bytes = float(sum(w.lengths)) * w.n_layers * w.n_kv_heads * 2 * w.head_dim * (2 if w.dtype == wl.BF16 else 4)
             offload_info = {"kv_placement": "page-locked host memory, rows fetched by the attention kernel over the host link",
                             "dense_step_us": ms_dense * 1e3, "dense_link_gbs": dense_bytes / (ms_dense * 1e-3) / 1e9,
                             "sparse_link_gbs": float(np.sum(att_bytes)) / (ms_step * 1e-3) / 1e9,
                             "sparse_speedup_over_dense": ms_dense / ms_step}
-        g_all = capture(lambda: (ctx.select_topk(0, w.n_layers, None, w.batch, qi, p),
-                                 [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)]))
-        ms_all = timed(g_all.replay, max(20, args.steps // 4), 3)
-        # The step before the path, reported beside it (not inside the timed step): the importance-query
-        # predictor of one producer layer, 8B-shaped (model dim 4096, hidden 512), random weights; 16 weight
-        # sets are cycled so that every call reads its 8 MB from HBM, not from L2.
-        E, HID, n_sets = 4096, 512, 16
-        n_out = GROUP_LAYERS * w.n_q_heads * w.imp_dim
-        pw = [(torch.randn(E, generator=gen, device="cuda").to(dt), torch.randn(E, generator=gen, device="cuda").to(dt),
-               (torch.randn(HID, E, generator=gen, device="cuda") * E ** -0.5).to(dt),
-               (torch.randn(n_out, HID, generator=gen, device="cuda") * HID ** -0.5).to(dt)) for _ in range(n_sets)]
-        hs = torch.randn(w.batch, E, generator=gen, device="cuda").to(dt)
-        p_scratch = torch.empty(w.batch * HID, device="cuda")
-        p_out = torch.empty(GROUP_LAYERS, w.batch, w.n_q_heads, w.imp_dim, device="cuda")
-        g_pred = capture(lambda: [tbh.predict_importance_queries(hs, a, b, w1, w2, w.dtype, w.n_q_heads, GROUP_LAYERS, w.imp_dim,
-                                                                 p_scratch, p_out, stream=stream) for (a, b, w1, w2) in pw])
-        ms_pred = timed(g_pred.replay, 20, 3) / n_sets
-        pred_bytes = (HID * E + n_out * HID + 2 * E + w.batch * E) * (2 if w.dtype == wl.BF16 else 4)
+        ms_all = ms_pred = pred_bytes = None
+        if not brief:
+            # Upper bound, not the method's schedule: the importance queries of all layers at once, so the
+            # selection runs as one call over every layer (many problems per launch) before the attentions.
+            g_all = capture(lambda: (ctx.select_topk(0, w.n_layers, None, w.batch, qi, p),
+                                     [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l]) for l in range(w.n_layers)]))
+            ms_all = timed(g_all.replay, max(20, args.steps // 4), 3, min_ms=100.0)
+            # The step before the path, reported beside it (not inside the timed step): the importance-query
+            # predictor of one producer layer, 8B-shaped (model dim 4096, hidden 512), random weights; 16 weight
+            # sets are cycled so that every call reads its 8 MB from HBM, not from L2.
+            E, HID, n_sets = 4096, 512, 16
+            n_out = GROUP_LAYERS * w.n_q_heads * w.imp_dim
+            pw = [(torch.randn(E, generator=gen, device="cuda").to(dt), torch.randn(E, generator=gen, device="cuda").to(dt),
+                   (torch.randn(HID, E, generator=gen, device="cuda") * E ** -0.5).to(dt),
+                   (torch.randn(n_out, HID, generator=gen, device="cuda") * HID ** -0.5).to(dt)) for _ in range(n_sets)]
+            hs = torch.randn(w.batch, E, generator=gen, device="cuda").to(dt)
+            p_scratch = torch.empty(w.batch * HID, device="cuda")
+            p_out = torch.empty(GROUP_LAYERS, w.batch, w.n_q_heads, w.imp_dim, device="cuda")
+            g_pred = capture(lambda: [tbh.predict_importance_queries(hs, a, b, w1, w2, w.dtype, w.n_q_heads, GROUP_LAYERS, w.imp_dim,
+                                                                     p_scratch, p_out, stream=stream) for (a, b, w1, w2) in pw])
+            ms_pred = timed(g_pred.replay, 20, 3, min_ms=50.0) / n_sets
+            pred_bytes = (HID * E + n_out * HID + 2 * E + w.batch * E) * (2 if w.dtype == wl.BF16 else 4)
         assert ctx.get_status(stream) == 0, "device status set during the timed region"
 
     peak, peak_kind = measured_peaks()
@@ -358,70 +421,68 @@ def run_ours(args, w):
     achieved = dom[1] / (dom[2] * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "warmup": args.warmup, "ms_per_step": ms_step, "us_per_step": ms_step * 1e3,
+        "us_per_step_min": step_stats["min"] * 1e3, "us_per_step_max": step_stats["max"] * 1e3, "timed_repeats": step_stats["repeats"],
+        "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": storage_name(w), "data": "synthetic",
         "config": {"workload": w.name + ("+offloaded_kv" if args.offload_kv else "") +
                    ("+lists_per_" + args.list_scope if args.list_scope != "kv_head" else ""), "layers": w.n_layers, "batch_per_gpu": w.batch,
                    "q_heads": w.n_q_heads,
                    "kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "imp_dim": w.imp_dim,
-                   "kv_storage": "bf16" if w.dtype == wl.BF16 else "f32", "context": w.lengths if len(set(w.lengths)) > 1 else w.lengths[0],
+                   "kv_storage": storage_name(w), "accumulation": "f32", "context": w.lengths if len(set(w.lengths)) > 1 else w.lengths[0],
                    "budget": w.budget, "sinks": w.sinks, "recent": w.recent, "radius": w.radius, "interval": w.interval,
                    "schedule": "score+select per %d layers, attention per layer, CUDA-graph replay" % GROUP_LAYERS,
+                   "timing": "median of %d repeats of %d steps (>= 0.3 s of device time)" % (step_stats["repeats"], args.steps),
                    "l2": "inputs larger than L2: %.0f MB touched per step" % (step_bytes / 1e6)},
         "step_hbm_gbs": step_bytes / (ms_step * 1e-3) / 1e9, "step_bytes": step_bytes,
         "step_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "step_frac_of_nominal_8tbs": step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0,
         "gpu_launches": int(launches_per_step * args.steps),
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
                 "h2d_bytes_per_step": q_host.numel() * q_host.element_size() + qi_host.numel() * 4,
-                "d2h_bytes_per_step": out_host.numel() * 4},
+                "d2h_bytes_per_step": out_host.numel() * 4,
+                "how": "copies on two copy streams, two sets of device buffers: a step's copies overlap its neighbours' compute"},
         "roofline": {"bound": "hbm", "kernel": dom[0], "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom[0])),
                      "bytes_per_launch": dom[1], "us_per_launch": dom[2] * 1e3},
         "kernels": {"select_kernel": {"us_per_launch": ms_sel * 1e3, "bytes_per_launch": sel_b,
-                                      "gbs": sel_b / (ms_sel * 1e-3) / 1e9, "launches_per_step": len(groups)},
+                                      "gbs": sel_b / (ms_sel * 1e-3) / 1e9, "frac": sel_b / (ms_sel * 1e-3) / 1e9 / peak,
+                                      "launches_per_step": len(groups)},
                     "attn_kernel": {"us_per_launch": ms_att * 1e3, "bytes_per_launch": att_b,
-                                    "gbs": att_b / (ms_att * 1e-3) / 1e9, "launches_per_step": w.n_layers}},
-        "upper_bound_all_layers_one_select_call": {"us_per_step": ms_all * 1e3,
-                                                    "step_frac_of_peak": step_bytes / (ms_all * 1e-3) / 1e9 / peak,
-                                                    "note": "selection for all layers in one call; needs every layer's importance "
-                                                            "query up front, which the per-producer schedule does not have"},
-        "predictor_forward": {"us_per_producer": ms_pred * 1e3, "bytes_per_producer": pred_bytes,
-                              "gbs": pred_bytes / (ms_pred * 1e-3) / 1e9, "producers_per_step": len(groups),
-                              "note": "importance-query MLP of one producer layer (two launches); the step before the path, "
-                                      "not part of the timed step"},
-        "offloaded_kv": offload_info,
+                                    "gbs": att_b / (ms_att * 1e-3) / 1e9, "frac": att_b / (ms_att * 1e-3) / 1e9 / peak,
+                                    "launches_per_step": w.n_layers}},
         "prefill_projection": proj_info,
         "clocks": sampler.summary(),
     }
-    if rank == 0:
-        if world == 1 and not args.no_cpu and args.list_scope == "kv_head":   # the oracle sample below is per KV head
-            leg = cpu_leg(w, args.cpu_layers, 3)
-            best = min(leg["times"])
-            line["cpu_baseline"] = {"value": w.batch / best, "unit": UNIT, "cores": leg["threads"], "kind": "oracle",
-                                    "sample": leg["sample"], "ms_per_step": best * 1e3}
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    if not brief:
+        line["upper_bound_all_layers_one_select_call"] = {
+            "us_per_step": ms_all * 1e3, "step_frac_of_peak": step_bytes / (ms_all * 1e-3) / 1e9 / peak,
+            "note": "selection for all layers in one call; needs every layer's importance query up front, which the "
+                    "per-producer schedule does not have"}
+        line["predictor_forward"] = {
+            "us_per_producer": ms_pred * 1e3, "bytes_per_producer": pred_bytes, "gbs": pred_bytes / (ms_pred * 1e-3) / 1e9,
+            "producers_per_step": len(groups), "step_incl_predictor_us": ms_step * 1e3 + len(groups) * ms_pred * 1e3,
+            "note": "importance-query MLP of one producer layer; the step before the path, timed alone and added to the "
+                    "step in step_incl_predictor_us"}
+        line["offloaded_kv"] = offload_info
+    del g_step, g_sel, g_att, ctx
+    torch.cuda.empty_cache()
+    return line
 
 
-def run_trajectory(args, w):
+def measure_trajectory(args, w):
     """Workloads that decode: every step appends one token per sequence and layer, keys are projected
     in deferred batches of `recent` tokens, the selection (with neighbour expansion) is refreshed every
     `interval` steps and reused in between, attention runs every step.  Lengths change each step, so
     the launches are issued directly (kernel parameters carry the lengths); a step's GPU time is
-    milliseconds, far above the launch cost."""
+    milliseconds, far above the launch cost.  Returns the JSON line as a dict."""
     import torch
     import torch.distributed as dist
     from paper_2503_07518_b200 import binding as tbh
     from paper_2503_07518_b200 import build
     build.build()
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    world, rank, local = dist_env(torch, dist)
     P, Wn = w.interval, w.recent
     steps = max(P, args.steps // P * P)                      # whole refresh periods
     warm = max(P, (args.warmup + P - 1) // P * P)
@@ -444,6 +505,11 @@ def run_trajectory(args, w):
     proj = list(w.lengths)                                    # projected length per sequence (same in every layer)
     ones = [1] * w.batch
     bytes_sel, bytes_att = [0.0], [0.0]
+    # the lists' realised lengths: copied out at every refresh (a copy kernel per producer group inside the timed
+    # region), read back after the run, so that the attention bytes are what was gathered, not the (2r+1) B bound
+    n_refresh_max = total // P + 2
+    cnt_log = torch.zeros(n_refresh_max, w.n_layers, w.batch, w.n_kv_heads, dtype=torch.int32, device="cuda")
+    es = 2 if w.dtype == wl.BF16 else 4
 
     def step(t):
         p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode, P, t)
@@ -453,12 +519,12 @@ def run_trajectory(args, w):
                 ctx.append_kv(l, 1, None, ones, k_new[l], v_new[l])
                 if refresh and t > 0:                         # the window wrapped: project its tokens in one batch
                     ctx.project_keys(l, 1, None, proj, [x + Wn for x in proj])
-            ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p)   # launches only on refresh steps
+            # launches only on refresh steps
+            ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p, None, cnt_log[t // P, l0:l0 + n] if refresh else None)
             if refresh:
                 bytes_sel[0] += ctx.last_step_bytes()
             for l in range(l0, l0 + n):
                 ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l])
-                bytes_att[0] += ctx.last_step_bytes()
         if refresh and t > 0:
             for b in range(w.batch):
                 proj[b] += Wn
@@ -475,6 +541,7 @@ def run_trajectory(args, w):
         if world > 1:
             dist.barrier()
         bytes_sel[0] = bytes_att[0] = 0.0
+        t_first = t
         n0 = ctx.launch_count()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         sampler.start()
@@ -493,8 +560,16 @@ def run_trajectory(args, w):
         ms_step = max_over_ranks(ev[0].elapsed_time(ev[-1]), "cuda") / steps
         refresh_ms = float(np.mean(per_step[0::P]))
         reuse_ms = float(np.mean([x for i, x in enumerate(per_step) if i % P]))
+        # rows gathered per timed step: sinks + the list stored at the step's last refresh + window, per KV head
+        cnt_host = cnt_log.cpu().numpy().astype(np.int64)
+        for ts in range(t_first, t_first + steps):
+            L_now = w.lengths[0] + ts + 1
+            rows = min(w.sinks, L_now) * cnt_host[ts // P].size + int(cnt_host[ts // P].sum()) + min(w.recent, L_now) * cnt_host[ts // P].size
+            bytes_att[0] += float(rows) * 2 * w.head_dim * es
         step_bytes = (bytes_sel[0] + bytes_att[0]) / steps
         att_bytes = bytes_att[0] / steps / w.n_layers
+        bound_rows = (w.sinks + ((2 * w.radius + 1) if w.nmode == 0 else (1 + w.radius)) * w.budget + w.recent) * w.batch * w.n_kv_heads
+        att_bytes_bound = float(bound_rows) * 2 * w.head_dim * es
         sel_bytes = bytes_sel[0] / max(1, steps // P) / len(groups)
         # end to end: the step's new K/V rows and queries come from pinned host memory, outputs go back
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -530,14 +605,16 @@ def run_trajectory(args, w):
     line = {
         "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
         "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": storage_name(w), "data": "synthetic",
         "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "context": w.lengths[0], "budget": w.budget,
                    "recent": w.recent, "radius": w.radius, "neighbor_mode": "dilate" if w.nmode == 0 else "cluster",
                    "interval": P, "schedule": "per layer: append, (deferred projection), attention; select+expand per 4 layers on "
                    "refresh steps; direct launches", "l2": "inputs larger than L2: %.0f MB touched per step" % (step_bytes / 1e6)},
         "refresh_step_us": refresh_ms * 1e3, "reuse_step_us": reuse_ms * 1e3,
         "step_hbm_gbs": step_bytes / (ms_step * 1e-3) / 1e9, "step_bytes": step_bytes,
-        "step_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak, "gpu_launches": int(launches),
+        "step_bytes_note": "realised: the stored lists' lengths read back after the run (upper bound per attention launch: %.1f MB)" % (att_bytes_bound / 1e6),
+        "step_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "step_frac_of_nominal_8tbs": step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0, "gpu_launches": int(launches),
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "us_per_step": ms_e2e * 1e3,
                 "h2d_bytes_per_step": sum(h.numel() * h.element_size() for h in host), "d2h_bytes_per_step": out_host.numel() * 4},
         "kernels": {"select_kernel+neighbor_kernel": {"us_per_launch": sel_ms * 1e3, "bytes_per_launch": sel_bytes,
@@ -550,10 +627,19 @@ def run_trajectory(args, w):
                      "bytes_per_launch": att_bytes, "us_per_launch": att_ms * 1e3},
         "clocks": sampler.summary(),
     }
-    if rank == 0:
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    del ctx
+    torch.cuda.empty_cache()
+    return line
+
+
+def brief_entry(line):
+    """What the default run's `workloads` block keeps of another workload's line."""
+    keep = ("us_per_step", "us_per_step_min", "us_per_step_max", "timed_repeats", "steps", "warmup", "value", "step_bytes",
+            "step_hbm_gbs", "step_frac_of_peak", "step_frac_of_nominal_8tbs", "refresh_step_us", "reuse_step_us", "roofline",
+            "kernels", "e2e", "clocks", "gpu_launches")
+    out = {k: line[k] for k in keep if k in line}
+    out["config"] = {k: line["config"][k] for k in ("workload", "layers", "batch_per_gpu", "context", "budget", "schedule") if k in line["config"]}
+    return out
 
 
 def main():
@@ -561,11 +647,14 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (default: the 32K Llama-3-8B-shaped decode)")
+    ap.add_argument("--config", type=int, default=0,
+                    help="workload 1..5; default: the 32K Llama-3-8B-shaped decode (2) as the line's value, plus a brief "
+                         "`workloads` block for 3, 4 and 5")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-layers", type=int, default=2, help="layers in the CPU oracle's sample")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="default run without the `workloads` block")
     ap.add_argument("--profile", action="store_true", help="only warm-up + steps of plain launches (for ncu)")
     ap.add_argument("--offload-kv", action="store_true",
                     help="K|V cache in page-locked host memory (selected rows cross the host link); also times the dense step")
@@ -576,7 +665,8 @@ def main():
     ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
                     help="neighbour rule of the interval workload (default: its own, +-r dilation)")
     args = ap.parse_args()
-    w = wl.workload(args.config)
+    default_run = args.config == 0
+    w = wl.workload(args.config or 2)
     if args.layers:
         w = w.scaled(n_layers=args.layers)
     if args.context:
@@ -585,15 +675,41 @@ def main():
         w = w.scaled(nmode=0 if args.neighbors == "dilate" else 1)
     if args.impl == "reference":
         run_reference(args, w)
-    else:
-        if args.warmup < 3:
-            args.warmup = 3
-        if w.decode_steps > 1:
-            if args.steps > w.decode_steps:
-                args.steps = w.decode_steps
-            run_trajectory(args, w)
-        else:
-            run_ours(args, w)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    def measure(wk, brief=False):
+        if wk.decode_steps > 1:
+            a2 = argparse.Namespace(**vars(args))
+            a2.steps = min(args.steps, wk.decode_steps if not brief else 10 * wk.interval)
+            return measure_trajectory(a2, wk)
+        return measure_static(args, wk, brief=brief)
+
+    line = measure(w)
+    world, rank = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0"))
+    if "profile_run" not in line:
+        extra = default_run and not args.no_extra and not args.profile and world == 1 and not args.offload_kv and \
+            args.list_scope == "kv_head" and not args.layers and not args.context
+        if extra:
+            line["workloads"] = {}
+            for cfg in (3, 4, 5):
+                wk = wl.workload(cfg)
+                if args.neighbors:
+                    wk = wk.scaled(nmode=0 if args.neighbors == "dilate" else 1) if cfg == 5 else wk
+                line["workloads"][wk.name] = brief_entry(measure(wk, brief=True))
+        if rank == 0 and world == 1 and not args.no_cpu and args.list_scope == "kv_head" and w.decode_steps <= 1:
+            leg = cpu_leg(w, args.cpu_layers, 3)                      # the oracle sample is per KV head
+            best = min(leg["times"])
+            one = cpu_leg(w, 1, 1, max_units=2, threads=1)            # and on one thread
+            line["cpu_baseline"] = {"value": w.batch / best, "unit": UNIT, "cores": leg["threads"], "kind": "oracle",
+                                    "sample": leg["sample"], "ms_per_step": best * 1e3,
+                                    "value_1_thread": w.batch / one["times"][0], "sample_1_thread": one["sample"]}
+    if rank == 0:
+        print(json.dumps(line))
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -131,7 +131,8 @@ int32_t tb_index_capacity(const tb_ctx* ctx);
  * (Sec. 3.1: learned matrix of the key-cache projection). */
 tb_status tb_set_projection(tb_ctx* ctx, int32_t layer, const void* W_dev, void* stream);
 
-/* Forget a sequence in every layer: length and projected length 0, stored selections dropped. */
+/* Forget a sequence in every layer: length and projected length 0 (host mirrors and device counters, the
+ * latter with a blocking clear: call it when no work on that sequence is in flight), stored selections dropped. */
 tb_status tb_reset_sequence(tb_ctx* ctx, int32_t seq);
 
 /* Host-side view of a sequence: tokens cached and tokens whose keys are projected. */
@@ -149,7 +150,9 @@ tb_status tb_append_kv(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, co
  * channel order for fp32 storage -- and one round-to-nearest-even to kv_dtype; a row's result does
  * not depend on which call or batch projected it).  Eager (one token) or deferred batches
  * (Sec. 3.3) are both just ranges.  Ranges must
- * lie inside the cached tokens and start at or before the sequence's projected length (no holes). */
+ * lie inside the cached tokens and start at or before the sequence's projected length (no holes).
+ * pos_begin == pos_end == NULL means "everything cached and not yet projected", [projected length, length) of
+ * every listed (layer, sequence), read on the device -- the form a captured graph can replay. */
 tb_status tb_project_keys(tb_ctx* ctx, int32_t layer_begin, int32_t layer_count, const int32_t* seq_ids,
                           const int32_t* pos_begin, const int32_t* pos_end, int32_t n_seq, void* stream);
 
@@ -263,6 +266,21 @@ tb_status tb_predict_importance_queries(const tb_predictor* p, const void* hidde
 /* Synchronise `stream`, return the device status word (TB_OK, TB_ERR_TIMEOUT or TB_ERR_BAD_INDEX)
  * in *device_status and clear it. */
 tb_status tb_get_status(tb_ctx* ctx, void* stream, int32_t* device_status);
+
+/* Where the kernels take the sequence lengths from (Sec. 3.3 / 3.4: the cache grows by a token every decode
+ * step and the window moves with it).  The context keeps the lengths twice: host mirrors, advanced when a
+ * call is made, which validate arguments; and device counters, advanced by the append and projection kernels
+ * themselves.  By default (on = 0) every launch carries the mirrors' values as kernel parameters: no dependent
+ * load at kernel start, but a captured CUDA graph then replays the lengths it was captured with.  With on = 1
+ * the kernels read the device counters, so a graph captured once replays a growing sequence: capture a
+ * decode step (append, projection with NULL ranges, selection, attention) and replay it every step.
+ * growth_reserve = how many tokens a sequence may grow beyond its mirror while graphs are replayed: grids and
+ * shared memory are sized for mirror + reserve.  While graphs replay the mirrors stand still; the checks
+ * that need true lengths then happen on the device (an append past max_seq_len is skipped and reported as
+ * TB_ERR_CAPACITY in the status word).  Call tb_sync_lengths before the next call that is not a replay. */
+tb_status tb_use_device_lengths(tb_ctx* ctx, int32_t on, int32_t growth_reserve);
+/* Synchronise `stream` and copy the device counters into the host mirrors (lengths and projected lengths). */
+tb_status tb_sync_lengths(tb_ctx* ctx, void* stream);
 
 /* Diagnostics of the bounded device waits (every wait of a kernel on a copy it requested polls at most
  * a fixed number of times -- seconds -- then the kernel records TB_ERR_TIMEOUT in the status word, stops

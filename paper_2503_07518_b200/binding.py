@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libtokenbutler.so")
 
 EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb_set_projection", "tb_reset_sequence",
            "tb_get_length", "tb_append_kv", "tb_project_keys", "tb_score_tokens", "tb_select_topk",
-           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_set_wait_diagnostics", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
+           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_set_wait_diagnostics", "tb_use_device_lengths", "tb_sync_lengths", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
 
 
 class tb_config(C.Structure):
@@ -84,6 +84,8 @@ def lib():
         L.tb_predict_importance_queries.argtypes = [vp, vp, i32, vp, vp, vp]
         L.tb_get_status.argtypes = [vp, vp, ip]
         L.tb_set_wait_diagnostics.argtypes = [vp, i32, i32]
+        L.tb_use_device_lengths.argtypes = [vp, i32, i32]
+        L.tb_sync_lengths.argtypes = [vp, vp]
         L.tb_last_step_bytes.argtypes = [vp]
         L.tb_launch_count.argtypes = [vp]
         L.tb_status_string.argtypes = [i32]
@@ -216,9 +218,17 @@ class Context:
         self._chk(lib().tb_append_kv(self.h, layer_begin, layer_count, _ints(seq_ids), _ints(n_new), len(n_new), _ptr(k),
                                      _ptr(v), _stream(stream)), "tb_append_kv")
 
-    def project_keys(self, layer_begin, layer_count, seq_ids, pos_begin, pos_end, stream=None):
+    def project_keys(self, layer_begin, layer_count, seq_ids, pos_begin, pos_end, stream=None, n_seq=None):
+        """pos_begin = pos_end = None: every listed sequence's unprojected tokens (n_seq says how many sequences)."""
+        n = len(pos_begin) if pos_begin is not None else n_seq
         self._chk(lib().tb_project_keys(self.h, layer_begin, layer_count, _ints(seq_ids), _ints(pos_begin), _ints(pos_end),
-                                        len(pos_begin), _stream(stream)), "tb_project_keys")
+                                        n, _stream(stream)), "tb_project_keys")
+
+    def use_device_lengths(self, on=True, growth_reserve=0):
+        self._chk(lib().tb_use_device_lengths(self.h, int(on), growth_reserve), "tb_use_device_lengths")
+
+    def sync_lengths(self, stream=None):
+        self._chk(lib().tb_sync_lengths(self.h, _stream(stream)), "tb_sync_lengths")
 
     def score_tokens(self, layer, seq_ids, n_seq, q_imp, scores, reduce=TB_GROUP_SUM, scale=1.0, stream=None):
         self._chk(lib().tb_score_tokens(self.h, layer, _ints(seq_ids), n_seq, _ptr(q_imp), reduce, scale, _ptr(scores),

@@ -16,7 +16,7 @@ int elem_size(int dtype) { return dtype == TB_BF16 ? 2 : 4; }
 
 struct Layout {
     size_t kv_bytes, kimp_bytes;
-    size_t off_W, off_idx, off_cnt, off_status, off_counter, state_bytes;
+    size_t off_W, off_idx, off_cnt, off_status, off_counter, off_len, off_len_proj, off_misc, state_bytes;
     size_t off_part_o, off_part_ml, off_sel_idx, off_sel_cnt, off_sel_keys, off_sel_bins, work_bytes;
     int idx_cap, sel_stride;
 };
@@ -63,6 +63,9 @@ void compute_layout(const tb_config* c, Layout* l) {
     l->off_cnt = o, o = align_up(o + units * 4, 256);
     l->off_status = o, o = align_up(o + 4, 256);
     l->off_counter = o, o = align_up(o + pairs * ha * 4, 256);
+    l->off_len = o, o = align_up(o + pairs * 4, 256);
+    l->off_len_proj = o, o = align_up(o + pairs * 4, 256);
+    l->off_misc = o, o = align_up(o + 8 * 4, 256);
     l->state_bytes = o;
     const size_t units_q = (size_t)c->n_layers * c->max_batch * c->n_q_heads;
     o = 0;
@@ -129,11 +132,20 @@ tb_status resolve_seqs(const tb_ctx* c, const int32_t* seq_ids, int n_seq, int* 
     return TB_OK;
 }
 
-void fill_table(const tb_ctx* c, UnitTable* ut, int lb, int lc, const int* seqs, int n_seq) {
+// Lengths of a launch's units: the host mirrors, or -- when the kernels read the device counters -- upper
+// bounds (mirror + declared growth) that the launchers size grids and shared memory with.
+void fill_table(const tb_ctx* c, UnitTable* ut, int lb, int lc, const int* seqs, int n_seq, bool projected = false) {
     ut->layer_begin = lb, ut->layer_count = lc, ut->n_seq = n_seq;
+    ut->use_dev_len = c->dev_lengths, ut->len_is_projected = projected;
+    ut->len_dev = c->st.len, ut->len_proj_dev = c->st.len_proj;
     for (int i = 0; i < n_seq; ++i) ut->seq_id[i] = seqs[i];
+    const std::vector<int>& src = projected ? c->len_proj : c->len;
     for (int l = 0; l < lc; ++l)
-        for (int i = 0; i < n_seq; ++i) ut->len[l * n_seq + i] = c->len[(size_t)(lb + l) * c->cfg.max_batch + seqs[i]];
+        for (int i = 0; i < n_seq; ++i) {
+            long long L = src[(size_t)(lb + l) * c->cfg.max_batch + seqs[i]];
+            if (c->dev_lengths) L = L + c->growth_reserve < c->cfg.max_seq_len ? L + c->growth_reserve : c->cfg.max_seq_len;
+            ut->len[l * n_seq + i] = (int)L;
+        }
 }
 
 int layers_per_launch(int n_seq) {
@@ -197,6 +209,9 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->st.cnt = (int32_t*)(sp + l.off_cnt);
     c->st.status = (int32_t*)(sp + l.off_status);
     c->st.attn_counter = (uint32_t*)(sp + l.off_counter);
+    c->st.len = (int32_t*)(sp + l.off_len);
+    c->st.len_proj = (int32_t*)(sp + l.off_len_proj);
+    c->st.misc_counter = (uint32_t*)(sp + l.off_misc);
     char* wp = (char*)workspace;
     c->wk.part_o = (float*)(wp + l.off_part_o);
     c->wk.part_ml = (float*)(wp + l.off_part_ml);
@@ -215,6 +230,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->len.assign(n, 0), c->len_proj.assign(n, 0), c->has_sel.assign(n, 0), c->sel_cnt.assign(n, -1);
     c->last_bytes = 0, c->launches = 0;
     c->wait_poll_limit = 0, c->drop_tile = -1;
+    c->dev_lengths = 0, c->growth_reserve = 0;
     c->last_cache_write = c->last_list_write = -4;
     c->tile_rows = 256;
     for (int i = 0; i < 17; ++i) c->attn_max_active[i] = 0;
@@ -251,6 +267,11 @@ tb_status tb_set_projection(tb_ctx* c, int32_t layer, const void* W_dev, void* s
 
 tb_status tb_reset_sequence(tb_ctx* c, int32_t seq) {
     if (!c || seq < 0 || seq >= c->cfg.max_batch) return TB_ERR_INVALID_ARG;
+    // the device counters of this sequence, one 4-byte entry per layer (a blocking strided clear)
+    const size_t pitch = (size_t)c->cfg.max_batch * 4;
+    if (cudaMemset2D(c->st.len + seq, pitch, 0, 4, c->cfg.n_layers) != cudaSuccess ||
+        cudaMemset2D(c->st.len_proj + seq, pitch, 0, 4, c->cfg.n_layers) != cudaSuccess)
+        return TB_ERR_CUDA;
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const size_t i = (size_t)l * c->cfg.max_batch + seq;
         c->len[i] = c->len_proj[i] = c->has_sel[i] = 0, c->sel_cnt[i] = -1;
@@ -302,16 +323,25 @@ tb_status tb_append_kv(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_ids
 
 tb_status tb_project_keys(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_ids, const int32_t* pos_begin,
                           const int32_t* pos_end, int32_t n_seq, void* stream) {
-    if (!c || !pos_begin || !pos_end || bad_layers(c, lb, lc)) return TB_ERR_INVALID_ARG;
+    if (!c || (pos_begin == nullptr) != (pos_end == nullptr) || bad_layers(c, lb, lc)) return TB_ERR_INVALID_ARG;
     int seqs[kMaxLaunchSeq];
     tb_status st = resolve_seqs(c, seq_ids, n_seq, seqs);
     if (st != TB_OK) return st;
+    const bool auto_range = pos_begin == nullptr;       // everything cached and not yet projected
+    int max_range = 0;
     for (int i = 0; i < n_seq; ++i) {
-        if (pos_begin[i] < 0 || pos_end[i] < pos_begin[i]) return TB_ERR_INVALID_ARG;
+        if (!auto_range && (pos_begin[i] < 0 || pos_end[i] < pos_begin[i])) return TB_ERR_INVALID_ARG;
         for (int l = lb; l < lb + lc; ++l) {
             const size_t u = (size_t)l * c->cfg.max_batch + seqs[i];
+            if (auto_range) {
+                int n = c->len[u] - c->len_proj[u] + (c->dev_lengths ? c->growth_reserve : 0);
+                if (n > c->cfg.max_seq_len) n = c->cfg.max_seq_len;
+                if (n > max_range) max_range = n;
+                continue;
+            }
             if (pos_end[i] > c->len[u]) return TB_ERR_INVALID_ARG;          // beyond the cached tokens
             if (pos_begin[i] > c->len_proj[u]) return TB_ERR_INVALID_ARG;   // would leave a hole
+            if (pos_end[i] - pos_begin[i] > max_range) max_range = pos_end[i] - pos_begin[i];
         }
     }
     const int step = layers_per_launch(n_seq);
@@ -319,14 +349,17 @@ tb_status tb_project_keys(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_
         const int n = l0 + step <= lb + lc ? step : lb + lc - l0;
         UnitTable ut;
         fill_table(c, &ut, l0, n, seqs, n_seq);
-        if (launch_project(c, ut, pos_begin, pos_end, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
-        c->last_cache_write = (long long)c->launches;
-        c->launches++;
+        if (max_range > 0) {
+            if (launch_project(c, ut, pos_begin, pos_end, max_range, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+            c->last_cache_write = (long long)c->launches;
+            c->launches++;
+        }
     }
     for (int l = lb; l < lb + lc; ++l)
         for (int i = 0; i < n_seq; ++i) {
             const size_t u = (size_t)l * c->cfg.max_batch + seqs[i];
-            if (pos_end[i] > c->len_proj[u]) c->len_proj[u] = pos_end[i];
+            const int end = auto_range ? c->len[u] : pos_end[i];
+            if (end > c->len_proj[u]) c->len_proj[u] = end;
         }
     return TB_OK;
 }
@@ -340,8 +373,7 @@ tb_status tb_score_tokens(tb_ctx* c, int32_t layer, const int32_t* seq_ids, int3
     tb_status st = resolve_seqs(c, seq_ids, n_seq, seqs);
     if (st != TB_OK) return st;
     UnitTable ut;
-    fill_table(c, &ut, layer, 1, seqs, n_seq);
-    for (int i = 0; i < n_seq; ++i) ut.len[i] = c->len_proj[(size_t)layer * c->cfg.max_batch + seqs[i]];   // projected tokens only
+    fill_table(c, &ut, layer, 1, seqs, n_seq, /*projected=*/true);   // projected tokens only
     if (launch_score(c, ut, q_imp, reduce, score_scale, scores, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     c->launches++;
     return TB_OK;
@@ -481,7 +513,7 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
         a.list_bound = bound;
         for (int l = 0; l < n; ++l)
             for (int i = 0; i < n_seq; ++i)
-                a.known_cnt[l * n_seq + i] = (dense || idx) ? -1 : c->sel_cnt[(size_t)(l0 + l) * mb + seqs[i]];
+                a.known_cnt[l * n_seq + i] = (dense || idx || c->dev_lengths) ? -1 : c->sel_cnt[(size_t)(l0 + l) * mb + seqs[i]];
         a.nsplit = 0;
         a.sm_scale = sm_scale > 0.f ? sm_scale : 1.0f / sqrtf((float)c->cfg.head_dim);
         a.early_ok = !idx && (long long)c->launches - c->last_cache_write >= 2 && (long long)c->launches - c->last_list_write >= 2;
@@ -499,6 +531,25 @@ tb_status tb_get_status(tb_ctx* c, void* stream, int32_t* device_status) {
     if (cudaMemsetAsync(c->st.status, 0, 4, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     *device_status = v;
+    return TB_OK;
+}
+
+tb_status tb_use_device_lengths(tb_ctx* c, int32_t on, int32_t growth_reserve) {
+    if (!c || growth_reserve < 0) return TB_ERR_INVALID_ARG;
+    c->dev_lengths = on ? 1 : 0;
+    c->growth_reserve = on ? growth_reserve : 0;
+    return TB_OK;
+}
+
+tb_status tb_sync_lengths(tb_ctx* c, void* stream) {
+    if (!c) return TB_ERR_INVALID_ARG;
+    const size_t n = (size_t)c->cfg.n_layers * c->cfg.max_batch;
+    std::vector<int32_t> a(n), b(n);
+    if (cudaMemcpyAsync(a.data(), c->st.len, n * 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess ||
+        cudaMemcpyAsync(b.data(), c->st.len_proj, n * 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess ||
+        cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess)
+        return TB_ERR_CUDA;
+    for (size_t i = 0; i < n; ++i) c->len[i] = a[i], c->len_proj[i] = b[i], c->sel_cnt[i] = -1;
     return TB_OK;
 }
 

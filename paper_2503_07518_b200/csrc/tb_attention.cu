@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int split = blockIdx.x, h = blockIdx.y;
     const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq;
-    const int L = ut.len[ll * ut.n_seq + s];
+    const int L = unit_len(gm, ut, ll, s);
     const int g = gm.ga;
     const AttnUnit au(gm, ut, ll, s, h);
     const int lu = au.lu;
@@ -385,7 +385,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const int gid = lane >> 2, tig = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y;
     const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq;
-    const int L = ut.len[ll * ut.n_seq + s];
+    const int L = unit_len(gm, ut, ll, s);
     const int g = gm.ga;
     const AttnUnit au(gm, ut, ll, s, h);
     const int lu = au.lu;
@@ -903,6 +903,7 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
     gm.max_batch = 1 << 20, gm.max_seq_len = max_seq_len, gm.idx_cap = idx_dev ? idx_stride : 0, gm.dtype = kv_dtype;
     UnitTable ut;
     ut.layer_begin = 0, ut.layer_count = 1, ut.n_seq = n_seq;
+    ut.use_dev_len = 0, ut.len_is_projected = 0, ut.len_dev = nullptr, ut.len_proj_dev = nullptr;   // lengths are the caller's
     int max_rows = 0;
     for (int i = 0; i < n_seq; ++i) {
         const int slot = seq_slots ? seq_slots[i] : i;

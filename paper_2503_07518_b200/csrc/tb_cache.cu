@@ -11,9 +11,12 @@ struct AppendTable {
 };
 
 // One thread per 16-byte chunk of a (token, head) K|V row pair.
+// The last block to finish advances the device length counters (read by every block of this launch at
+// its start, so they may only change once all have arrived).
 template <typename T>
 __global__ void append_kernel(Geom gm, UnitTable ut, AppendTable at, int total_new, const T* __restrict__ k_new,
-                              const T* __restrict__ v_new, T* __restrict__ kv) {
+                              const T* __restrict__ v_new, T* __restrict__ kv, int32_t* __restrict__ len_dev,
+                              uint32_t* __restrict__ counter, int32_t* __restrict__ status) {
     constexpr int kPer16 = Elem<T>::kPer16;
     const int chunks_per_row = gm.D / kPer16;          // 16-byte chunks in one K (or V) row
     const int chunks_per_pair = 2 * chunks_per_row;
@@ -31,13 +34,24 @@ __global__ void append_kernel(Geom gm, UnitTable ut, AppendTable at, int total_n
         int tok = (int)(th / gm.Hkv);                  // index into the concatenated new tokens
         int s = 0;
         while (s + 1 < ut.n_seq && at.tok_off[s + 1] <= tok) ++s;
-        int pos = ut.len[ll * ut.n_seq + s] + (tok - at.tok_off[s]);
+        const int base = unit_len(gm, ut, ll, s);
+        if (base + (at.tok_off[s + 1] - at.tok_off[s]) > gm.max_seq_len) continue;   // only a replayed graph gets here (reported below)
+        int pos = base + (tok - at.tok_off[s]);
         int is_v = chunk >= chunks_per_row;
         int c16 = is_v ? chunk - chunks_per_row : chunk;
         const T* src = (is_v ? v_new : k_new) + (((size_t)ll * total_new + tok) * gm.Hkv + h) * gm.D;
         size_t row = (((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h) * gm.max_seq_len + pos;
         T* dst = kv + row * 2 * gm.D + (size_t)is_v * gm.D;
         reinterpret_cast<uint4*>(dst)[c16] = reinterpret_cast<const uint4*>(src)[c16];
+    }
+    if (last_block_arrives(counter, gridDim.x * gridDim.y)) {
+        for (int i = threadIdx.x; i < ut.layer_count * ut.n_seq; i += blockDim.x) {
+            const int l2 = i / ut.n_seq, s2 = i % ut.n_seq;
+            const size_t pair = (size_t)(ut.layer_begin + l2) * gm.max_batch + ut.seq_id[s2];
+            const int base = unit_len(gm, ut, l2, s2), n = at.tok_off[s2 + 1] - at.tok_off[s2];
+            if (base + n > gm.max_seq_len) atomicExch(status, kStatusCapacity);
+            else len_dev[pair] = base + n;
+        }
     }
 }
 
@@ -60,24 +74,48 @@ cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new
     cfg.attrs = attr, cfg.numAttrs = 1;
     if (gm.dtype == TB_BF16)
         return cudaLaunchKernelEx(&cfg, append_kernel<__nv_bfloat16>, gm, ut, at, total_new, (const __nv_bfloat16*)k,
-                                  (const __nv_bfloat16*)v, (__nv_bfloat16*)c->kv);
-    return cudaLaunchKernelEx(&cfg, append_kernel<float>, gm, ut, at, total_new, (const float*)k, (const float*)v, (float*)c->kv);
+                                  (const __nv_bfloat16*)v, (__nv_bfloat16*)c->kv, c->st.len, c->st.misc_counter, c->st.status);
+    return cudaLaunchKernelEx(&cfg, append_kernel<float>, gm, ut, at, total_new, (const float*)k, (const float*)v, (float*)c->kv,
+                              c->st.len, c->st.misc_counter, c->st.status);
 }
 
 // ---------------------------------------------------------------------------------------------
 // K_imp[t][j] = round( sum_c K[t][c] * W[c][j] ), channels in ascending order, fp32 FMA chain.
 
 struct ProjectTable {
+    int auto_range;                  // 1: [projected length, length) of every (layer, sequence), from the device counters
     int pos_begin[kMaxLaunchSeq];
     int pos_end[kMaxLaunchSeq];
 };
+
+// Token range of a projection block's (layer, sequence).
+__device__ __forceinline__ void project_range(const Geom& gm, const UnitTable& ut, const ProjectTable& pt, int ll, int s, int& begin, int& end) {
+    if (pt.auto_range) {
+        const size_t pair = (size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s];
+        begin = ut.len_proj_dev[pair], end = ut.len_dev[pair];
+    } else {
+        begin = pt.pos_begin[s], end = pt.pos_end[s];
+    }
+}
+// The last block of a projection launch to finish advances the device counters of the projected lengths.
+__device__ __forceinline__ void project_finish(const Geom& gm, const UnitTable& ut, const ProjectTable& pt, int32_t* len_proj_dev,
+                                               uint32_t* counter) {
+    if (!last_block_arrives(counter, gridDim.x * gridDim.y * gridDim.z)) return;
+    for (int i = threadIdx.x; i < ut.layer_count * ut.n_seq; i += blockDim.x) {
+        int b, e;
+        project_range(gm, ut, pt, i / ut.n_seq, i % ut.n_seq, b, e);
+        const size_t pair = (size_t)(ut.layer_begin + i / ut.n_seq) * gm.max_batch + ut.seq_id[i % ut.n_seq];
+        if (e > len_proj_dev[pair]) len_proj_dev[pair] = e;
+    }
+}
 
 constexpr int kProjTokens = 32;   // tokens per block
 constexpr int kProjThreads = 128; // 4 threads per token, each owning dp/4 outputs
 
 template <typename T, int DP>
 __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTable ut, ProjectTable pt, const T* __restrict__ kv,
-                                                               const T* __restrict__ Wall, T* __restrict__ kimp) {
+                                                               const T* __restrict__ Wall, T* __restrict__ kimp,
+                                                               int32_t* __restrict__ len_proj_dev, uint32_t* __restrict__ counter) {
     constexpr int D = 128;
     constexpr int JPT = DP / 4;                       // outputs per thread
     __shared__ float Ws[D * DP];
@@ -85,10 +123,10 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTabl
 
     const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq, h = blockIdx.y;
     const int layer = ut.layer_begin + ll;
-    const int t0 = pt.pos_begin[s] + blockIdx.x * kProjTokens;
-    const int t_end = pt.pos_end[s];
-    if (t0 >= t_end) return;
-    const int nt = min(kProjTokens, t_end - t0);
+    int r_begin, t_end;
+    project_range(gm, ut, pt, ll, s, r_begin, t_end);
+    const int t0 = r_begin + blockIdx.x * kProjTokens;
+    const int nt = max(0, min(kProjTokens, t_end - t0));               // 0: nothing for this block (it still reports in at the end)
 
     // One key stream per KV head, or (one list per layer) a single stream that sums the heads'
     // projections: K_imp[t] = sum_h K[t][h] . W[h], heads in ascending order on one fp32 chain.
@@ -103,6 +141,7 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTabl
         const T* W = Wall + ((size_t)layer * gm.Hkv + hk) * D * DP;
         if (hs) __syncthreads();
         for (int i = threadIdx.x; i < D * DP; i += kProjThreads) Ws[i] = Elem<T>::to_f32(W[i]);
+        if (nt == 0) break;
         const size_t krow0 = (pair * gm.Hkv + hk) * gm.max_seq_len + t0;
         for (int i = threadIdx.x; i < nt * D; i += kProjThreads) {
             int tt = i / D, ch = i % D;
@@ -118,11 +157,13 @@ __global__ void __launch_bounds__(kProjThreads) project_kernel(Geom gm, UnitTabl
             }
         }
     }
-    if (t >= nt) return;
-    const size_t row0 = (pair * gm.Hi + h) * gm.max_seq_len + t0;
-    T* dst = kimp + (row0 + t) * DP + jq * JPT;
+    if (t < nt) {
+        const size_t row0 = (pair * gm.Hi + h) * gm.max_seq_len + t0;
+        T* dst = kimp + (row0 + t) * DP + jq * JPT;
 #pragma unroll
-    for (int j = 0; j < JPT; ++j) dst[j] = Elem<T>::from_f32(acc[j]);
+        for (int j = 0; j < JPT; ++j) dst[j] = Elem<T>::from_f32(acc[j]);
+    }
+    project_finish(gm, ut, pt, len_proj_dev, counter);
 }
 
 // bf16 storage: the projection is the one dense contraction of the path ([tokens x 128] . [128 x d']
@@ -138,7 +179,8 @@ template <int DP>
 __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTable ut, ProjectTable pt,
                                                                  const __nv_bfloat16* __restrict__ kv,
                                                                  const __nv_bfloat16* __restrict__ Wall,
-                                                                 __nv_bfloat16* __restrict__ kimp) {
+                                                                 __nv_bfloat16* __restrict__ kimp, int32_t* __restrict__ len_proj_dev,
+                                                                 uint32_t* __restrict__ counter) {
     constexpr int D = 128;
     constexpr int kWPitch = DP * 2 + 16;  // bytes per W row (one channel, d' outputs) + pad
     constexpr int NT = DP / 8;            // 8-wide output tiles
@@ -148,9 +190,13 @@ __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTa
 
     const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq, h = blockIdx.y;
     const int layer = ut.layer_begin + ll;
-    const int t0 = pt.pos_begin[s] + blockIdx.x * kPmTokens;
-    const int t_end = pt.pos_end[s];
-    if (t0 >= t_end) return;
+    int r_begin, t_end;
+    project_range(gm, ut, pt, ll, s, r_begin, t_end);
+    const int t0 = r_begin + blockIdx.x * kPmTokens;
+    if (t0 >= t_end) {                                                 // nothing for this block: it only reports in
+        project_finish(gm, ut, pt, len_proj_dev, counter);
+        return;
+    }
     const int nt_valid = min(kPmTokens, t_end - t0);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gid = lane >> 2, tig = lane & 3;
@@ -232,15 +278,15 @@ __global__ void __launch_bounds__(kPmThreads) project_mma_kernel(Geom gm, UnitTa
             }
         }
     }
+    project_finish(gm, ut, pt, len_proj_dev, counter);
 }
 
-cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, cudaStream_t s) {
+cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, int max_range, cudaStream_t s) {
     ProjectTable pt;
-    int max_range = 0;
+    pt.auto_range = pos_begin == nullptr;
     for (int i = 0; i < ut.n_seq; ++i) {
-        pt.pos_begin[i] = pos_begin[i];
-        pt.pos_end[i] = pos_end[i];
-        if (pos_end[i] - pos_begin[i] > max_range) max_range = pos_end[i] - pos_begin[i];
+        pt.pos_begin[i] = pt.auto_range ? 0 : pos_begin[i];
+        pt.pos_end[i] = pt.auto_range ? 0 : pos_end[i];
     }
     if (max_range <= 0) return cudaSuccess;
     const Geom& gm = c->geom;
@@ -255,7 +301,7 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
                 cudaError_t e = cudaFuncSetAttribute(project_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 if (e != cudaSuccess) return e;
             }
-            project_mma_kernel<32><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp);
+            project_mma_kernel<32><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp, c->st.len_proj, c->st.misc_counter + 1);
         } else {
             const size_t smem = kPmTokens * kPmKPitch + 128 * (16 * 2 + 16);
             static unsigned char seen[64];
@@ -263,13 +309,13 @@ cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_
                 cudaError_t e = cudaFuncSetAttribute(project_mma_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
                 if (e != cudaSuccess) return e;
             }
-            project_mma_kernel<16><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp);
+            project_mma_kernel<16><<<grid_mma, kPmThreads, smem, s>>>(gm, ut, pt, kvp, wp, (__nv_bfloat16*)c->kimp, c->st.len_proj, c->st.misc_counter + 1);
         }
         return cudaGetLastError();
     }
     dim3 grid((max_range + kProjTokens - 1) / kProjTokens, gm.Hi, ut.layer_count * ut.n_seq);
 #define TB_PROJ(T, DP) \
-    project_kernel<T, DP><<<grid, kProjThreads, 0, s>>>(gm, ut, pt, (const T*)c->kv, (const T*)c->st.W, (T*)c->kimp)
+    project_kernel<T, DP><<<grid, kProjThreads, 0, s>>>(gm, ut, pt, (const T*)c->kv, (const T*)c->st.W, (T*)c->kimp, c->st.len_proj, c->st.misc_counter + 1)
     if (gm.dp == 32) TB_PROJ(float, 32); else TB_PROJ(float, 16);
 #undef TB_PROJ
     return cudaGetLastError();

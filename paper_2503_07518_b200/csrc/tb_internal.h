@@ -31,8 +31,17 @@ struct Geom {
 };
 
 // Per-launch table of (layer-local, sequence) pairs: which cache slot and how many tokens.
+// Lengths come two ways.  By default they travel here, as kernel parameters copied from the host's
+// mirrors (no dependent load at kernel start; a captured CUDA graph then replays the lengths it was
+// captured with).  With use_dev_len the kernels read the context's device counters, which the append
+// and projection kernels advance themselves, so a captured graph replays a growing sequence; `len`
+// then holds upper bounds (length + the reserve the caller declared) that size grids and shared memory.
 struct UnitTable {
     int layer_begin, layer_count, n_seq;
+    int use_dev_len;            // 1: kernels read len_dev / len_proj_dev
+    int len_is_projected;       // 1: "length" means projected length (materialised scores cover projected tokens)
+    const int32_t* len_dev;     // [n_layers * max_batch] tokens cached
+    const int32_t* len_proj_dev;   // [n_layers * max_batch] tokens whose keys are projected
     int seq_id[kMaxLaunchSeq];
     int len[kMaxLaunchUnits];   // [layer_local * n_seq + s]
 };
@@ -71,7 +80,13 @@ struct AttnArgs {
     int known_cnt[kMaxLaunchUnits];
 };
 
+constexpr int kStatusCapacity = -3;      // device status: an append in a replayed graph ran past max_seq_len
+constexpr int kStatusUnprojected = -4;   // device status: a replayed selection found candidates that are not projected
+
 struct DevState {
+    int32_t* len;         // [n_layers * max_batch] device copies of the lengths, advanced by the append kernel
+    int32_t* len_proj;    // ... and of the projected lengths, advanced by the projection kernels
+    uint32_t* misc_counter;   // arrival counters of the append / projection kernels (self-resetting)
     void* W;              // [n_layers][Hkv][D][dp] kv_dtype
     int32_t* idx;         // [n_layers][max_batch][Hl][idx_cap]
     int32_t* cnt;         // [n_layers][max_batch][Hl]
@@ -106,6 +121,8 @@ struct tb_ctx {
     int tile_rows;                        // rows per TMA box of the score pass
     int sm_count;
     int attn_max_active[17];              // co-resident attention clusters per cluster size (0 = not asked yet)
+    int dev_lengths;                      // 1: kernels read the device counters (graph-replayable growth)
+    int growth_reserve;                   // tokens a sequence may grow beyond the host mirror while graphs are replayed
     int wait_poll_limit;                  // polls per bounded wait of the selection kernels; 0 = the default (seconds)
     int drop_tile;                        // diagnostics: tile whose copy the next single-block selection leaves out, -1 = none
     uint64_t last_bytes, launches;
@@ -115,6 +132,29 @@ struct tb_ctx {
 };
 
 namespace tb {
+
+#ifdef __CUDACC__
+// Tokens of launch unit (layer-local ll, sequence s): a kernel parameter, or the device counter.
+__device__ __forceinline__ int unit_len(const Geom& gm, const UnitTable& ut, int ll, int s) {
+    if (!ut.use_dev_len) return ut.len[ll * ut.n_seq + s];
+    const size_t pair = (size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s];
+    return ut.len_is_projected ? ut.len_proj_dev[pair] : ut.len_dev[pair];
+}
+// Last block of a grid to get here (after its global writes): true for exactly one block, which also
+// resets the counter for the next launch.  Called by all threads of the block.
+__device__ __forceinline__ bool last_block_arrives(uint32_t* counter, unsigned n_blocks) {
+    __shared__ int s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned prev = atomicAdd(counter, 1u);
+        s_last = prev == n_blocks - 1u;
+        if (s_last) *counter = 0u;
+    }
+    __syncthreads();
+    return s_last != 0;
+}
+#endif
 
 // Kernel attributes (dynamic shared-memory limit, non-portable cluster sizes) belong to a device's
 // context, so each launcher configures its kernels on first use per device.
@@ -129,7 +169,9 @@ inline bool first_use_on_this_device(unsigned char (&seen)[64]) {
 // tb_cache.cu
 cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new, const int* tok_off, int total_new,
                           const void* k, const void* v, cudaStream_t s);
-cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, cudaStream_t s);
+// pos_begin == nullptr: every listed sequence's unprojected tokens [projected length, length), taken from the
+// device counters; max_range then bounds the tokens of any one (layer, sequence)
+cudaError_t launch_project(const tb_ctx* c, const UnitTable& ut, const int* pos_begin, const int* pos_end, int max_range, cudaStream_t s);
 
 // tb_select.cu
 cudaError_t launch_score(const tb_ctx* c, const UnitTable& ut, const float* q_imp, int reduce, float scale, float* scores,

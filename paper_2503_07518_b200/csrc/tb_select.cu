@@ -210,11 +210,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
 
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
-    const int L = ut.len[ll * ut.n_seq + s];
+    const int L = unit_len(gm, ut, ll, s);
     const int lo = min(a.sinks, L);
     const int hi = max(lo, L - a.recent);
     const int ncand = hi - lo;
     const int k = min(a.budget, ncand);
+    check_candidates_projected(gm, ut, ll, s, hi, status);
     const size_t cu = list_unit(gm, ut, ll, s, h);
     const size_t dst_row = a.dst_is_state ? cu : (size_t)blockIdx.y;
     int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;

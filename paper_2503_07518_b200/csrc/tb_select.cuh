@@ -122,4 +122,13 @@ __device__ __forceinline__ size_t query_row(const Geom& gm, const UnitTable& ut,
     return ((size_t)(ll * ut.n_seq + s) * gm.Hl + h) * gm.gl;
 }
 
+// With device-resident lengths the host cannot check, at replay time, that every candidate has a projected
+// key: one thread per block does, and reports through the status word (the selection itself goes on).
+__device__ __forceinline__ void check_candidates_projected(const Geom& gm, const UnitTable& ut, int ll, int s, int hi, int32_t* status) {
+    if (ut.use_dev_len && threadIdx.x == 0) {
+        const size_t pair = (size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s];
+        if (ut.len_proj_dev[pair] < hi) atomicExch(status, kStatusUnprojected);
+    }
+}
+
 }  // namespace tb

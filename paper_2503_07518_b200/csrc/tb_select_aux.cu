@@ -13,7 +13,7 @@ __global__ void __launch_bounds__(256) score_kernel(Geom gm, UnitTable ut, const
     __shared__ __align__(16) float qs[kMaxGroup * 32];
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
-    const int L = ut.len[ll * ut.n_seq + s];
+    const int L = unit_len(gm, ut, ll, s);
     GroupScorer<T, DP, RED> scorer;
     scorer.load(q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, qs);
     if (RED != TB_GROUP_SUM) __syncthreads();
@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(kNbThreads) neighbor_kernel(Geom gm, UnitTable
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.x, ll, s, h);
-    const int L = ut.len[ll * ut.n_seq + s];
+    const int L = unit_len(gm, ut, ll, s);
     const int lo = min(a.sinks, L), hi = max(lo, L - a.recent);
     const int span = hi - lo;
     const int n_words = (span + 31) / 32;

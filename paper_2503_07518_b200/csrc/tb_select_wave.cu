@@ -480,11 +480,12 @@ __global__ void __launch_bounds__(kThreads, 4)
     const int tid = threadIdx.x, lane = tid & 31;
     const int pair = order.pair[blockIdx.x / gm.Hl], h = blockIdx.x % gm.Hl;
     const int ll = pair / ut.n_seq, s = pair % ut.n_seq;
-    const int L = ut.len[pair];
+    const int L = unit_len(gm, ut, ll, s);
     const int lo = min(a.sinks, L);
     const int hi = max(lo, L - a.recent);
     const int ncand = hi - lo;
     const int k = min(a.budget, ncand);
+    check_candidates_projected(gm, ut, ll, s, hi, status);
     const size_t cu = list_unit(gm, ut, ll, s, h);
     const size_t dst_row = a.dst_is_state ? cu : (size_t)pair * gm.Hl + h;
     int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;
@@ -750,8 +751,9 @@ __global__ void __launch_bounds__(kThreads, 2)
     const int tid = threadIdx.x, lane = tid & 31;
     int ll, s, h;
     decode_unit(gm, ut, blockIdx.y, ll, s, h);
-    const int L = ut.len[ll * ut.n_seq + s];
+    const int L = unit_len(gm, ut, ll, s);
     const int lo = min(a.sinks, L), ncand = max(lo, L - a.recent) - lo, k = min(a.budget, ncand);
+    check_candidates_projected(gm, ut, ll, s, lo + ncand, status);
     const size_t cu = list_unit(gm, ut, ll, s, h);
     const size_t dst_row = a.dst_is_state ? cu : (size_t)blockIdx.y;
     int32_t* idx_dst = (a.dst_is_state ? state_idx : a.idx_dst) + dst_row * a.idx_stride;

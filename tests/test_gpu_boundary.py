@@ -109,3 +109,100 @@ def test_byte_counter_reproduces_the_papers_bandwidth_reduction(H):
     assert sparse == (S + B + W) * 8 * 2 * 128 * 2 == 8192 * 8 * 512
     assert dense == L * 8 * 512 and dense / sparse == 8.0
     assert ctx.get_status() == 0
+
+
+def test_captured_graphs_replay_a_growing_sequence(H):
+    """Device-resident lengths: two CUDA graphs, captured once -- a refresh step (append, projection of the
+    unprojected tokens, selection with neighbours, attention) and a reuse step (append, attention from the stale
+    lists) -- are replayed over a decode trajectory.  Every replay must see the sequence one token longer:
+    lists and attention are checked against the oracle at each step's true length, the projected keys
+    against the oracle's projection, and the device counters against the lengths at the end."""
+    b_ = tb()
+    P, Wn, steps = 4, 8, 11
+    w = wl.workload(5, n_layers=2, batch=2, n_q_heads=8, n_kv_heads=2, lengths=[1200, 700], budget=90, recent=Wn,
+                    radius=1, interval=P, decode_steps=steps)
+    case = H.Case(w, extra_len=steps + 2)
+    ctx = case.ctx
+    ctx.use_device_lengths(True, growth_reserve=steps + 2)
+    dt = torch.bfloat16
+    k_new = torch.zeros(w.n_layers, w.batch, w.n_kv_heads, w.head_dim, dtype=dt, device="cuda")
+    v_new = torch.zeros_like(k_new)
+    q_d = torch.zeros(w.n_layers, w.batch, w.n_q_heads, w.head_dim, dtype=dt, device="cuda")
+    qi_d = torch.zeros(w.n_layers, w.batch, w.n_q_heads, w.imp_dim, device="cuda")
+    out = torch.zeros(w.n_layers, w.batch, w.n_q_heads, w.head_dim, device="cuda")
+    cap = ctx.index_capacity
+    idx = torch.zeros(w.n_layers, w.batch, w.n_kv_heads, cap, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(w.n_layers, w.batch, w.n_kv_heads, dtype=torch.int32, device="cuda")
+    p_refresh = b_.select_params(w.budget, 0, Wn, 1, 0, P, 0)
+    p_reuse = b_.select_params(w.budget, 0, Wn, 1, 0, P, 1)
+
+    def one_step(p):
+        for l in range(w.n_layers):
+            ctx.append_kv(l, 1, None, [1] * w.batch, k_new[l], v_new[l])
+        if p.step % P == 0:
+            ctx.project_keys(0, w.n_layers, None, None, None, n_seq=w.batch)
+        ctx.select_topk(0, w.n_layers, None, w.batch, qi_d, p, idx, cnt)
+        for l in range(w.n_layers):
+            ctx.sparse_decode_attention(l, 1, None, w.batch, q_d[l], p, out[l])
+
+    stream = torch.cuda.Stream()
+    graphs = {}
+    with torch.cuda.stream(stream):
+        for name, p in (("refresh", p_refresh), ("reuse", p_reuse)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                one_step(p)
+            graphs[name] = g
+        ctx.sync_lengths(stream)                       # capturing advanced only the host mirrors: back to the truth
+        assert [ctx.get_length(0, b) for b in range(w.batch)] == [(1200, 1200), (700, 700)]
+        stored = None
+        for t in range(steps):
+            # this step's inputs, and the host copies of the rows the graph will append
+            Ks = [[wl.gen_KV(w, l, b, n_tokens=1, start=t + 1) for b in range(w.batch)] for l in range(w.n_layers)]
+            for l in range(w.n_layers):
+                for b in range(w.batch):
+                    K, V = Ks[l][b]
+                    case.K[l][b][:, case.cur[b]] = K[:, 0]
+                    case.V[l][b][:, case.cur[b]] = V[:, 0]
+                    k_new[l, b] = H.to_dev(K[:, 0], w.dtype)
+                    v_new[l, b] = H.to_dev(V[:, 0], w.dtype)
+            case.cur = [c + 1 for c in case.cur]
+            q, qi = H.queries(w, t)
+            q_d.copy_(H.to_dev(q, w.dtype))
+            qi_d.copy_(torch.from_numpy(qi).cuda())
+            refresh = H.orc.is_prediction_step(t, P)
+            graphs["refresh" if refresh else "reuse"].replay()
+            torch.cuda.synchronize()
+            assert ctx.get_status(stream) == 0
+            p = b_.select_params(w.budget, 0, Wn, 1, 0, P, t)
+            idx_h, cnt_h, out_h = idx.cpu().numpy(), cnt.cpu().numpy(), out.cpu().numpy()
+            lists = [[[idx_h[l, b, h, :cnt_h[l, b, h]] for h in range(2)] for b in range(w.batch)] for l in range(w.n_layers)]
+            if refresh:
+                for l in range(w.n_layers):
+                    for b in range(w.batch):
+                        L = case.cur[b]
+                        dev = H.to_host(ctx.kimp[l, b, :, :L], w.dtype)           # the device's own projected keys
+                        for h in range(2):
+                            # newly projected rows obey the projection's error bound
+                            lo_new = case.proj[b]
+                            ref = H.orc.project_keys(np.ascontiguousarray(case.K[l][b][h, lo_new:L]), np.ascontiguousarray(case.W[l][h]), w.dtype)
+                            assert H.projection_excess(dev[h, lo_new:L], ref, case.K[l][b][h, lo_new:L], case.W[l][h], w.dtype) <= 1.0
+                            s = H.orc.score(qi[l, b][h * 4:(h + 1) * 4], np.ascontiguousarray(dev[h]), w.dtype)
+                            base = H.orc.select(s, 0, Wn, w.budget)
+                            lo, hi = H.orc.candidate_range(L, 0, Wn)
+                            assert np.array_equal(lists[l][b][h], H.orc.neighbors(base, 1, 0, lo, hi)), (t, l, b, h)
+                case.proj = list(case.cur)
+                stored = [[[x.copy() for x in lb_] for lb_ in ll_] for ll_ in lists]
+            else:
+                assert all(np.array_equal(lists[l][b][h], stored[l][b][h]) for l in range(2) for b in range(2) for h in range(2))
+            for l in range(w.n_layers):
+                for b in range(w.batch):
+                    for h in range(2):
+                        ref, _ = case.oracle_attention(l, b, h, q[l, b], stored[l][b][h], p)
+                        assert np.abs(out_h[l, b, h * 4:(h + 1) * 4] - ref).max() <= 2e-3, (t, l, b, h)
+        ctx.sync_lengths(stream)
+        assert [ctx.get_length(1, b) for b in range(w.batch)] == [(1200 + steps, 1200 + 9), (700 + steps, 700 + 9)]   # last refresh at t = 8
+    ctx.use_device_lengths(False)
+    # back on host-carried lengths the same context goes on as usual
+    full = H.gpu_select(case, H.queries(w, 99)[1], b_.select_params(w.budget, 0, Wn, 0))
+    assert ctx.get_status() == 0 and len(full[0][0][0]) == w.budget

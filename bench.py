@@ -486,7 +486,7 @@ def measure_trajectory(args, w):
     P, Wn = w.interval, w.recent
     steps = max(P, args.steps // P * P)                      # whole refresh periods
     warm = max(P, (args.warmup + P - 1) // P * P)
-    total = warm + 2 * steps                                  # device-timed pass + end-to-end pass
+    total = 2 * warm + 3 * steps                              # device-timed pass + end-to-end pass + graph-replay pass
     ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + total + Wn,
                       w.budget, w.radius, device=local)
     fill_caches(ctx, w, torch, tbh)
@@ -600,6 +600,46 @@ def measure_trajectory(args, w):
         sel_ms = alone(lambda: [ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], pr) for (l0, n) in groups], 3) / len(groups)
         assert ctx.get_status(stream) == 0, "device status set during the timed region"
 
+        # The same trajectory as two CUDA graphs captured once (refresh step / reuse step) and replayed: the
+        # kernels read the lengths from the device counters that the append and projection kernels advance.
+        ctx.use_device_lengths(True, growth_reserve=warm + steps + 2 * P)
+        cnt_g = torch.zeros(w.n_layers, w.batch, w.n_kv_heads, dtype=torch.int32, device="cuda")
+
+        def graph_step(refresh):
+            p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode, P, 0 if refresh else 1)
+            for (l0, n) in groups:
+                for l in range(l0, l0 + n):
+                    ctx.append_kv(l, 1, None, ones, k_new[l], v_new[l])
+                    if refresh:                               # the tokens that left the window since the last refresh
+                        ctx.project_keys(l, 1, None, None, None, n_seq=w.batch)
+                ctx.select_topk(l0, n, None, w.batch, qi[l0:l0 + n], p, None, cnt_g[l0:l0 + n] if refresh else None)
+                for l in range(l0, l0 + n):
+                    ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l])
+
+        graphs = {}
+        for refresh in (True, False):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                graph_step(refresh)
+            graphs[refresh] = g
+        ctx.sync_lengths(stream)                              # capturing moved only the host mirrors
+        for i in range(warm):
+            graphs[i % P == 0].replay()
+        torch.cuda.synchronize()
+        gv = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        gv[0].record(stream)
+        for i in range(steps):
+            graphs[i % P == 0].replay()
+            gv[i + 1].record(stream)
+        torch.cuda.synchronize()
+        assert ctx.get_status(stream) == 0, "device status set during the graph-replay pass"
+        g_per = [gv[i].elapsed_time(gv[i + 1]) for i in range(steps)]
+        ms_graph = max_over_ranks(gv[0].elapsed_time(gv[-1]), "cuda") / steps
+        graph_refresh_ms = float(np.mean(g_per[0::P]))
+        graph_reuse_ms = float(np.mean([x for i, x in enumerate(g_per) if i % P]))
+        ctx.sync_lengths(stream)
+        ctx.use_device_lengths(False)
+
     peak, peak_kind = measured_peaks()
     tokens = w.batch * world
     line = {
@@ -611,6 +651,10 @@ def measure_trajectory(args, w):
                    "interval": P, "schedule": "per layer: append, (deferred projection), attention; select+expand per 4 layers on "
                    "refresh steps; direct launches", "l2": "inputs larger than L2: %.0f MB touched per step" % (step_bytes / 1e6)},
         "refresh_step_us": refresh_ms * 1e3, "reuse_step_us": reuse_ms * 1e3,
+        "graph_replay": {"us_per_step": ms_graph * 1e3, "refresh_step_us": graph_refresh_ms * 1e3, "reuse_step_us": graph_reuse_ms * 1e3,
+                         "step_frac_of_peak": step_bytes / (ms_graph * 1e-3) / 1e9 / peak,
+                         "note": "the same steps as two CUDA graphs captured once (refresh / reuse) and replayed; lengths read "
+                                 "from device counters advanced by the append and projection kernels"},
         "step_hbm_gbs": step_bytes / (ms_step * 1e-3) / 1e9, "step_bytes": step_bytes,
         "step_bytes_note": "realised: the stored lists' lengths read back after the run (upper bound per attention launch: %.1f MB)" % (att_bytes_bound / 1e6),
         "step_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak,
@@ -634,7 +678,7 @@ def measure_trajectory(args, w):
 
 def brief_entry(line):
     """What the default run's `workloads` block keeps of another workload's line."""
-    keep = ("us_per_step", "us_per_step_min", "us_per_step_max", "timed_repeats", "steps", "warmup", "value", "step_bytes",
+    keep = ("us_per_step", "us_per_step_min", "us_per_step_max", "timed_repeats", "steps", "warmup", "value", "step_bytes", "graph_replay",
             "step_hbm_gbs", "step_frac_of_peak", "step_frac_of_nominal_8tbs", "refresh_step_us", "reuse_step_us", "roofline",
             "kernels", "e2e", "clocks", "gpu_launches")
     out = {k: line[k] for k in keep if k in line}

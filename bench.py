@@ -676,6 +676,79 @@ def measure_trajectory(args, w):
     return line
 
 
+def measure_list_layouts(args, w):
+    """Does it matter to the attention kernel where the listed rows lie?  (The paper's design migrates the
+    selected rows into a contiguous Important buffer, Sec. 3.3; this build gathers them by index from the
+    cache where they are.)  Same shapes, same list length, three layouts of the caller-supplied lists:
+    random positions, runs of three consecutive positions, one contiguous block.  Prints one JSON line."""
+    import torch
+    import torch.distributed as dist
+    from paper_2503_07518_b200 import binding as tbh
+    from paper_2503_07518_b200 import build
+    build.build()
+    dist_env(torch, dist)
+    ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + 8,
+                      w.budget, w.radius)
+    fill_caches(ctx, w, torch, tbh)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(wl.seed_for(w.cfg_id, 0, 0, wl.TAG_Q))
+    q = torch.randn(w.n_layers, w.batch, w.n_q_heads, w.head_dim, generator=gen, device="cuda").to(tbh.torch_dtype(w.dtype))
+    out = torch.empty(w.n_layers, w.batch, w.n_q_heads, w.head_dim, device="cuda")
+    cap = ctx.index_capacity
+    n_list = min(cap, ((2 * w.radius + 1) if w.nmode == 0 else (1 + w.radius)) * w.budget) // 3 * 3
+    L = min(w.lengths)
+    lo, hi = min(w.sinks, L), L - w.recent
+    r = np.random.Generator(np.random.PCG64(wl.seed_for(w.cfg_id, 0, 0, wl.TAG_AUX)))
+    units = w.n_layers * w.batch * w.n_kv_heads
+
+    def lists(kind):
+        rows = np.zeros((units, cap), np.int32)
+        for u in range(units):
+            if kind == "random":
+                rows[u, :n_list] = np.sort(r.choice(np.arange(lo, hi), n_list, replace=False))
+            elif kind == "runs_of_3":
+                c = np.sort(r.choice(np.arange(lo, hi - 3, 3), n_list // 3, replace=False))
+                rows[u, :n_list] = (c[:, None] + np.arange(3)[None, :]).reshape(-1)
+            else:
+                start = int(r.integers(lo, hi - n_list))
+                rows[u, :n_list] = np.arange(start, start + n_list)
+        return torch.from_numpy(rows.reshape(w.n_layers, w.batch, w.n_kv_heads, cap)).cuda()
+
+    cnt = torch.full((w.n_layers, w.batch, w.n_kv_heads), n_list, dtype=torch.int32, device="cuda")
+    p = tbh.select_params(w.budget, w.sinks, w.recent, w.radius, w.nmode)
+    res = {}
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for kind in ("random", "runs_of_3", "contiguous"):
+            idx = lists(kind)
+            g = torch.cuda.CUDAGraph()
+            for _ in range(2):
+                for l in range(w.n_layers):
+                    ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l], idx=idx[l:l + 1], cnt=cnt[l:l + 1])
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                for l in range(w.n_layers):
+                    ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p, out[l], idx=idx[l:l + 1], cnt=cnt[l:l + 1])
+            reps = []
+            for _ in range(12):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(4):
+                    g.replay()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                reps.append(e0.elapsed_time(e1) / 4 / w.n_layers * 1e3)
+            res[kind] = {"us_per_layer": float(np.median(reps)), "min": float(np.min(reps)), "max": float(np.max(reps))}
+        assert ctx.get_status(stream) == 0
+    rows = (min(w.sinks, L) + n_list + min(w.recent, L)) * w.batch * w.n_kv_heads
+    bytes_layer = rows * 2 * w.head_dim * (2 if w.dtype == wl.BF16 else 4)
+    for v in res.values():
+        v["gbs"] = bytes_layer / (v["us_per_layer"] * 1e-6) / 1e9
+    print(json.dumps({"attention_list_layouts": res, "workload": w.name, "layers": w.n_layers, "batch": w.batch,
+                      "rows_per_kv_head": rows // (w.batch * w.n_kv_heads), "bytes_per_layer": bytes_layer,
+                      "note": "caller-supplied lists of equal length; the K|V rows are gathered by index from the cache in all three"}))
+
+
 def brief_entry(line):
     """What the default run's `workloads` block keeps of another workload's line."""
     keep = ("us_per_step", "us_per_step_min", "us_per_step_max", "timed_repeats", "steps", "warmup", "value", "step_bytes", "graph_replay",
@@ -706,6 +779,8 @@ def main():
                     help="which heads share an index list (configs 1-4; default: one list per KV head)")
     ap.add_argument("--context", type=int, default=0,
                     help="override every sequence's context length (e.g. --config 4 --context 1048576 --layers 8)")
+    ap.add_argument("--list-layouts", action="store_true",
+                    help="time the attention kernel on random / runs-of-3 / contiguous caller lists of the workload's shapes")
     ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
                     help="neighbour rule of the interval workload (default: its own, +-r dilation)")
     args = ap.parse_args()
@@ -722,6 +797,9 @@ def main():
         return
     if args.warmup < 3:
         args.warmup = 3
+    if args.list_layouts:
+        measure_list_layouts(args, w)
+        return
 
     def measure(wk, brief=False):
         if wk.decode_steps > 1:

@@ -484,6 +484,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
             }
             phase_stamp(11);
             if (C > 1) cluster.sync(); else __syncthreads();   // barrier 2: the list is complete everywhere
+            // What is left is short and local.  A successor launched as a programmatic dependent (the first
+            // layer's attention) may be set up now; it waits for this grid's completion before it reads a list.
+            pdl_launch_dependents();
             phase_stamp(12);
             if (!whole) {
                 // every block ranks the list itself: an entry counts the entries ranked before it (larger key, or

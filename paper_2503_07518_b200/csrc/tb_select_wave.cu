@@ -796,7 +796,10 @@ __global__ void __launch_bounds__(kThreads, 2)
     // parked keys are kept in L2 for the block's return to them, unless the launch parks more than L2 can hold
     const uint64_t stream_policy = l2_policy_evict_first(), keep_policy = keep_in_l2 ? l2_policy_evict_last() : stream_policy;
 
-    // sample row and query first, then the ring's opening requests (see the kernel above)
+    // The sample rows and the queries are requested first, then the ring's opening tiles; nothing waits for
+    // the sample here.  Behind the whole grid's opening burst of bulk copies the sample rows take several
+    // microseconds, during which the ring would fill up and stall: the rows stay in registers and the digit
+    // is placed a few tiles into the stream; what was scored before that is digitised then from its parked keys.
     const bool sampled = ncand >= kMinSampled;
     uint4 srow[NCH];
 #pragma unroll
@@ -807,16 +810,24 @@ __global__ void __launch_bounds__(kThreads, 2)
 #pragma unroll
         for (int c = 0; c < NCH; ++c) srow[c] = __ldg(rowp + c);
     }
-    GroupScorer<T, DP, RED> scorer;
-    scorer.load(a.q_imp + query_row(gm, ut, ll, s, h) * DP, gm.gl, sm->qs);
-    if (RED != TB_GROUP_SUM) __syncthreads();
+    {
+        const float* q_unit = a.q_imp + query_row(gm, ut, ll, s, h) * DP;
+        if (tid < gm.gl * DP)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(sm->qs + tid)), "l"(q_unit + tid) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     if (tid == 0)
         for (int i = 0; i < n_stages && i < my_tiles; ++i) {
             mbar_arrive_expect_tx(&sm->full[i], kTileBytes);
             tma_load_2d_hint(stage_base + i * kTileBytes, &tmap, 0, (int)(row_base + slot0 + (long long)i * kRows), &sm->full[i], stream_policy);
         }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    GroupScorer<T, DP, RED> scorer;
+    scorer.load_staged(sm->qs, gm.gl);
     Digit dg = {0u, 21};
-    if (sampled) {                                     // identical in every block of the cluster: same rows, same arithmetic
+    // identical in every block of the cluster: same rows, same arithmetic.  Called by all threads, once.
+    auto place_digit = [&](int done_tiles) {
         if (tid < kSampleRows) sm->sample[tid] = order_key(scorer.score([&](int c) { return srow[c]; }));
         __syncthreads();
         if (tid < kSampleRows) {
@@ -848,7 +859,23 @@ __global__ void __launch_bounds__(kThreads, 2)
         range = wide > 0xffffffffull ? 0xffffffffu : (uint32_t)wide;
         dg.base = s_lo, dg.shift = 0;
         while ((range >> dg.shift) >= 2046u) ++dg.shift;
-    }
+        uint32_t kk[8];                                // this thread's own earlier keys, back from L2 together
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int slot = i * kRows + tid;
+            kk[i] = (i < done_tiles && slot < n_local) ? __ldcg(keys_unit + slot0 + slot) : 0u;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int slot = i * kRows + tid;
+            if (i < done_tiles && slot < n_local) {
+                const uint16_t b = (uint16_t)dg.bin(kk[i]);
+                hist_add(&hist[b]);
+                bins[slot] = b;
+            }
+        }
+    };
+    const int place_at = sampled ? min(my_tiles, 6) : -1;   // at most 8 (the catch-up's register array)
 
     CW_MARK(1);
     // ---- stream: score, park the key, keep the first digit ---------------------------------------------
@@ -857,6 +884,8 @@ __global__ void __launch_bounds__(kThreads, 2)
     int st = 0;
     uint32_t phase = 0;
     for (int i = 0; i < my_tiles; ++i) {
+        if (i == place_at) place_digit(i);
+        const bool placed = !sampled || i >= place_at;
         const bool ok = i < issued && mbar_wait(&sm->full[st], phase);
         const unsigned char* tile = stage_base + st * kTileBytes;
         const int slot = i * kRows + tid;
@@ -877,8 +906,10 @@ __global__ void __launch_bounds__(kThreads, 2)
 #else
             st_global_hint(keys_unit + slot0 + slot, key, keep_policy);
 #endif
-            b = (uint16_t)dg.bin(key);
-            hist_add(&hist[b]);
+            if (placed) {
+                b = (uint16_t)dg.bin(key);
+                hist_add(&hist[b]);
+            }
         }
         bins[slot] = b;
         if (__syncthreads_or(!ok)) dead = true;
@@ -894,6 +925,7 @@ __global__ void __launch_bounds__(kThreads, 2)
         if (++st == n_stages) st = 0, phase ^= 1u;
     }
     if (dead && tid == 0) atomicExch(status, kStatusTimeout);
+    if (place_at == my_tiles) place_digit(my_tiles);   // a short share: the digit is placed after its last tile
     __syncthreads();
     CW_MARK(2);
 #ifdef TB_PHASE_TIMING

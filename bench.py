@@ -244,6 +244,10 @@ def measure_static(args, w, brief=False):
     scope = {"kv_head": tbh.TB_SCOPE_KV_HEAD, "q_head": tbh.TB_SCOPE_Q_HEAD, "layer": tbh.TB_SCOPE_LAYER}[args.list_scope]
     ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + 8,
                       w.budget, w.radius, device=local, kv_on_host=args.offload_kv, list_scope=scope)
+    if args.resident_rows:                                   # device copies of the sink and window rows (offloaded KV)
+        ctx.bind_resident_rows(max(w.sinks, 1), max(w.recent, 1))
+    if args.important_buffer:
+        ctx.bind_important_buffer()
     proj_info = fill_caches(ctx, w, torch, tbh)
     dt = tbh.torch_dtype(w.dtype)
     gen = torch.Generator(device="cuda")
@@ -275,6 +279,30 @@ def measure_static(args, w, brief=False):
                     att_bytes.append(ctx.last_step_bytes())
 
     stream = torch.cuda.Stream()
+    s_sel = torch.cuda.Stream()
+
+    def step_overlapped(b=0):
+        # The same launches with each producer group's selection on a second stream, beside the attention of
+        # the group before it (a producer predicts for the layers after it, Sec. 3.1, so its selection does not
+        # wait for their attention).  Pays where attention is slow: rows fetched over the host link.
+        q_, qi_, out_ = bufs[b]
+        ev = [torch.cuda.Event() for _ in groups]
+        start = torch.cuda.Event()
+        start.record(stream)
+        s_sel.wait_event(start)
+        with torch.cuda.stream(s_sel):
+            ctx.select_topk(groups[0][0], groups[0][1], None, w.batch, qi_[groups[0][0]:groups[0][0] + groups[0][1]], p)
+            ev[0].record(s_sel)
+        for gi, (l0, n) in enumerate(groups):
+            stream.wait_event(ev[gi])
+            if gi + 1 < len(groups):
+                l1, n1 = groups[gi + 1]
+                with torch.cuda.stream(s_sel):
+                    ctx.select_topk(l1, n1, None, w.batch, qi_[l1:l1 + n1], p)
+                    ev[gi + 1].record(s_sel)
+            for l in range(l0, l0 + n):
+                ctx.sparse_decode_attention(l, 1, None, w.batch, q_[l], p, out_[l])
+
     with torch.cuda.stream(stream):
         n0 = ctx.launch_count()
         step_launches(record=True)
@@ -385,10 +413,19 @@ def measure_static(args, w, brief=False):
             g_dense = capture(lambda: [ctx.sparse_decode_attention(l, 1, None, w.batch, q[l], p_dense, out[l]) for l in range(w.n_layers)])
             ms_dense = timed(g_dense.replay, 3, 1, min_ms=0.0)
             dense_bytes = float(sum(w.lengths)) * w.n_layers * w.n_kv_heads * 2 * w.head_dim * (2 if w.dtype == wl.BF16 else 4)
+            g_ov = capture(step_overlapped)
+            ms_ov = timed(g_ov.replay, 3, 1, min_ms=0.0)
+            res_rows = (min(w.sinks, min(w.lengths)) + min(w.recent, min(w.lengths))) if args.resident_rows else 0
+            link_bytes = float(np.sum(att_bytes)) - float(res_rows) * w.n_layers * w.batch * w.n_kv_heads * 2 * w.head_dim * (2 if w.dtype == wl.BF16 else 4)
             offload_info = {"kv_placement": "page-locked host memory, rows fetched by the attention kernel over the host link",
+                            "resident_sink_and_window_rows": bool(args.resident_rows),
                             "dense_step_us": ms_dense * 1e3, "dense_link_gbs": dense_bytes / (ms_dense * 1e-3) / 1e9,
-                            "sparse_link_gbs": float(np.sum(att_bytes)) / (ms_step * 1e-3) / 1e9,
-                            "sparse_speedup_over_dense": ms_dense / ms_step}
+                            "sparse_step_us": ms_step * 1e3, "sparse_link_bytes_per_step": link_bytes,
+                            "sparse_link_gbs": link_bytes / (ms_step * 1e-3) / 1e9,
+                            "sparse_step_us_selection_overlapped": ms_ov * 1e3,
+                            "selection_us_per_step": ms_sel * len(groups) * 1e3,
+                            "overlap_achieved": (ms_step - ms_ov) / max(1e-9, ms_sel * len(groups)),
+                            "sparse_speedup_over_dense": ms_dense / min(ms_step, ms_ov)}
         ms_all = ms_pred = pred_bytes = None
         if not brief:
             # Upper bound, not the method's schedule: the importance queries of all layers at once, so the
@@ -488,7 +525,11 @@ def measure_trajectory(args, w):
     warm = max(P, (args.warmup + P - 1) // P * P)
     total = 2 * warm + 3 * steps                              # device-timed pass + end-to-end pass + graph-replay pass
     ctx = tbh.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, max(w.lengths) + total + Wn,
-                      w.budget, w.radius, device=local)
+                      w.budget, w.radius, device=local, kv_on_host=args.offload_kv)
+    if args.resident_rows:
+        ctx.bind_resident_rows(max(w.sinks, 1), max(w.recent, 1))
+    if args.important_buffer:
+        ctx.bind_important_buffer()
     fill_caches(ctx, w, torch, tbh)
     dt = tbh.torch_dtype(w.dtype)
     gen = torch.Generator(device="cuda")
@@ -646,7 +687,9 @@ def measure_trajectory(args, w):
         "metric": METRIC, "value": whole_job_tokens_per_s(w.batch, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warm,
         "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": storage_name(w), "data": "synthetic",
-        "config": {"workload": w.name, "layers": w.n_layers, "batch_per_gpu": w.batch, "context": w.lengths[0], "budget": w.budget,
+        "config": {"workload": w.name + ("+offloaded_kv" if args.offload_kv else "") + ("+resident_rows" if args.resident_rows else "") +
+                   ("+important_buffer" if args.important_buffer else ""),
+                   "layers": w.n_layers, "batch_per_gpu": w.batch, "context": w.lengths[0], "budget": w.budget,
                    "recent": w.recent, "radius": w.radius, "neighbor_mode": "dilate" if w.nmode == 0 else "cluster",
                    "interval": P, "schedule": "per layer: append, (deferred projection), attention; select+expand per 4 layers on "
                    "refresh steps; direct launches", "l2": "inputs larger than L2: %.0f MB touched per step" % (step_bytes / 1e6)},
@@ -775,6 +818,10 @@ def main():
     ap.add_argument("--profile", action="store_true", help="only warm-up + steps of plain launches (for ncu)")
     ap.add_argument("--offload-kv", action="store_true",
                     help="K|V cache in page-locked host memory (selected rows cross the host link); also times the dense step")
+    ap.add_argument("--resident-rows", action="store_true",
+                    help="with --offload-kv: device copies of the sink and window rows (only the selected rows cross the link)")
+    ap.add_argument("--important-buffer", action="store_true",
+                    help="the paper's contiguous Important buffer: selected rows migrated at every refresh, attended from there")
     ap.add_argument("--list-scope", default="kv_head", choices=["kv_head", "q_head", "layer"],
                     help="which heads share an index list (configs 1-4; default: one list per KV head)")
     ap.add_argument("--context", type=int, default=0,
@@ -812,6 +859,7 @@ def main():
     world, rank = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0"))
     if "profile_run" not in line:
         extra = default_run and not args.no_extra and not args.profile and world == 1 and not args.offload_kv and \
+            not args.important_buffer and \
             args.list_scope == "kv_head" and not args.layers and not args.context
         if extra:
             line["workloads"] = {}

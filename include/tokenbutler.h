@@ -267,6 +267,31 @@ tb_status tb_predict_importance_queries(const tb_predictor* p, const void* hidde
  * in *device_status and clear it. */
 tb_status tb_get_status(tb_ctx* ctx, void* stream, int32_t* device_status);
 
+/* Resident sink and window rows for an offloaded cache (paper Sec. 4.4 "CPU-offloaded KV": the full K/V in
+ * host memory, only selected rows cross the link).  With the K|V cache in page-locked host memory, every
+ * attended row crosses the host link each step -- the sinks and the recent window too, although they are the
+ * same rows step after step.  This binds a device region in which the library keeps, per (layer, sequence, KV
+ * head), copies of the first `sinks` tokens and of the `window` most recent ones (a ring indexed by position);
+ * tb_append_kv writes them beside the cache rows, attention reads sink and window rows from there whenever
+ * they are covered (S <= sinks, W <= window) and from the cache otherwise.  Results are the same bits.
+ * Bind while every sequence is empty (TB_ERR_STATE otherwise); rows_dev == NULL unbinds.  bytes must be at
+ * least tb_resident_rows_bytes(); 256-byte aligned device memory owned by the caller. */
+size_t tb_resident_rows_bytes(const tb_config* cfg, int32_t sinks, int32_t window);
+tb_status tb_bind_resident_rows(tb_ctx* ctx, void* rows_dev, size_t bytes, int32_t sinks, int32_t window);
+
+/* The paper's contiguous Important buffer (Sec. 3.3: "Sink / Local-Window / Important buffers"; Sec. 3.3 and
+ * 3.4: on a prediction step the selected K/V pairs are migrated into it, and the steps in between attend from
+ * it).  Once bound, every refreshing tb_select_topk ends with a migration kernel that copies the K|V rows of the
+ * stored lists into the buffer, in list order, and tb_sparse_decode_attention reads the list's rows from there
+ * (contiguous, no index lookup) when it attends from the stored lists; sinks and window still come from the cache
+ * (or the resident rows).  Same bits as gathering from the cache.  With the cache on the device it buys nothing
+ * measurable (a 512-byte row is already four full memory sectors) and costs a copy of every selected row per
+ * refresh; with an offloaded cache and a prediction interval P it cuts the link traffic P-fold.  Contexts with one
+ * list per KV head only (TB_ERR_UNSUPPORTED otherwise).  bytes >= tb_important_buffer_bytes(); buf_dev == NULL
+ * unbinds.  Binding drops the stored selections (TB_ERR_STATE from attention until the next selection). */
+size_t tb_important_buffer_bytes(const tb_config* cfg);
+tb_status tb_bind_important_buffer(tb_ctx* ctx, void* buf_dev, size_t bytes);
+
 /* Where the kernels take the sequence lengths from (Sec. 3.3 / 3.4: the cache grows by a token every decode
  * step and the window moves with it).  The context keeps the lengths twice: host mirrors, advanced when a
  * call is made, which validate arguments; and device counters, advanced by the append and projection kernels

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libtokenbutler.so")
 
 EXPORTS = ["tb_query_sizes", "tb_create", "tb_destroy", "tb_index_capacity", "tb_set_projection", "tb_reset_sequence",
            "tb_get_length", "tb_append_kv", "tb_project_keys", "tb_score_tokens", "tb_select_topk",
-           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_set_wait_diagnostics", "tb_use_device_lengths", "tb_sync_lengths", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
+           "tb_sparse_decode_attention", "tb_sparse_decode_attention_static", "tb_static_get_status", "tb_predict_importance_queries", "tb_get_status", "tb_set_wait_diagnostics", "tb_use_device_lengths", "tb_sync_lengths", "tb_resident_rows_bytes", "tb_bind_resident_rows", "tb_important_buffer_bytes", "tb_bind_important_buffer", "tb_last_step_bytes", "tb_launch_count", "tb_status_string"]
 
 
 class tb_config(C.Structure):
@@ -86,6 +86,12 @@ def lib():
         L.tb_set_wait_diagnostics.argtypes = [vp, i32, i32]
         L.tb_use_device_lengths.argtypes = [vp, i32, i32]
         L.tb_sync_lengths.argtypes = [vp, vp]
+        L.tb_resident_rows_bytes.restype = C.c_size_t
+        L.tb_resident_rows_bytes.argtypes = [C.POINTER(tb_config), i32, i32]
+        L.tb_bind_resident_rows.argtypes = [vp, vp, C.c_size_t, i32, i32]
+        L.tb_important_buffer_bytes.restype = C.c_size_t
+        L.tb_important_buffer_bytes.argtypes = [C.POINTER(tb_config)]
+        L.tb_bind_important_buffer.argtypes = [vp, vp, C.c_size_t]
         L.tb_last_step_bytes.argtypes = [vp]
         L.tb_launch_count.argtypes = [vp]
         L.tb_status_string.argtypes = [i32]
@@ -223,6 +229,18 @@ class Context:
         n = len(pos_begin) if pos_begin is not None else n_seq
         self._chk(lib().tb_project_keys(self.h, layer_begin, layer_count, _ints(seq_ids), _ints(pos_begin), _ints(pos_end),
                                         n, _stream(stream)), "tb_project_keys")
+
+    def bind_resident_rows(self, sinks, window):
+        """Allocates (torch) and binds device copies of the first `sinks` and the `window` most recent tokens' rows."""
+        n = lib().tb_resident_rows_bytes(C.byref(self.cfg), sinks, window)
+        self.resident_rows = torch.empty(max(n, 256), dtype=torch.uint8, device=self.device)
+        self._chk(lib().tb_bind_resident_rows(self.h, _ptr(self.resident_rows), n, sinks, window), "tb_bind_resident_rows")
+
+    def bind_important_buffer(self):
+        """Allocates (torch) and binds the contiguous Important buffer."""
+        n = lib().tb_important_buffer_bytes(C.byref(self.cfg))
+        self.important_buffer = torch.empty(max(n, 256), dtype=torch.uint8, device=self.device)
+        self._chk(lib().tb_bind_important_buffer(self.h, _ptr(self.important_buffer), n), "tb_bind_important_buffer")
 
     def use_device_lengths(self, on=True, growth_reserve=0):
         self._chk(lib().tb_use_device_lengths(self.h, int(on), growth_reserve), "tb_use_device_lengths")

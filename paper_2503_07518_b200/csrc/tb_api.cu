@@ -231,6 +231,7 @@ tb_status tb_create(const tb_config* cfg, void* kv, void* kimp, void* state, voi
     c->last_bytes = 0, c->launches = 0;
     c->wait_poll_limit = 0, c->drop_tile = -1;
     c->dev_lengths = 0, c->growth_reserve = 0;
+    c->res_rows = nullptr, c->res_sinks = c->res_window = 0, c->imp_rows = nullptr;
     c->last_cache_write = c->last_list_write = -4;
     c->tile_rows = 256;
     for (int i = 0; i < 17; ++i) c->attn_max_active[i] = 0;
@@ -440,6 +441,10 @@ tb_status tb_select_topk(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_i
                     if (e != cudaSuccess) return dry ? TB_ERR_UNSUPPORTED : TB_ERR_CUDA;
                     if (!dry) c->last_list_write = (long long)c->launches, c->launches++;
                 }
+                if (!dry && c->imp_rows) {               // KV migration into the Important buffer
+                    if (launch_migrate(c, ut, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+                    c->last_list_write = (long long)c->launches, c->launches++;
+                }
             }
             if (!dry && (idx_out || cnt_out)) {
                 if (launch_copy_lists(c, ut, idx_out ? idx_out + unit_off * c->geom.idx_cap : nullptr,
@@ -504,6 +509,8 @@ tb_status tb_sparse_decode_attention(tb_ctx* c, int32_t lb, int32_t lc, const in
         const size_t hq_off = (size_t)(l0 - lb) * n_seq * c->cfg.n_q_heads;
         const size_t unit_off = (size_t)(l0 - lb) * n_seq * c->geom.Hl;
         AttnArgs a;
+        a.res_rows = c->res_rows, a.res_sinks = c->res_sinks, a.res_window = c->res_window;
+        a.imp_rows = (dense || idx) ? nullptr : c->imp_rows;
         a.q = (const char*)q + hq_off * c->cfg.head_dim * es;
         a.idx = idx ? idx + unit_off * c->geom.idx_cap : nullptr;
         a.cnt = cnt ? cnt + unit_off : nullptr;
@@ -531,6 +538,51 @@ tb_status tb_get_status(tb_ctx* c, void* stream, int32_t* device_status) {
     if (cudaMemsetAsync(c->st.status, 0, 4, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
     *device_status = v;
+    return TB_OK;
+}
+
+size_t tb_resident_rows_bytes(const tb_config* cfg, int32_t sinks, int32_t window) {
+    if (check_config(cfg) != TB_OK || sinks < 0 || window < 0) return 0;
+    return (size_t)cfg->n_layers * cfg->max_batch * cfg->n_kv_heads * ((size_t)sinks + window) * 2 * cfg->head_dim * elem_size(cfg->kv_dtype);
+}
+
+size_t tb_important_buffer_bytes(const tb_config* cfg) {
+    if (check_config(cfg) != TB_OK || cfg->list_scope != TB_SCOPE_KV_HEAD) return 0;
+    Layout l;
+    compute_layout(cfg, &l);
+    return (size_t)cfg->n_layers * cfg->max_batch * cfg->n_kv_heads * (size_t)l.idx_cap * 2 * cfg->head_dim * elem_size(cfg->kv_dtype);
+}
+
+namespace {
+bool device_memory(const void* p) {
+    cudaPointerAttributes pa;
+    if (cudaPointerGetAttributes(&pa, p) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    return pa.type == cudaMemoryTypeDevice || pa.type == cudaMemoryTypeManaged;
+}
+bool all_sequences_empty(const tb_ctx* c) {
+    for (int v : c->len) if (v) return false;
+    return true;
+}
+}  // namespace
+
+tb_status tb_bind_resident_rows(tb_ctx* c, void* rows_dev, size_t bytes, int32_t sinks, int32_t window) {
+    if (!c || sinks < 0 || window < 0) return TB_ERR_INVALID_ARG;
+    if (!rows_dev) { c->res_rows = nullptr, c->res_sinks = c->res_window = 0; return TB_OK; }
+    if (sinks + window == 0 || ((uintptr_t)rows_dev & 255) || !device_memory(rows_dev)) return TB_ERR_INVALID_ARG;
+    if (bytes < tb_resident_rows_bytes(&c->cfg, sinks, window)) return TB_ERR_CAPACITY;
+    if (!all_sequences_empty(c)) return TB_ERR_STATE;   // the copies are kept current by the appends: bind before the first one
+    c->res_rows = rows_dev, c->res_sinks = sinks, c->res_window = window;
+    return TB_OK;
+}
+
+tb_status tb_bind_important_buffer(tb_ctx* c, void* buf_dev, size_t bytes) {
+    if (!c) return TB_ERR_INVALID_ARG;
+    if (!buf_dev) { c->imp_rows = nullptr; return TB_OK; }
+    if (c->cfg.list_scope != TB_SCOPE_KV_HEAD) return TB_ERR_UNSUPPORTED;
+    if (((uintptr_t)buf_dev & 255) || !device_memory(buf_dev)) return TB_ERR_INVALID_ARG;
+    if (bytes < tb_important_buffer_bytes(&c->cfg)) return TB_ERR_CAPACITY;
+    for (int& v : c->has_sel) v = 0;                    // stored lists have no rows in the buffer yet: select first
+    c->imp_rows = buf_dev;
     return TB_OK;
 }
 

@@ -21,30 +21,46 @@ constexpr int kAttnMaxCluster = 16;      // splits that can be merged inside a t
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-// Which token does attended row r refer to?  Rows are sinks, then the index list, then the window.
+// Which row does attended row r refer to?  Rows are sinks, then the index list, then the window.  The answer
+// is a row reference (see kRowSrcShift): a token of the cache or, when the context has them, a slot of the
+// resident sink / window copies or of the Important buffer.
 struct RowMap {
     int n_sink, n_list, w_begin, L, dense;
+    int res_sinks, res_window;      // 0 = no resident copies
+    int use_imp;                    // list rows come from the Important buffer, in list order
     const int32_t* list;
+    // token t in the resident copies if they hold it (one of the first res_sinks tokens, else one of the
+    // res_window most recent), else in the cache
+    __device__ __forceinline__ int res_ref(int t) const {
+        if (t < res_sinks) return (kRowSrcResident << kRowSrcShift) | t;
+        return (res_window > 0 && t >= L - res_window) ? (kRowSrcResident << kRowSrcShift) | (res_sinks + t % res_window) : t;
+    }
+    __device__ __forceinline__ int sink_ref(int t) const { return res_ref(t); }
+    __device__ __forceinline__ int window_ref(int t) const { return res_ref(t); }
     __device__ __forceinline__ int token(int r, bool& bad) const {
         bad = false;
-        if (dense || r < n_sink) return r;
+        if (dense) return r;
+        if (r < n_sink) return sink_ref(r);
         r -= n_sink;
         if (r < n_list) {
+            if (use_imp) return (kRowSrcImportant << kRowSrcShift) | r;
             int t = list[r];
             if (t < 0 || t >= L) { bad = true; return 0; }
             return t;
         }
-        return w_begin + (r - n_list);
+        return window_ref(w_begin + (r - n_list));
     }
     // the same with a bad list entry reported as -1 (nothing else depends on the loaded value)
     __device__ __forceinline__ int token_or_neg(int r) const {
-        if (dense || r < n_sink) return r;
+        if (dense) return r;
+        if (r < n_sink) return sink_ref(r);
         r -= n_sink;
         if (r < n_list) {
+            if (use_imp) return (kRowSrcImportant << kRowSrcShift) | r;
             const int t = list[r];
             return (t < 0 || t >= L) ? -1 : t;
         }
-        return w_begin + (r - n_list);
+        return window_ref(w_begin + (r - n_list));
     }
 };
 
@@ -170,6 +186,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
 
     RowMap rm;
     rm.L = L, rm.dense = a.dense;
+    rm.res_sinks = a.res_rows ? a.res_sinks : 0, rm.res_window = a.res_rows ? a.res_window : 0;
+    rm.use_imp = a.imp_rows != nullptr && a.idx == nullptr;
     rm.n_sink = a.dense ? 0 : min(a.sinks, L);
     rm.w_begin = a.dense ? 0 : max(rm.n_sink, L - a.recent);
     int n_list = 0;
@@ -209,7 +227,10 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
         acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.f;
     }
 
-    const T* kv_unit = kv + au.kv_c * gm.max_seq_len * 2 * D;
+    // the unit's rows in the cache and in the optional copies, indexed by a row reference's source
+    const T* src_base[3] = {kv + au.kv_c * gm.max_seq_len * 2 * D,
+                            reinterpret_cast<const T*>(a.res_rows) + au.kv_c * (size_t)(a.res_sinks + a.res_window) * 2 * D,
+                            reinterpret_cast<const T*>(a.imp_rows) + au.list_c * (size_t)gm.idx_cap * 2 * D};
     bool any_bad = false;
     for (int r0 = wb; r0 < we; r0 += kRowsPerIter) {
         RowVec<T> kr[kRowsPerIter], vr[kRowsPerIter];
@@ -220,7 +241,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
             valid[i] = r0 + i < we;
             int t = valid[i] ? rm.token(r0 + i, bad) : 0;
             if (bad) valid[i] = false, any_bad = true;
-            const T* row = kv_unit + (size_t)t * 2 * D;
+            const int which = t >> kRowSrcShift;
+            const T* row = (which == 0 ? src_base[0] : which == 1 ? src_base[1] : src_base[2]) + (size_t)(t & kRowIdxMask) * 2 * D;
             kr[i].load(row, lane);
             vr[i].load(row + D, lane);
         }
@@ -392,6 +414,8 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
 
     RowMap rm;
     rm.L = L, rm.dense = a.dense;
+    rm.res_sinks = a.res_rows ? a.res_sinks : 0, rm.res_window = a.res_rows ? a.res_window : 0;
+    rm.use_imp = a.imp_rows != nullptr && a.idx == nullptr;
     rm.n_sink = a.dense ? 0 : min(a.sinks, L);
     rm.w_begin = a.dense ? 0 : max(rm.n_sink, L - a.recent);
     int n_list = 0;
@@ -414,7 +438,10 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const int n_tiles = (we - wb + kTileTok - 1) / kTileTok;
 
     unsigned char* my_stage = smem_dyn + (size_t)warp * kMmaStages * kStageBytes;
+    // the unit's rows in the cache and in the optional copies (see RowMap), 512 bytes per K|V row pair
     const unsigned char* kv_unit = reinterpret_cast<const unsigned char*>(kv) + au.kv_c * gm.max_seq_len * 2 * D * 2;
+    const unsigned char* res_unit = reinterpret_cast<const unsigned char*>(a.res_rows) + au.kv_c * (size_t)(a.res_sinks + a.res_window) * 2 * D * 2;
+    const unsigned char* imp_unit = reinterpret_cast<const unsigned char*>(a.imp_rows) + au.list_c * (size_t)gm.idx_cap * 2 * D * 2;
 
     bool any_bad = false;
     // Gather of one tile: the whole warp copies each 512-byte K|V row with one 16-byte cp.async per
@@ -426,12 +453,13 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const uint32_t stage_u32 = smem_u32(my_stage);
     auto issue_token = [&](int tile, int t) {     // t: lane i < 16 holds the token of row i
         const uint32_t dst = stage_u32 + (tile % kMmaStages) * kStageBytes;
-        const unsigned char* src = kv_unit + lane * 16;
 #pragma unroll
         for (int i = 0; i < kTileTok; ++i) {
             const int ti = __shfl_sync(0xffffffffu, t, i);
+            const int which = ti >> kRowSrcShift;
+            const unsigned char* src = (which == 0 ? kv_unit : which == 1 ? res_unit : imp_unit) + lane * 16;
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * kRowPitch + ((lane ^ (i & 7)) << 4)),
-                         "l"(src + (size_t)ti * 512) : "memory");
+                         "l"(src + (size_t)(ti & kRowIdxMask) * 512) : "memory");
         }
     };
     auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
@@ -918,6 +946,7 @@ extern "C" tb_status tb_sparse_decode_attention_static(const void* kv_dev, int32
         if (rows > max_rows) max_rows = rows;
     }
     AttnArgs a;
+    a.res_rows = nullptr, a.res_sinks = a.res_window = 0, a.imp_rows = nullptr;
     a.q = q_dev, a.idx = idx_dev, a.cnt = cnt_dev, a.out = out_dev, a.lse = lse_dev;
     a.dense = idx_dev ? 0 : 1, a.sinks = idx_dev ? sinks : 0, a.recent = idx_dev ? recent : 0;
     a.list_bound = idx_dev ? idx_stride : 0;

@@ -16,7 +16,8 @@ struct AppendTable {
 template <typename T>
 __global__ void append_kernel(Geom gm, UnitTable ut, AppendTable at, int total_new, const T* __restrict__ k_new,
                               const T* __restrict__ v_new, T* __restrict__ kv, int32_t* __restrict__ len_dev,
-                              uint32_t* __restrict__ counter, int32_t* __restrict__ status) {
+                              uint32_t* __restrict__ counter, int32_t* __restrict__ status, T* __restrict__ res_rows,
+                              int res_sinks, int res_window) {
     constexpr int kPer16 = Elem<T>::kPer16;
     const int chunks_per_row = gm.D / kPer16;          // 16-byte chunks in one K (or V) row
     const int chunks_per_pair = 2 * chunks_per_row;
@@ -42,7 +43,20 @@ __global__ void append_kernel(Geom gm, UnitTable ut, AppendTable at, int total_n
         const T* src = (is_v ? v_new : k_new) + (((size_t)ll * total_new + tok) * gm.Hkv + h) * gm.D;
         size_t row = (((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h) * gm.max_seq_len + pos;
         T* dst = kv + row * 2 * gm.D + (size_t)is_v * gm.D;
-        reinterpret_cast<uint4*>(dst)[c16] = reinterpret_cast<const uint4*>(src)[c16];
+        const uint4 val = reinterpret_cast<const uint4*>(src)[c16];
+        reinterpret_cast<uint4*>(dst)[c16] = val;
+        if (res_rows) {
+            // resident copies (offloaded KV): the first res_sinks tokens, and a ring of the res_window most recent
+            const int n_s = at.tok_off[s + 1] - at.tok_off[s];
+            int slot = -1;
+            if (pos < res_sinks) slot = pos;
+            else if (res_window > 0 && pos >= base + n_s - res_window) slot = res_sinks + pos % res_window;
+            if (slot >= 0) {
+                const size_t unit = ((size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s]) * gm.Hkv + h;
+                T* rdst = res_rows + (unit * (size_t)(res_sinks + res_window) + slot) * 2 * gm.D + (size_t)is_v * gm.D;
+                reinterpret_cast<uint4*>(rdst)[c16] = val;
+            }
+        }
     }
     if (last_block_arrives(counter, gridDim.x * gridDim.y)) {
         for (int i = threadIdx.x; i < ut.layer_count * ut.n_seq; i += blockDim.x) {
@@ -74,9 +88,45 @@ cudaError_t launch_append(const tb_ctx* c, const UnitTable& ut, const int* n_new
     cfg.attrs = attr, cfg.numAttrs = 1;
     if (gm.dtype == TB_BF16)
         return cudaLaunchKernelEx(&cfg, append_kernel<__nv_bfloat16>, gm, ut, at, total_new, (const __nv_bfloat16*)k,
-                                  (const __nv_bfloat16*)v, (__nv_bfloat16*)c->kv, c->st.len, c->st.misc_counter, c->st.status);
+                                  (const __nv_bfloat16*)v, (__nv_bfloat16*)c->kv, c->st.len, c->st.misc_counter, c->st.status,
+                                  (__nv_bfloat16*)c->res_rows, c->res_sinks, c->res_window);
     return cudaLaunchKernelEx(&cfg, append_kernel<float>, gm, ut, at, total_new, (const float*)k, (const float*)v, (float*)c->kv,
-                              c->st.len, c->st.misc_counter, c->st.status);
+                              c->st.len, c->st.misc_counter, c->st.status, (float*)c->res_rows, c->res_sinks, c->res_window);
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV migration (paper Sec. 3.3: on a prediction step the selected K/V pairs are moved into the contiguous
+// Important buffer, from which the following steps attend): rows list[j] of the cache -> row j of the
+// unit's buffer, 16 bytes per thread.  One block column per list; the count is read on the device.
+template <typename T>
+__global__ void __launch_bounds__(256) migrate_kernel(Geom gm, UnitTable ut, const T* __restrict__ kv, const int32_t* __restrict__ state_idx,
+                                                      const int32_t* __restrict__ state_cnt, T* __restrict__ imp) {
+    constexpr int kPer16 = Elem<T>::kPer16;
+    const int chunks = 2 * gm.D / kPer16;              // 16-byte chunks of a K|V row pair
+    const int u = blockIdx.y, h = u % gm.Hl, s = (u / gm.Hl) % ut.n_seq, ll = u / (gm.Hl * ut.n_seq);
+    const size_t pc = (size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s];
+    const size_t lc = pc * gm.Hl + h, kc = pc * gm.Hkv + h;               // lists are per KV head here
+    const int n = min(state_cnt[lc], gm.idx_cap);
+    const int32_t* list = state_idx + lc * gm.idx_cap;
+    const uint4* src = reinterpret_cast<const uint4*>(kv + kc * gm.max_seq_len * 2 * gm.D);
+    uint4* dst = reinterpret_cast<uint4*>(imp + lc * (size_t)gm.idx_cap * 2 * gm.D);
+    for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < (long long)n * chunks; w += (long long)gridDim.x * blockDim.x) {
+        const int j = (int)(w / chunks), c = (int)(w % chunks);
+        dst[(size_t)j * chunks + c] = src[(size_t)list[j] * chunks + c];
+    }
+}
+
+cudaError_t launch_migrate(const tb_ctx* c, const UnitTable& ut, cudaStream_t s) {
+    const Geom& gm = c->geom;
+    const int units = ut.layer_count * ut.n_seq * gm.Hl;
+    int bx = 2 * c->sm_count / units;                  // about two blocks per SM over the launch
+    bx = bx < 1 ? 1 : bx > 64 ? 64 : bx;
+    dim3 grid(bx, units);
+    if (gm.dtype == TB_BF16)
+        migrate_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(gm, ut, (const __nv_bfloat16*)c->kv, c->st.idx, c->st.cnt, (__nv_bfloat16*)c->imp_rows);
+    else
+        migrate_kernel<float><<<grid, 256, 0, s>>>(gm, ut, (const float*)c->kv, c->st.idx, c->st.cnt, (float*)c->imp_rows);
+    return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------------

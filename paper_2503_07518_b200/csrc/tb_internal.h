@@ -63,7 +63,20 @@ struct NeighborArgs {
     int radius, nmode, sinks, recent;
 };
 
+// Where an attended row is read from: the K|V cache, or one of two optional copies in device memory.
+// A row reference is one int: bits 0..28 the row inside its source, bits 29..30 the source.
+constexpr int kRowSrcShift = 29;
+constexpr int kRowIdxMask = (1 << kRowSrcShift) - 1;
+constexpr int kRowSrcCache = 0, kRowSrcResident = 1, kRowSrcImportant = 2;
+
 struct AttnArgs {
+    // Resident rows (offloaded KV): per (layer, sequence, KV head) the first res_sinks tokens and a ring of the
+    // res_window most recent ones (token t in slot res_sinks + t % res_window), kept current by the append kernel.
+    const void* res_rows;   // NULL = not bound
+    int res_sinks, res_window;
+    // Important buffer: per (layer, sequence, KV head) the K|V rows of the stored list, in list order,
+    // written by the migration kernel at every refresh (NULL = not bound, or caller-supplied lists).
+    const void* imp_rows;
     const void* q;          // [layer_count][n_seq][Hq][D]
     const int32_t* idx;     // caller lists (launch-unit indexed) or NULL = stored lists
     const int32_t* cnt;
@@ -121,6 +134,9 @@ struct tb_ctx {
     int tile_rows;                        // rows per TMA box of the score pass
     int sm_count;
     int attn_max_active[17];              // co-resident attention clusters per cluster size (0 = not asked yet)
+    void* res_rows;                       // resident sink + window rows (tb_bind_resident_rows), or NULL
+    int res_sinks, res_window;
+    void* imp_rows;                       // Important buffer (tb_bind_important_buffer), or NULL
     int dev_lengths;                      // 1: kernels read the device counters (graph-replayable growth)
     int growth_reserve;                   // tokens a sequence may grow beyond the host mirror while graphs are replayed
     int wait_poll_limit;                  // polls per bounded wait of the selection kernels; 0 = the default (seconds)
@@ -184,6 +200,8 @@ cudaError_t launch_select_wave(const tb_ctx* c, const UnitTable& ut, const Selec
 // few, long problems: a cluster per problem on parked keys
 cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectArgs& a, cudaStream_t s, bool dry = false);
 cudaError_t launch_neighbors(const tb_ctx* c, const UnitTable& ut, const NeighborArgs& a, cudaStream_t s, bool dry = false);
+// copies the rows of the stored lists into the Important buffer (after a refresh)
+cudaError_t launch_migrate(const tb_ctx* c, const UnitTable& ut, cudaStream_t s);
 cudaError_t launch_copy_lists(const tb_ctx* c, const UnitTable& ut, int32_t* idx_out, int32_t* cnt_out, cudaStream_t s);
 
 // tb_attention.cu

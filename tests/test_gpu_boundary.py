@@ -206,3 +206,79 @@ def test_captured_graphs_replay_a_growing_sequence(H):
     # back on host-carried lengths the same context goes on as usual
     full = H.gpu_select(case, H.queries(w, 99)[1], b_.select_params(w.budget, 0, Wn, 0))
     assert ctx.get_status() == 0 and len(full[0][0][0]) == w.budget
+
+
+@pytest.mark.parametrize("on_host", [False, True])
+def test_resident_rows_and_important_buffer_give_the_same_bits(H, on_host):
+    """Offloaded-KV options (Sec. 4.4) and the paper's contiguous Important buffer (Sec. 3.3): device copies of
+    the sink and window rows kept current by the appends, and the selected rows migrated into a contiguous
+    buffer at every refresh.  Both only change where a row is read from, so every output must be bit-equal to
+    the plain index-driven gather -- over a trajectory in which the window slides, the selection is reused for
+    P steps, and the sink / window sizes asked for are smaller than, equal to and larger than the copies."""
+    b_ = tb()
+    P, steps = 3, 7
+    w = wl.workload(5, n_layers=2, batch=2, n_q_heads=8, n_kv_heads=2, lengths=[900, 333], budget=60, sinks=5, recent=12,
+                    radius=1, interval=P, decode_steps=steps)
+
+    def run(resident, important):
+        outs = []
+        ctx_args = dict(extra_len=steps + 2, kv_on_host=on_host, project=None)
+        # the copies must be bound before the first append: build the context by hand, then fill it
+        case = H.Case.__new__(H.Case)
+        case.w, case.lengths = w, list(w.lengths)
+        case.cap = max(case.lengths) + steps + 2
+        case.ctx = b_.Context(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.imp_dim, w.dtype, w.batch, case.cap, w.budget,
+                              w.radius, kv_on_host=on_host)
+        if resident:
+            case.ctx.bind_resident_rows(sinks=8, window=16)
+        if important:
+            case.ctx.bind_important_buffer()
+        case.Hi = case.Hl = case.Ha = w.n_kv_heads
+        case.gl = case.ga = w.group
+        case.K = [[None] * w.batch for _ in range(w.n_layers)]
+        case.V = [[None] * w.batch for _ in range(w.n_layers)]
+        case.Kimp = [[np.zeros((2, case.cap, w.imp_dim), np.uint16) for _ in range(w.batch)] for _ in range(w.n_layers)]
+        case.W = []
+        for l in range(w.n_layers):
+            case.W.append(wl.gen_W(w, l))
+            case.ctx.set_projection(l, H.to_dev(case.W[l], w.dtype))
+            Ks, Vs = [], []
+            for b in range(w.batch):
+                K, V = wl.gen_KV(w, l, b)
+                case.K[l][b] = np.zeros((2, case.cap, w.head_dim), K.dtype)
+                case.V[l][b] = np.zeros_like(case.K[l][b])
+                case.K[l][b][:, :w.lengths[b]] = K
+                case.V[l][b][:, :w.lengths[b]] = V
+                Ks.append(K), Vs.append(V)
+            case._append_layer(l, Ks, Vs)
+        case.cur, case.proj = list(w.lengths), [0] * w.batch
+        case.project_all(compare=False)
+        for t in range(steps):
+            if t > 0:
+                case.append_step(t)
+                case.project_range(list(case.proj), list(case.cur), compare=False)
+            q, qi = H.queries(w, t)
+            # sink / window sizes below, at and above what the copies hold
+            S, Wn = [(5, 12), (8, 16), (11, 20)][t % 3] if t % P == 0 else last
+            last = (S, Wn)
+            p = b_.select_params(w.budget, S, Wn, 1, 0, P, t)
+            lists = H.gpu_select(case, qi, p)
+            out, lse = H.gpu_attention(case, q, p)
+            assert case.ctx.get_status() == 0
+            outs.append((lists, out, lse))
+        return case, outs
+
+    base_case, base = run(False, False)
+    for resident, important in ((True, False), (False, True), (True, True)):
+        _, got = run(resident, important)
+        for t in range(steps):
+            assert all(np.array_equal(x, y) for l in range(2) for s in range(2) for x, y in zip(base[t][0][l][s], got[t][0][l][s]))
+            assert np.array_equal(base[t][1], got[t][1]) and np.array_equal(base[t][2], got[t][2]), (resident, important, t)
+    # and the common result is the oracle's (last step, stored lists)
+    q, _ = H.queries(w, steps - 1)
+    p = b_.select_params(w.budget, *[(5, 12), (8, 16), (11, 20)][((steps - 1) // P * P) % 3], 1, 0, P, steps - 1)
+    for l in range(2):
+        for b in range(2):
+            for h in range(2):
+                ref, _ = base_case.oracle_attention(l, b, h, q[l, b], base[-1][0][l][b][h], p)
+                assert np.abs(base[-1][1][l, b, h * 4:(h + 1) * 4] - ref).max() <= 2e-3

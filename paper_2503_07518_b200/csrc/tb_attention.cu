@@ -24,6 +24,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 // Which row does attended row r refer to?  Rows are sinks, then the index list, then the window.  The answer
 // is a row reference (see kRowSrcShift): a token of the cache or, when the context has them, a slot of the
 // resident sink / window copies or of the Important buffer.
+template <bool kSources>           // false: every row comes from the cache (the copies are not bound)
 struct RowMap {
     int n_sink, n_list, w_begin, L, dense;
     int res_sinks, res_window;      // 0 = no resident copies
@@ -32,6 +33,7 @@ struct RowMap {
     // token t in the resident copies if they hold it (one of the first res_sinks tokens, else one of the
     // res_window most recent), else in the cache
     __device__ __forceinline__ int res_ref(int t) const {
+        if constexpr (!kSources) return t;
         if (t < res_sinks) return (kRowSrcResident << kRowSrcShift) | t;
         return (res_window > 0 && t >= L - res_window) ? (kRowSrcResident << kRowSrcShift) | (res_sinks + t % res_window) : t;
     }
@@ -43,7 +45,7 @@ struct RowMap {
         if (r < n_sink) return sink_ref(r);
         r -= n_sink;
         if (r < n_list) {
-            if (use_imp) return (kRowSrcImportant << kRowSrcShift) | r;
+            if (kSources && use_imp) return (kRowSrcImportant << kRowSrcShift) | r;
             int t = list[r];
             if (t < 0 || t >= L) { bad = true; return 0; }
             return t;
@@ -56,7 +58,7 @@ struct RowMap {
         if (r < n_sink) return sink_ref(r);
         r -= n_sink;
         if (r < n_list) {
-            if (use_imp) return (kRowSrcImportant << kRowSrcShift) | r;
+            if (kSources && use_imp) return (kRowSrcImportant << kRowSrcShift) | r;
             const int t = list[r];
             return (t < 0 || t >= L) ? -1 : t;
         }
@@ -184,7 +186,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
     const AttnUnit au(gm, ut, ll, s, h);
     const int lu = au.lu;
 
-    RowMap rm;
+    RowMap<true> rm;
     rm.L = L, rm.dense = a.dense;
     rm.res_sinks = a.res_rows ? a.res_sinks : 0, rm.res_window = a.res_rows ? a.res_window : 0;
     rm.use_imp = a.imp_rows != nullptr && a.idx == nullptr;
@@ -385,7 +387,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // distributed shared memory, one cluster barrier, and rank 0 merges in rank order -- no partials in
 // global memory, no last-block round trips.  Without it (more splits than a cluster holds) the splits
 // go through the global workspace and the last block to arrive merges them (NW must be 4 then).
-template <int NW, int kMmaStages>
+// kSources: the resident sink / window copies or the Important buffer are bound and a row reference names
+// its source; without them (the usual case) the gather carries no trace of the option.
+template <int NW, int kMmaStages, bool kSources = false>
 __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut, AttnArgs a, const __nv_bfloat16* __restrict__ kv,
                                                            const int32_t* __restrict__ state_idx,
                                                            const int32_t* __restrict__ state_cnt, float* __restrict__ part_o,
@@ -412,7 +416,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const AttnUnit au(gm, ut, ll, s, h);
     const int lu = au.lu;
 
-    RowMap rm;
+    RowMap<kSources> rm;
     rm.L = L, rm.dense = a.dense;
     rm.res_sinks = a.res_rows ? a.res_sinks : 0, rm.res_window = a.res_rows ? a.res_window : 0;
     rm.use_imp = a.imp_rows != nullptr && a.idx == nullptr;
@@ -456,10 +460,15 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
 #pragma unroll
         for (int i = 0; i < kTileTok; ++i) {
             const int ti = __shfl_sync(0xffffffffu, t, i);
-            const int which = ti >> kRowSrcShift;
-            const unsigned char* src = (which == 0 ? kv_unit : which == 1 ? res_unit : imp_unit) + lane * 16;
+            const unsigned char* src = kv_unit;
+            int row = ti;
+            if constexpr (kSources) {
+                const int which = ti >> kRowSrcShift;
+                src = which == 0 ? kv_unit : which == 1 ? res_unit : imp_unit;
+                row = ti & kRowIdxMask;
+            }
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + i * kRowPitch + ((lane ^ (i & 7)) << 4)),
-                         "l"(src + (size_t)(ti & kRowIdxMask) * 512) : "memory");
+                         "l"(src + lane * 16 + (size_t)row * 512) : "memory");
         }
     };
     auto commit = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
@@ -723,14 +732,17 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         static unsigned char seen[64];
         int* max_active = const_cast<tb_ctx*>(c)->attn_max_active;
         if (first_use_on_this_device(seen)) {
-            cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+            cudaError_t e = cudaSuccess;
+            auto prepare = [&](auto kernel, int max_kb, bool required) {
+                cudaError_t r = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_kb * 1024);
+                if (r == cudaSuccess) (void)cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+                if (r != cudaSuccess && required && e == cudaSuccess) e = r;
+            };
+            prepare(attn_mma_kernel<4, 2, false>, 113, true), prepare(attn_mma_kernel<4, 2, true>, 113, true);
+            prepare(attn_mma_kernel<8, 2, false>, 220, true), prepare(attn_mma_kernel<8, 2, true>, 220, true);
+            prepare(attn_mma_kernel<8, 3, false>, 220, true), prepare(attn_mma_kernel<8, 3, true>, 220, true);
+            prepare(attn_mma_kernel<12, 2, false>, 224, false), prepare(attn_mma_kernel<12, 2, true>, 224, false);
             if (e != cudaSuccess) return e;
-            (void)cudaFuncSetAttribute(attn_mma_kernel<8, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-            (void)cudaFuncSetAttribute(attn_mma_kernel<8, 3>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-            if (cudaFuncSetAttribute(attn_mma_kernel<12, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) == cudaSuccess)
-                (void)cudaFuncSetAttribute(attn_mma_kernel<12, 2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             (void)cudaGetLastError();
         }
         auto clusters_that_fit = [&](int csize) {     // how many clusters of `csize` 8-warp blocks run at once
@@ -819,17 +831,17 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         cfg.attrs = attr;
         cfg.numAttrs = 2;
         const __nv_bfloat16* kvp = (const __nv_bfloat16*)c->kv;
-        if (nw == 12)
-            return cudaLaunchKernelEx(&cfg, attn_mma_kernel<12, 2>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
-                                      c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
-        if (nw == 8 && nst == 3)
-            return cudaLaunchKernelEx(&cfg, attn_mma_kernel<8, 3>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
-                                      c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
-        if (nw == 8)
-            return cudaLaunchKernelEx(&cfg, attn_mma_kernel<8, 2>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
-                                      c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
-        return cudaLaunchKernelEx(&cfg, attn_mma_kernel<4, 2>, gm, ut, a, kvp, (const int32_t*)c->st.idx, (const int32_t*)c->st.cnt,
-                                  c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status);
+        const bool sources = a.res_rows != nullptr || a.imp_rows != nullptr;
+#define TB_MMA(NW_, ST_)                                                                                                          \
+    (sources ? cudaLaunchKernelEx(&cfg, attn_mma_kernel<NW_, ST_, true>, gm, ut, a, kvp, (const int32_t*)c->st.idx,               \
+                                  (const int32_t*)c->st.cnt, c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status)       \
+             : cudaLaunchKernelEx(&cfg, attn_mma_kernel<NW_, ST_, false>, gm, ut, a, kvp, (const int32_t*)c->st.idx,              \
+                                  (const int32_t*)c->st.cnt, c->wk.part_o, c->wk.part_ml, c->st.attn_counter, c->st.status))
+        if (nw == 12) return TB_MMA(12, 2);
+        if (nw == 8 && nst == 3) return TB_MMA(8, 3);
+        if (nw == 8) return TB_MMA(8, 2);
+        return TB_MMA(4, 2);
+#undef TB_MMA
     } else {
         TB_ATTN_G(float);
     }

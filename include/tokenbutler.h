@@ -131,8 +131,9 @@ int32_t tb_index_capacity(const tb_ctx* ctx);
  * (Sec. 3.1: learned matrix of the key-cache projection). */
 tb_status tb_set_projection(tb_ctx* ctx, int32_t layer, const void* W_dev, void* stream);
 
-/* Forget a sequence in every layer: length and projected length 0 (host mirrors and device counters, the
- * latter with a blocking clear: call it when no work on that sequence is in flight), stored selections dropped. */
+/* Forget a sequence in every layer: length and projected length 0 (host mirrors and, when the kernels read
+ * them, the device counters, with a blocking clear: call it when no work on that sequence is in flight), stored
+ * selections dropped. */
 tb_status tb_reset_sequence(tb_ctx* ctx, int32_t seq);
 
 /* Host-side view of a sequence: tokens cached and tokens whose keys are projected. */
@@ -295,7 +296,7 @@ tb_status tb_bind_important_buffer(tb_ctx* ctx, void* buf_dev, size_t bytes);
 /* Where the kernels take the sequence lengths from (Sec. 3.3 / 3.4: the cache grows by a token every decode
  * step and the window moves with it).  The context keeps the lengths twice: host mirrors, advanced when a
  * call is made, which validate arguments; and device counters, advanced by the append and projection kernels
- * themselves.  By default (on = 0) every launch carries the mirrors' values as kernel parameters: no dependent
+ * themselves while they are in use (switching them on copies the mirrors over, blocking).  By default (on = 0) every launch carries the mirrors' values as kernel parameters: no dependent
  * load at kernel start, but a captured CUDA graph then replays the lengths it was captured with.  With on = 1
  * the kernels read the device counters, so a graph captured once replays a growing sequence: capture a
  * decode step (append, projection with NULL ranges, selection, attention) and replay it every step.

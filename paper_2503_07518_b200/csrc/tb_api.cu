@@ -268,11 +268,13 @@ tb_status tb_set_projection(tb_ctx* c, int32_t layer, const void* W_dev, void* s
 
 tb_status tb_reset_sequence(tb_ctx* c, int32_t seq) {
     if (!c || seq < 0 || seq >= c->cfg.max_batch) return TB_ERR_INVALID_ARG;
-    // the device counters of this sequence, one 4-byte entry per layer (a blocking strided clear)
-    const size_t pitch = (size_t)c->cfg.max_batch * 4;
-    if (cudaMemset2D(c->st.len + seq, pitch, 0, 4, c->cfg.n_layers) != cudaSuccess ||
-        cudaMemset2D(c->st.len_proj + seq, pitch, 0, 4, c->cfg.n_layers) != cudaSuccess)
-        return TB_ERR_CUDA;
+    if (c->dev_lengths) {
+        // the device counters of this sequence, one 4-byte entry per layer (a blocking strided clear)
+        const size_t pitch = (size_t)c->cfg.max_batch * 4;
+        if (cudaMemset2D(c->st.len + seq, pitch, 0, 4, c->cfg.n_layers) != cudaSuccess ||
+            cudaMemset2D(c->st.len_proj + seq, pitch, 0, 4, c->cfg.n_layers) != cudaSuccess)
+            return TB_ERR_CUDA;
+    }
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         const size_t i = (size_t)l * c->cfg.max_batch + seq;
         c->len[i] = c->len_proj[i] = c->has_sel[i] = 0, c->sel_cnt[i] = -1;
@@ -345,15 +347,33 @@ tb_status tb_project_keys(tb_ctx* c, int32_t lb, int32_t lc, const int32_t* seq_
             if (pos_end[i] - pos_begin[i] > max_range) max_range = pos_end[i] - pos_begin[i];
         }
     }
-    const int step = layers_per_launch(n_seq);
-    for (int l0 = lb; l0 < lb + lc; l0 += step) {
-        const int n = l0 + step <= lb + lc ? step : lb + lc - l0;
-        UnitTable ut;
-        fill_table(c, &ut, l0, n, seqs, n_seq);
-        if (max_range > 0) {
-            if (launch_project(c, ut, pos_begin, pos_end, max_range, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+    if (auto_range && !c->dev_lengths) {
+        // lengths are the host's: the ranges are worked out here, layer by layer (they may differ between layers)
+        for (int l = lb; l < lb + lc; ++l) {
+            int b[kMaxLaunchSeq], e[kMaxLaunchSeq], mr = 0;
+            for (int i = 0; i < n_seq; ++i) {
+                const size_t u = (size_t)l * c->cfg.max_batch + seqs[i];
+                b[i] = c->len_proj[u], e[i] = c->len[u] > c->len_proj[u] ? c->len[u] : c->len_proj[u];
+                if (e[i] - b[i] > mr) mr = e[i] - b[i];
+            }
+            if (mr == 0) continue;
+            UnitTable ut;
+            fill_table(c, &ut, l, 1, seqs, n_seq);
+            if (launch_project(c, ut, b, e, mr, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
             c->last_cache_write = (long long)c->launches;
             c->launches++;
+        }
+    } else {
+        const int step = layers_per_launch(n_seq);
+        for (int l0 = lb; l0 < lb + lc; l0 += step) {
+            const int n = l0 + step <= lb + lc ? step : lb + lc - l0;
+            UnitTable ut;
+            fill_table(c, &ut, l0, n, seqs, n_seq);
+            if (max_range > 0) {
+                if (launch_project(c, ut, pos_begin, pos_end, max_range, (cudaStream_t)stream) != cudaSuccess) return TB_ERR_CUDA;
+                c->last_cache_write = (long long)c->launches;
+                c->launches++;
+            }
         }
     }
     for (int l = lb; l < lb + lc; ++l)
@@ -588,6 +608,13 @@ tb_status tb_bind_important_buffer(tb_ctx* c, void* buf_dev, size_t bytes) {
 
 tb_status tb_use_device_lengths(tb_ctx* c, int32_t on, int32_t growth_reserve) {
     if (!c || growth_reserve < 0) return TB_ERR_INVALID_ARG;
+    if (on && !c->dev_lengths) {
+        // the counters are only kept while they are read: bring them up to the mirrors (blocking copies)
+        const size_t n = (size_t)c->cfg.n_layers * c->cfg.max_batch * 4;
+        if (cudaMemcpy(c->st.len, c->len.data(), n, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(c->st.len_proj, c->len_proj.data(), n, cudaMemcpyHostToDevice) != cudaSuccess)
+            return TB_ERR_CUDA;
+    }
     c->dev_lengths = on ? 1 : 0;
     c->growth_reserve = on ? growth_reserve : 0;
     return TB_OK;

@@ -58,7 +58,9 @@ __global__ void append_kernel(Geom gm, UnitTable ut, AppendTable at, int total_n
             }
         }
     }
-    if (last_block_arrives(counter, gridDim.x * gridDim.y)) {
+    // (only when the kernels read the device counters: otherwise the host's mirrors carry the lengths and
+    // the counters are brought up to date when that mode is switched on)
+    if (ut.use_dev_len && last_block_arrives(counter, gridDim.x * gridDim.y)) {
         for (int i = threadIdx.x; i < ut.layer_count * ut.n_seq; i += blockDim.x) {
             const int l2 = i / ut.n_seq, s2 = i % ut.n_seq;
             const size_t pair = (size_t)(ut.layer_begin + l2) * gm.max_batch + ut.seq_id[s2];
@@ -150,7 +152,7 @@ __device__ __forceinline__ void project_range(const Geom& gm, const UnitTable& u
 // The last block of a projection launch to finish advances the device counters of the projected lengths.
 __device__ __forceinline__ void project_finish(const Geom& gm, const UnitTable& ut, const ProjectTable& pt, int32_t* len_proj_dev,
                                                uint32_t* counter) {
-    if (!last_block_arrives(counter, gridDim.x * gridDim.y * gridDim.z)) return;
+    if (!ut.use_dev_len || !last_block_arrives(counter, gridDim.x * gridDim.y * gridDim.z)) return;
     for (int i = threadIdx.x; i < ut.layer_count * ut.n_seq; i += blockDim.x) {
         int b, e;
         project_range(gm, ut, pt, i / ut.n_seq, i % ut.n_seq, b, e);

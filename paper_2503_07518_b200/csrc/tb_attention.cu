@@ -650,44 +650,50 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     }
     attn_stamp(5);
     if (a.cluster_merge) {
+        // Merge of the blocks' results inside the cluster, sliced by channels: the 128 channels are eight slices
+        // of 16, slice j belongs to block j mod C.  Every block sends each slice of its (o) to the slice's owner
+        // and its (m, l) to every owner -- 2 KB per block in all --, one cluster barrier, and every owner merges
+        // its 16 channels of all heads from the C partials (blocks in rank order: bit-reproducible) and writes
+        // them out.  No single merging block: the work behind the barrier is C terms per output, not C x 8.
         cg::cluster_group cluster = cg::this_cluster();
         const int rank = (int)cluster.block_rank(), C = (int)cluster.num_blocks();
-        float* area = reinterpret_cast<float*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [C][g][kMergePitch]
-        float* area0 = cluster.map_shared_rank(area, 0);
+        const int T = (8 + C - 1) / C;                               // slices per owner
+        float* area = reinterpret_cast<float*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [T][C][g][16]
+        float* ml = area + (size_t)T * C * g * 16;                   // [C][g][2]
         if (tid < D) {
+            const int j = tid >> 4, cc = tid & 15;
+            float* dst = cluster.map_shared_rank(area, j % C) + ((size_t)((j / C) * C + rank) * g) * 16 + cc;
 #pragma unroll
             for (int u = 0; u < kMaxGroup; ++u)
-                if (u < g) {
-                    float* slot = area0 + (size_t)(rank * g + u) * kMergePitch;
-                    slot[tid] = cO[u];
-                    if (tid == 0) slot[D] = cM[u], slot[D + 1] = cL[u];
-                }
+                if (u < g) dst[u * 16] = cO[u];
+        }
+        if (tid < g) {                                               // cM / cL are the same in every thread with tid < D: thread u sends head u's
+            float mu = 0.f, lu_ = 0.f;
+#pragma unroll
+            for (int u = 0; u < kMaxGroup; ++u)
+                if (u == tid) mu = cM[u], lu_ = cL[u];
+            for (int r = 0; r < C && r < 8; ++r) {
+                float* d2 = cluster.map_shared_rank(ml, r) + ((size_t)rank * g + tid) * 2;
+                d2[0] = mu, d2[1] = lu_;
+            }
         }
         cluster.sync();
-        if (rank == 0) {
-            __shared__ float cw[kAttnMaxCluster][kMaxGroup], cMx[kMaxGroup];
-            if (tid < C * kMaxGroup) {
-                const int r = tid / kMaxGroup, u = tid % kMaxGroup;
-                if (u < g) {
-                    float M = -INFINITY;
-                    for (int x = 0; x < C; ++x) M = fmaxf(M, area[(size_t)(x * g + u) * kMergePitch + D]);
-                    cw[r][u] = exp2f(area[(size_t)(r * g + u) * kMergePitch + D] - (M == -INFINITY ? 0.f : M));
-                    if (r == 0) cMx[u] = M;
+        if (rank < 8) {
+            for (int i = tid; i < T * g * 16; i += NW * 32) {
+                const int ts = i / (g * 16), u = (i / 16) % g, cc = i & 15;
+                const int j = ts * C + rank;                         // the slice
+                if (j >= 8) continue;
+                float M = -INFINITY;
+                for (int r = 0; r < C; ++r) M = fmaxf(M, ml[(r * g + u) * 2]);
+                const float Ms = M == -INFINITY ? 0.f : M;
+                float lsum = 0.f, acc = 0.f;
+                for (int r = 0; r < C; ++r) {
+                    const float e = exp2f(ml[(r * g + u) * 2] - Ms);
+                    lsum = fmaf(ml[(r * g + u) * 2 + 1], e, lsum);
+                    acc = fmaf(area[((size_t)(ts * C + r) * g + u) * 16 + cc], e, acc);
                 }
-            }
-            __syncthreads();
-            if (tid < D) {
-                for (int u = 0; u < g; ++u) {
-                    float lsum = 0.f, acc = 0.f;
-                    for (int r = 0; r < C; ++r) {
-                        const float* slot = area + (size_t)(r * g + u) * kMergePitch;
-                        const float e = cw[r][u];
-                        lsum += slot[D + 1] * e;
-                        acc = fmaf(slot[tid], e, acc);
-                    }
-                    a.out[(hq0 + u) * D + tid] = acc / lsum;
-                    if (a.lse && tid == 0) a.lse[hq0 + u] = (cMx[u] + log2f(lsum)) * kLn2;
-                }
+                a.out[(hq0 + u) * D + j * 16 + cc] = acc / lsum;
+                if (a.lse && j == 0 && cc == 0) a.lse[hq0 + u] = (M + log2f(lsum)) * kLn2;
             }
         }
     } else if constexpr (NW == kAttnWarps) {

@@ -202,6 +202,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
     int* merged_late = reinterpret_cast<int*>(stage_base);                        // 2 * kBins ints
     uint32_t* mask = reinterpret_cast<uint32_t*>(stage_base);                     // one bit per local slot: up to 4 KB
     uint2* cand = reinterpret_cast<uint2*>(stage_base + kMaxKeysPerBlock / 8);    // kFastCand (key, candidate index) pairs
+    uint2* cand_mine = cand + kFastCand;                                          // this block's own, before they are sent
 
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
@@ -477,11 +478,14 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const __grid_consta
                 while (eqm) {                          // rare: a handful of keys per block
                     const int e = __ffs(eqm) - 1;
                     eqm &= eqm - 1;
-                    const int i = cand_base + atomicAdd(&sm->n_cand, 1);
-                    const uint2 ent = make_uint2(kk[e], (uint32_t)(slot0 + v * 4 + e));
-                    for (int r = 0; r < C; ++r) *cluster.map_shared_rank(&cand[i], (rank + r) % C) = ent;
+                    cand_mine[atomicAdd(&sm->n_cand, 1)] = make_uint2(kk[e], (uint32_t)(slot0 + v * 4 + e));
                 }
             }
+            // ... sent to every block's list one (entry, peer) pair per thread: remote stores issued one after
+            // the other by the thread that found the key held its whole warp up
+            __syncthreads();
+            for (int t = tid; t < sm->n_cand * C; t += kSelThreads)
+                *cluster.map_shared_rank(&cand[cand_base + t / C], (rank + t % C) % C) = cand_mine[t / C];
             phase_stamp(11);
             if (C > 1) cluster.sync(); else __syncthreads();   // barrier 2: the list is complete everywhere
             // What is left is short and local.  A successor launched as a programmatic dependent (the first

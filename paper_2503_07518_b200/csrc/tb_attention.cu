@@ -326,13 +326,14 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
 
 #ifdef TB_PHASE_TIMING
 __device__ unsigned long long g_attn_phase_ns[2][16];
-__device__ unsigned long long g_attn_blk_ns[7][1024];   // per block of the last launch: every stamp
-__device__ __forceinline__ void attn_stamp(int i) {
+__device__ unsigned long long g_attn_blk_ns[2][8][1024];   // per block of the last launches on an even and on an odd layer: every stamp
+#define attn_stamp(i) attn_stamp_((i), ut.layer_begin & 1)
+__device__ __forceinline__ void attn_stamp_(int i, int par) {
     if (threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         const int b = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        if (b < 1024 && i < 7) g_attn_blk_ns[i][b] = t;
+        if (b < 1024 && i < 8) g_attn_blk_ns[par][i][b] = t;
     }
     if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
         unsigned long long t;
@@ -347,7 +348,7 @@ extern "C" int tb_debug_attn_blocks_ns(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, g_attn_blk_ns, sizeof(g_attn_blk_ns));
 }
 #else
-__device__ __forceinline__ void attn_stamp(int) {}
+#define attn_stamp(i) ((void)0)
 #endif
 
 constexpr int kTileTok = 16;
@@ -382,10 +383,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// One of the block's 16 hardware barriers (0 is __syncthreads'), met by `count` threads; orders their shared-memory accesses.
+__device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+
+// Shared memory behind the warps' stages for the merge inside a cluster of C blocks: the accumulator slices this
+// block owns from every block ([slices per owner][C][32 lanes] float4) and every block's (m, l) ([C][4] float4).
+static inline size_t cluster_merge_bytes(int C) { return (size_t)((8 + C - 1) / C) * C * 32 * 16 + (size_t)C * 4 * 16; }
+
 // NW warps per block.  With a.cluster_merge the blocks of one (sequence, KV head) form a thread-block
-// cluster (one block per split): every block writes its (m, l, o) into rank 0's shared memory through
-// distributed shared memory, one cluster barrier, and rank 0 merges in rank order -- no partials in
-// global memory, no last-block round trips.  Without it (more splits than a cluster holds) the splits
+// cluster (one block per split): the warps of a block fold their results in a tree, the blocks exchange
+// channel slices of theirs through distributed shared memory, one cluster barrier, and every block merges
+// and writes the slices it owns -- no partials in global memory, no last-block round trips.  Without it (more splits than a cluster holds) the splits
 // go through the global workspace and the last block to arrive merges them (NW must be 4 then).
 // kSources: the resident sink / window copies or the Important buffer are bound and a row reference names
 // its source; without them (the usual case) the gather carries no trace of the option.
@@ -436,9 +444,11 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const int r_begin = (int)((long long)n_rows * split / a.nsplit);
     const int r_end = (int)((long long)n_rows * (split + 1) / a.nsplit);
     const int tiles_all = (r_end - r_begin + kTileTok - 1) / kTileTok;
-    const int tiles_per_warp = (tiles_all + NW - 1) / NW;
-    const int wb = min(r_end, r_begin + warp * tiles_per_warp * kTileTok);
-    const int we = min(r_end, wb + tiles_per_warp * kTileTok);
+    // dealt evenly: no warp gets more than one tile above another (a tile beyond a warp's stages waits for
+    // a stage to drain and then for its rows, a whole memory latency)
+    const int tiles_lo = tiles_all / NW, tiles_rem = tiles_all % NW;
+    const int wb = min(r_end, r_begin + (warp * tiles_lo + min(warp, tiles_rem)) * kTileTok);
+    const int we = min(r_end, wb + (tiles_lo + (warp < tiles_rem ? 1 : 0)) * kTileTok);
     const int n_tiles = (we - wb + kTileTok - 1) / kTileTok;
 
     unsigned char* my_stage = smem_dyn + (size_t)warp * kMmaStages * kStageBytes;
@@ -496,6 +506,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     attn_stamp(2);
 
     if (a.early_ok) pdl_wait();                        // the queries are this call's input
+    attn_stamp(7);
     // Q^T as the B operand of S = K Q^T: k = channels, n = query heads (gid; heads >= g are zero padding)
     uint32_t qb[8][2];
     {
@@ -600,7 +611,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     if (any_bad && lane < kTileTok) atomicExch(status, kStatusBadIndex);
 
-    // ---- warp result -> shared (reusing the warp's own stages), block combine, publish ------------------
+    // ---- the warps' results become the block's, the blocks' the problem's -------------------------------
     attn_stamp(4);
 #pragma unroll
     for (int off = 4; off < 32; off <<= 1) {
@@ -608,95 +619,133 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
         l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
     }
     __syncwarp();
-    float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][kMergePitch]
-#pragma unroll
-    for (int mt = 0; mt < 8; ++mt) {
-        wo[(2 * tig) * kMergePitch + mt * 16 + gid] = o[mt][0];          // pitch 132: the 32 lanes hit 32 banks
-        wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid] = o[mt][1];
-        wo[(2 * tig) * kMergePitch + mt * 16 + gid + 8] = o[mt][2];
-        wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid + 8] = o[mt][3];
-    }
-    if (gid == 0) {
-        sh_m[warp][2 * tig] = m_run[0], sh_l[warp][2 * tig] = l_run[0];
-        sh_m[warp][2 * tig + 1] = m_run[1], sh_l[warp][2 * tig + 1] = l_run[1];
-    }
-    __syncthreads();
     const size_t hq0 = (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g;
-    // weights 2^(m_w - M) of every (warp, head), computed once by NW*8 threads
-    __shared__ float sh_w[NW][kMaxGroup], sh_M[kMaxGroup];
-    if (tid < NW * kMaxGroup) {
-        const int w = tid / kMaxGroup, u = tid % kMaxGroup;
-        float M = -INFINITY;
-#pragma unroll
-        for (int x = 0; x < NW; ++x) M = fmaxf(M, sh_m[x][u]);
-        sh_w[w][u] = exp2f(sh_m[w][u] - (M == -INFINITY ? 0.f : M));
-        if (w == 0) sh_M[u] = M;
-    }
-    __syncthreads();
-    float cM[kMaxGroup], cL[kMaxGroup], cO[kMaxGroup];        // block result per head; cO: channel tid (tid < 128)
-#pragma unroll
-    for (int u = 0; u < kMaxGroup; ++u) {
-        cM[u] = -INFINITY, cL[u] = 0.f, cO[u] = 0.f;
-        if (u < g && tid < D) {
-            float lsum = 0.f, acc = 0.f;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float e = sh_w[w][u];
-                lsum += sh_l[w][u] * e;
-                acc = fmaf(reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * kMergePitch + tid], e, acc);
-            }
-            cM[u] = sh_M[u], cL[u] = lsum, cO[u] = acc;
-        }
-    }
-    attn_stamp(5);
     if (a.cluster_merge) {
+        // Block result: a binary tree over the warps.  At every level the upper half of the remaining warps
+        // parks its accumulators in its own (drained) stages, lane by lane in the MMA layout, and the partner
+        // in the lower half folds them into its registers -- same lane, same elements, so nothing is
+        // transposed and a level costs 9 conflict-free 16-byte stores and loads per lane.  Each pair meets at a
+        // named barrier of its own (64 threads); the order of the folds is fixed, so the result is
+        // bit-reproducible.  (A flat combine -- every warp's result to shared memory, two block barriers,
+        // 128 threads summing NW terms per head -- was 0.12 us slower per launch.)
+        static_assert(NW <= 16, "the named barriers below are numbered 1..15: 8, 4, 2 and 1 pairs per level");
+        float4* tbuf = reinterpret_cast<float4*>(my_stage);             // [8][32] o, then [32] (m0, l0, m1, l1)
+        constexpr int kTop = NW > 8 ? 8 : NW > 4 ? 4 : NW > 2 ? 2 : 1;
+#pragma unroll
+        for (int stride = kTop; stride >= 1; stride >>= 1) {
+            if (warp >= stride && warp < 2 * stride) {
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) tbuf[mt * 32 + lane] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+                tbuf[8 * 32 + lane] = make_float4(m_run[0], l_run[0], m_run[1], l_run[1]);
+                named_bar_sync(17 - 2 * stride + (warp - stride), 64);
+            } else if (warp < stride && warp + stride < NW) {
+                named_bar_sync(17 - 2 * stride + warp, 64);
+                const float4* pb = reinterpret_cast<const float4*>(smem_dyn + (size_t)(warp + stride) * kMmaStages * kStageBytes);
+                const float4 pm = pb[8 * 32 + lane];
+                const float M0 = fmaxf(m_run[0], pm.x), M1 = fmaxf(m_run[1], pm.z);
+                const float M0s = M0 == -INFINITY ? 0.f : M0, M1s = M1 == -INFINITY ? 0.f : M1;
+                const float ea0 = exp2f(m_run[0] - M0s), eb0 = exp2f(pm.x - M0s);
+                const float ea1 = exp2f(m_run[1] - M1s), eb1 = exp2f(pm.z - M1s);
+                l_run[0] = fmaf(pm.y, eb0, l_run[0] * ea0), l_run[1] = fmaf(pm.w, eb1, l_run[1] * ea1);
+                m_run[0] = M0, m_run[1] = M1;
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    const float4 v = pb[mt * 32 + lane];
+                    o[mt][0] = fmaf(v.x, eb0, o[mt][0] * ea0), o[mt][1] = fmaf(v.y, eb1, o[mt][1] * ea1);
+                    o[mt][2] = fmaf(v.z, eb0, o[mt][2] * ea0), o[mt][3] = fmaf(v.w, eb1, o[mt][3] * ea1);
+                }
+            }
+        }
+        attn_stamp(5);
         // Merge of the blocks' results inside the cluster, sliced by channels: the 128 channels are eight slices
-        // of 16, slice j belongs to block j mod C.  Every block sends each slice of its (o) to the slice's owner
-        // and its (m, l) to every owner -- 2 KB per block in all --, one cluster barrier, and every owner merges
-        // its 16 channels of all heads from the C partials (blocks in rank order: bit-reproducible) and writes
-        // them out.  No single merging block: the work behind the barrier is C terms per output, not C x 8.
+        // of 16 (one accumulator tile of the MMA layout each), slice j belongs to block j mod C.  Warp 0 of every
+        // block sends each slice of its (o) to the slice's owner and its (m, l) to every owner -- 4.5 KB per block
+        // in all --, one cluster barrier, and every owner merges its 16 channels of all heads from the C partials
+        // (blocks in rank order: bit-reproducible) and writes them out.  No single merging block: the work behind
+        // the barrier is C terms per output, not C x 8.
         cg::cluster_group cluster = cg::this_cluster();
         const int rank = (int)cluster.block_rank(), C = (int)cluster.num_blocks();
         const int T = (8 + C - 1) / C;                               // slices per owner
-        float* area = reinterpret_cast<float*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [T][C][g][16]
-        float* ml = area + (size_t)T * C * g * 16;                   // [C][g][2]
-        if (tid < D) {
-            const int j = tid >> 4, cc = tid & 15;
-            float* dst = cluster.map_shared_rank(area, j % C) + ((size_t)((j / C) * C + rank) * g) * 16 + cc;
+        float4* area = reinterpret_cast<float4*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [T][C][32 lanes]
+        float4* ml = area + (size_t)T * C * 32;                      // [C][4]: (m, l) of heads 2 tig, 2 tig + 1
+        if (warp == 0) {
 #pragma unroll
-            for (int u = 0; u < kMaxGroup; ++u)
-                if (u < g) dst[u * 16] = cO[u];
-        }
-        if (tid < g) {                                               // cM / cL are the same in every thread with tid < D: thread u sends head u's
-            float mu = 0.f, lu_ = 0.f;
-#pragma unroll
-            for (int u = 0; u < kMaxGroup; ++u)
-                if (u == tid) mu = cM[u], lu_ = cL[u];
-            for (int r = 0; r < C && r < 8; ++r) {
-                float* d2 = cluster.map_shared_rank(ml, r) + ((size_t)rank * g + tid) * 2;
-                d2[0] = mu, d2[1] = lu_;
-            }
+            for (int mt = 0; mt < 8; ++mt)
+                cluster.map_shared_rank(area, mt % C)[((mt / C) * C + rank) * 32 + lane] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+            if (gid < C) cluster.map_shared_rank(ml, gid)[rank * 4 + tig] = make_float4(m_run[0], l_run[0], m_run[1], l_run[1]);
         }
         cluster.sync();
         if (rank < 8) {
-            for (int i = tid; i < T * g * 16; i += NW * 32) {
-                const int ts = i / (g * 16), u = (i / 16) % g, cc = i & 15;
+            for (int i = tid; i < T * 32; i += NW * 32) {
+                const int ts = i >> 5, ln = i & 31, tg = ln & 3, gd = ln >> 2;
                 const int j = ts * C + rank;                         // the slice
                 if (j >= 8) continue;
-                float M = -INFINITY;
-                for (int r = 0; r < C; ++r) M = fmaxf(M, ml[(r * g + u) * 2]);
-                const float Ms = M == -INFINITY ? 0.f : M;
-                float lsum = 0.f, acc = 0.f;
+                float M0 = -INFINITY, M1 = -INFINITY;
+                for (int r = 0; r < C; ++r) M0 = fmaxf(M0, ml[r * 4 + tg].x), M1 = fmaxf(M1, ml[r * 4 + tg].z);
+                const float M0s = M0 == -INFINITY ? 0.f : M0, M1s = M1 == -INFINITY ? 0.f : M1;
+                float ls0 = 0.f, ls1 = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int r = 0; r < C; ++r) {
-                    const float e = exp2f(ml[(r * g + u) * 2] - Ms);
-                    lsum = fmaf(ml[(r * g + u) * 2 + 1], e, lsum);
-                    acc = fmaf(area[((size_t)(ts * C + r) * g + u) * 16 + cc], e, acc);
+                    const float4 q = ml[r * 4 + tg];
+                    const float e0 = exp2f(q.x - M0s), e1 = exp2f(q.z - M1s);
+                    ls0 = fmaf(q.y, e0, ls0), ls1 = fmaf(q.w, e1, ls1);
+                    const float4 v = area[(ts * C + r) * 32 + ln];
+                    acc.x = fmaf(v.x, e0, acc.x), acc.y = fmaf(v.y, e1, acc.y);
+                    acc.z = fmaf(v.z, e0, acc.z), acc.w = fmaf(v.w, e1, acc.w);
                 }
-                a.out[(hq0 + u) * D + j * 16 + cc] = acc / lsum;
-                if (a.lse && j == 0 && cc == 0) a.lse[hq0 + u] = (M + log2f(lsum)) * kLn2;
+                const int u0 = 2 * tg, u1 = u0 + 1, ch = j * 16 + gd;
+                if (u0 < g) {
+                    a.out[(hq0 + u0) * D + ch] = acc.x / ls0, a.out[(hq0 + u0) * D + ch + 8] = acc.z / ls0;
+                    if (a.lse && j == 0 && gd == 0) a.lse[hq0 + u0] = (M0 + log2f(ls0)) * kLn2;
+                }
+                if (u1 < g) {
+                    a.out[(hq0 + u1) * D + ch] = acc.y / ls1, a.out[(hq0 + u1) * D + ch + 8] = acc.w / ls1;
+                    if (a.lse && j == 0 && gd == 0) a.lse[hq0 + u1] = (M1 + log2f(ls1)) * kLn2;
+                }
             }
         }
     } else if constexpr (NW == kAttnWarps) {
+        // splits through the global workspace: flat combine into one channel per thread, then the sink
+        float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][kMergePitch]
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+            wo[(2 * tig) * kMergePitch + mt * 16 + gid] = o[mt][0];          // pitch 132: the 32 lanes hit 32 banks
+            wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid] = o[mt][1];
+            wo[(2 * tig) * kMergePitch + mt * 16 + gid + 8] = o[mt][2];
+            wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid + 8] = o[mt][3];
+        }
+        if (gid == 0) {
+            sh_m[warp][2 * tig] = m_run[0], sh_l[warp][2 * tig] = l_run[0];
+            sh_m[warp][2 * tig + 1] = m_run[1], sh_l[warp][2 * tig + 1] = l_run[1];
+        }
+        __syncthreads();
+        // weights 2^(m_w - M) of every (warp, head), computed once by NW*8 threads
+        __shared__ float sh_w[NW][kMaxGroup], sh_M[kMaxGroup];
+        if (tid < NW * kMaxGroup) {
+            const int w = tid / kMaxGroup, u = tid % kMaxGroup;
+            float M = -INFINITY;
+#pragma unroll
+            for (int x = 0; x < NW; ++x) M = fmaxf(M, sh_m[x][u]);
+            sh_w[w][u] = exp2f(sh_m[w][u] - (M == -INFINITY ? 0.f : M));
+            if (w == 0) sh_M[u] = M;
+        }
+        __syncthreads();
+        float cM[kMaxGroup], cL[kMaxGroup], cO[kMaxGroup];        // block result per head; cO: channel tid (tid < 128)
+#pragma unroll
+        for (int u = 0; u < kMaxGroup; ++u) {
+            cM[u] = -INFINITY, cL[u] = 0.f, cO[u] = 0.f;
+            if (u < g && tid < D) {
+                float lsum = 0.f, acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) {
+                    const float e = sh_w[w][u];
+                    lsum += sh_l[w][u] * e;
+                    acc = fmaf(reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * kMergePitch + tid], e, acc);
+                }
+                cM[u] = sh_M[u], cL[u] = lsum, cO[u] = acc;
+            }
+        }
+        attn_stamp(5);
         SplitSink sink{part_o, part_ml, counters, a.out, a.lse, hq0, lu, split, a.nsplit};
 #pragma unroll
         for (int u = 0; u < kMaxGroup; ++u)
@@ -755,7 +804,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             if (max_active[csize] == 0) {
                 cudaLaunchConfig_t q = {};
                 q.gridDim = dim3(csize, 1, 1), q.blockDim = dim3(256, 1, 1);
-                const size_t mb = (size_t)csize * gm.ga * 132 * sizeof(float);
+                const size_t mb = cluster_merge_bytes(csize);
                 const bool three = csize <= 8 && 8 * 3 * kStageBytes + mb <= 220 * 1024;
                 q.dynamicSmemBytes = 8 * (three ? 3 : 2) * kStageBytes + mb;
                 cudaLaunchAttribute at[1];
@@ -796,7 +845,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
             // more than two tiles per warp would leave the third waiting for a free stage: 12 warps
             // per block when their rings and the merge area still fit the SM
             const int rows_per_block = (max_rows + n - 1) / n;
-            if (rows_per_block > 8 * 2 * kTileTok && 12 * 2 * kStageBytes + (size_t)n * gm.ga * 132 * sizeof(float) <= 224 * 1024) nw = 12;
+            if (rows_per_block > 8 * 2 * kTileTok && 12 * 2 * kStageBytes + cluster_merge_bytes(n) <= 224 * 1024) nw = 12;
         } else {
             a.nsplit = pick_nsplit(c, units, max_rows);
             // clusters only when the whole launch is resident at once: in multi-wave launches the
@@ -818,7 +867,7 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         else TB_ATTN(T, 8);                           \
     } while (0)
     if (gm.dtype == TB_BF16) {
-        const size_t merge_bytes = a.cluster_merge ? (size_t)a.nsplit * gm.ga * 132 * sizeof(float) : 0;
+        const size_t merge_bytes = a.cluster_merge ? cluster_merge_bytes(a.nsplit) : 0;
         // three stages per warp when the 8-warp block still fits the SM with them
         const int nst = (nw == 8 && 8 * 3 * kStageBytes + merge_bytes <= 220 * 1024 && a.nsplit <= 8) ? 3 : 2;
         const size_t smem = (size_t)nw * nst * kStageBytes + merge_bytes;

@@ -326,14 +326,16 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
 
 #ifdef TB_PHASE_TIMING
 __device__ unsigned long long g_attn_phase_ns[2][16];
-__device__ unsigned long long g_attn_blk_ns[2][8][1024];   // per block of the last launches on an even and on an odd layer: every stamp
+__device__ unsigned long long g_attn_blk_ns[2][12][1024];   // per block of the last launches on an even and on an odd layer: every stamp
+__device__ long long g_attn_blk_clk[2][12][1024];            // the same stamps in SM cycles (differences inside one block only)
 #define attn_stamp(i) attn_stamp_((i), ut.layer_begin & 1)
 __device__ __forceinline__ void attn_stamp_(int i, int par) {
     if (threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         const int b = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        if (b < 1024 && i < 8) g_attn_blk_ns[par][i][b] = t;
+        if (b < 1024 && i < 12) g_attn_blk_ns[par][i][b] = t;
+        if (b < 1024 && i < 12) g_attn_blk_clk[par][i][b] = clock64();
     }
     if (threadIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) {
         unsigned long long t;
@@ -343,6 +345,9 @@ __device__ __forceinline__ void attn_stamp_(int i, int par) {
 }
 extern "C" int tb_debug_attn_phase_ns(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, g_attn_phase_ns, sizeof(g_attn_phase_ns));
+}
+extern "C" int tb_debug_attn_blocks_clk(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_attn_blk_clk, sizeof(g_attn_blk_clk));
 }
 extern "C" int tb_debug_attn_blocks_ns(unsigned long long* out) {
     return (int)cudaMemcpyFromSymbol(out, g_attn_blk_ns, sizeof(g_attn_blk_ns));
@@ -521,6 +526,10 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
         }
     }
     const float qscale = a.sm_scale * kLog2e;
+#ifdef TB_PHASE_TIMING
+    if (qb[7][1] == 0x7fc1dead) any_bad = true;            // the stamp below waits for the queries
+    attn_stamp(8);
+#endif
 
     // O^T accumulators: 8 tiles of (16 channels x 8 heads); this thread: channels mt*16 + gid (+8),
     // heads 2*tig and 2*tig+1 -- the same two heads as its columns of S.
@@ -536,7 +545,75 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const uint32_t k_row_off = ((mi & 1) * 8 + r8) * kRowPitch, k_swz = (uint32_t)((mi >> 1) ^ r8) << 4;        // ^ ks * 32   (A of S = K Q^T)
     const uint32_t v_row_off = ((mi >> 1) * 8 + r8) * kRowPitch + 256, v_swz = (uint32_t)((mi & 1) ^ r8) << 4;  // ^ mt * 32   (A of O^T = V^T P^T)
 
-    for (int tile = 0; tile < n_tiles; ++tile) {
+    // A warp whose rows all fit its stages (two or three tiles: the latency-bound launches, where a block holds a
+    // few hundred rows) takes its first two tiles as one 32-token tile: the two S = K Q^T chains interleave, there
+    // is one softmax update instead of two, and every O^T accumulator gets four MMAs behind two loads.  One tile
+    // at a time is a chain of ~1500 dependent cycles per tile with nothing to overlap it in the warp.
+    int tile_first = 0;
+    if (n_tiles >= 2 && n_tiles <= kMmaStages) {
+        const bool inA = lane < kTileTok && wb + lane < we, inB = lane < kTileTok && wb + kTileTok + lane < we;
+        const bool badA = inA && (bad_bits & 1u), badB = inB && (bad_bits & 2u);
+        any_bad |= badA | badB;
+        bad_bits >>= 2;
+        const unsigned vmA = __ballot_sync(0xffffffffu, inA && !badA), vmB = __ballot_sync(0xffffffffu, inB && !badB);
+        asm volatile("cp.async.wait_group %0;" ::"n"(kMmaStages - 2) : "memory");
+        __syncwarp();
+        attn_stamp(3);
+        const uint32_t sA = stage_u32, sB = stage_u32 + kStageBytes;
+        float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
+            ldmatrix_x4(sA + k_row_off + ((ks * 32) ^ k_swz), a0, a1, a2, a3);
+            ldmatrix_x4(sB + k_row_off + ((ks * 32) ^ k_swz), b0, b1, b2, b3);
+            mma_bf16(ca, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            mma_bf16(cb, b0, b1, b2, b3, qb[ks][0], qb[ks][1]);
+        }
+        const bool vA0 = (vmA >> gid) & 1u, vA1 = (vmA >> (gid + 8)) & 1u, vB0 = (vmB >> gid) & 1u, vB1 = (vmB >> (gid + 8)) & 1u;
+        float x[8];
+        x[0] = vA0 ? ca[0] * qscale : -INFINITY, x[1] = vA0 ? ca[1] * qscale : -INFINITY;
+        x[2] = vA1 ? ca[2] * qscale : -INFINITY, x[3] = vA1 ? ca[3] * qscale : -INFINITY;
+        x[4] = vB0 ? cb[0] * qscale : -INFINITY, x[5] = vB0 ? cb[1] * qscale : -INFINITY;
+        x[6] = vB1 ? cb[2] * qscale : -INFINITY, x[7] = vB1 ? cb[3] * qscale : -INFINITY;
+        float tmax[2] = {fmaxf(fmaxf(x[0], x[2]), fmaxf(x[4], x[6])), fmaxf(fmaxf(x[1], x[3]), fmaxf(x[5], x[7]))};
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+            tmax[0] = fmaxf(tmax[0], __shfl_xor_sync(0xffffffffu, tmax[0], off));
+            tmax[1] = fmaxf(tmax[1], __shfl_xor_sync(0xffffffffu, tmax[1], off));
+        }
+        // these are the warp's first rows: nothing accumulated yet to rescale
+        m_run[0] = tmax[0], m_run[1] = tmax[1];
+        const float ms0 = tmax[0] == -INFINITY ? 0.f : tmax[0], ms1 = tmax[1] == -INFINITY ? 0.f : tmax[1];
+        float p[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) p[i] = exp2f(x[i] - ((i & 1) ? ms1 : ms0));
+        l_run[0] = (p[0] + p[2]) + (p[4] + p[6]);
+        l_run[1] = (p[1] + p[3]) + (p[5] + p[7]);
+        float ph[8], pl[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            ph[i] = __bfloat162float(__float2bfloat16_rn(p[i]));
+            pl[i] = p[i] - ph[i];
+        }
+        const uint32_t hA0 = movmatrix_trans(pack_bf16(ph[0], ph[1])), hA1 = movmatrix_trans(pack_bf16(ph[2], ph[3]));
+        const uint32_t lA0 = movmatrix_trans(pack_bf16(pl[0], pl[1])), lA1 = movmatrix_trans(pack_bf16(pl[2], pl[3]));
+        const uint32_t hB0 = movmatrix_trans(pack_bf16(ph[4], ph[5])), hB1 = movmatrix_trans(pack_bf16(ph[6], ph[7]));
+        const uint32_t lB0 = movmatrix_trans(pack_bf16(pl[4], pl[5])), lB1 = movmatrix_trans(pack_bf16(pl[6], pl[7]));
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+            uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
+            ldmatrix_x4_trans(sA + v_row_off + ((mt * 32) ^ v_swz), a0, a1, a2, a3);
+            ldmatrix_x4_trans(sB + v_row_off + ((mt * 32) ^ v_swz), b0, b1, b2, b3);
+            mma_bf16(o[mt], a0, a1, a2, a3, hA0, hA1);
+            mma_bf16(o[mt], a0, a1, a2, a3, lA0, lA1);
+            mma_bf16(o[mt], b0, b1, b2, b3, hB0, hB1);
+            mma_bf16(o[mt], b0, b1, b2, b3, lB0, lB1);
+        }
+        __syncwarp();
+        commit(), commit();                            // the two tile slots' groups of the loop below
+        tile_first = 2;
+    }
+    for (int tile = tile_first; tile < n_tiles; ++tile) {
         const int st = tile % kMmaStages;
         const int r0 = wb + tile * kTileTok;
         // validity of the tile's 16 rows (past-the-end and out-of-range list entries are masked)
@@ -558,6 +635,9 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
             ldmatrix_x4(sb + k_row_off + ((ks * 32) ^ k_swz), a0, a1, a2, a3);
             mma_bf16(sc, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
         }
+#ifdef TB_PHASE_TIMING
+        if (tile == 0) { if (sc[0] == 1.2345e33f) any_bad = true; attn_stamp(9); }
+#endif
         const bool v0 = (vmask >> gid) & 1u, v1 = (vmask >> (gid + 8)) & 1u;
         float x[4];
         x[0] = v0 ? sc[0] * qscale : -INFINITY, x[1] = v0 ? sc[1] * qscale : -INFINITY;
@@ -600,6 +680,9 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
             mma_bf16(o[mt], a0, a1, a2, a3, bh0, bh1);
             mma_bf16(o[mt], a0, a1, a2, a3, bl0, bl1);
         }
+#ifdef TB_PHASE_TIMING
+        if (tile == 0) { if (o[7][3] == 1.2345e33f) any_bad = true; attn_stamp(10); }
+#endif
         __syncwarp();                                  // the warp is done reading this stage
         if (tile + kMmaStages < n_tiles) {
             const int t = tokens_of(tile + kMmaStages);

@@ -101,6 +101,12 @@ struct SplitSink {
         part_o[pq * 128 + threadIdx.x] = o;
         if (threadIdx.x == 0) part_ml[pq * 2] = M, part_ml[pq * 2 + 1] = lsum;
     }
+    // the same, for a thread that holds channel `ch` of head u / the head's statistics
+    __device__ __forceinline__ void publish_at(int u, int ch, float o) const { part_o[((hq0 + u) * kMaxSplits + split) * 128 + ch] = o; }
+    __device__ __forceinline__ void publish_stat(int u, float M, float lsum) const {
+        const size_t pq = (hq0 + u) * kMaxSplits + split;
+        part_ml[pq * 2] = M, part_ml[pq * 2 + 1] = lsum;
+    }
     __device__ __forceinline__ void merge_if_last(int g, int* sh_last) const {
         const int tid = threadIdx.x;
         __threadfence();
@@ -388,15 +394,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// One of the block's 16 hardware barriers (0 is __syncthreads'), met by `count` threads; orders their shared-memory accesses.
-__device__ __forceinline__ void named_bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-
 // Shared memory behind the warps' stages for the merge inside a cluster of C blocks: the accumulator slices this
 // block owns from every block ([slices per owner][C][32 lanes] float4) and every block's (m, l) ([C][4] float4).
 static inline size_t cluster_merge_bytes(int C) { return (size_t)((8 + C - 1) / C) * C * 32 * 16 + (size_t)C * 4 * 16; }
 
 // NW warps per block.  With a.cluster_merge the blocks of one (sequence, KV head) form a thread-block
-// cluster (one block per split): the warps of a block fold their results in a tree, the blocks exchange
+// cluster (one block per split): the warps of a block fold their results through shared memory, the blocks exchange
 // channel slices of theirs through distributed shared memory, one cluster barrier, and every block merges
 // and writes the slices it owns -- no partials in global memory, no last-block round trips.  Without it (more splits than a cluster holds) the splits
 // go through the global workspace and the last block to arrive merges them (NW must be 4 then).
@@ -409,9 +412,7 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
                                                            float* __restrict__ part_ml, uint32_t* __restrict__ counters,
                                                            int32_t* __restrict__ status) {
     constexpr int D = 128;
-    constexpr int kMergePitch = 132;                  // floats per (rank, head) slot: 128 channels, m, l, pad
     extern __shared__ __align__(128) unsigned char smem_dyn[];
-    __shared__ float sh_m[NW][kMaxGroup], sh_l[NW][kMaxGroup];
     __shared__ int sh_last;
 
     attn_stamp(0);
@@ -703,78 +704,87 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     }
     __syncwarp();
     const size_t hq0 = (size_t)(ll * ut.n_seq + s) * gm.Hq + h * g;
-    if (a.cluster_merge) {
-        // Block result: a binary tree over the warps.  At every level the upper half of the remaining warps
-        // parks its accumulators in its own (drained) stages, lane by lane in the MMA layout, and the partner
-        // in the lower half folds them into its registers -- same lane, same elements, so nothing is
-        // transposed and a level costs 9 conflict-free 16-byte stores and loads per lane.  Each pair meets at a
-        // named barrier of its own (64 threads); the order of the folds is fixed, so the result is
-        // bit-reproducible.  (A flat combine -- every warp's result to shared memory, two block barriers,
-        // 128 threads summing NW terms per head -- was 0.12 us slower per launch.)
-        static_assert(NW <= 16, "the named barriers below are numbered 1..15: 8, 4, 2 and 1 pairs per level");
-        float4* tbuf = reinterpret_cast<float4*>(my_stage);             // [8][32] o, then [32] (m0, l0, m1, l1)
-        constexpr int kTop = NW > 8 ? 8 : NW > 4 ? 4 : NW > 2 ? 2 : 1;
+    // Every warp parks its accumulators in its own (drained) stages, lane by lane in the MMA layout -- float4
+    // number mt * 32 + lane is accumulator tile mt (16 channels) of that lane, number 256 + lane its (m, l) of
+    // heads 2 tig and 2 tig + 1 -- so that nothing is transposed and every access is a conflict-free 16 bytes.
+    // After one block barrier a thread owns one (tile, lane) slot: it folds the NW warps' values of that slot,
+    // all loads independent of one another, and holds a piece of the block's result in registers.
+    // (Measured alternatives, all within 0.03 us per launch of this one: a binary tree over the warps with a
+    // named barrier per pair; two barriers with the weights computed once.  Parking only the lanes of real heads
+    // when the group has at most four -- half the shared-memory traffic, 16 shuffles -- was 0.5 us slower.)
+    {
+        float4* tbuf = reinterpret_cast<float4*>(my_stage);
 #pragma unroll
-        for (int stride = kTop; stride >= 1; stride >>= 1) {
-            if (warp >= stride && warp < 2 * stride) {
+        for (int mt = 0; mt < 8; ++mt) tbuf[mt * 32 + lane] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+        tbuf[8 * 32 + lane] = make_float4(m_run[0], l_run[0], m_run[1], l_run[1]);
+    }
+    __syncthreads();
+    auto warp_buf = [&](int w) { return reinterpret_cast<const float4*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes); };
+    // block result of slot (mt, ln): acc = (head 2tg ch, head 2tg+1 ch, head 2tg ch+8, head 2tg+1 ch+8), ch = mt*16 + ln/4
+    auto fold_slot = [&](int mt, int ln, float4& acc, float4& stat) {
+        float4 q[NW];
 #pragma unroll
-                for (int mt = 0; mt < 8; ++mt) tbuf[mt * 32 + lane] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
-                tbuf[8 * 32 + lane] = make_float4(m_run[0], l_run[0], m_run[1], l_run[1]);
-                named_bar_sync(17 - 2 * stride + (warp - stride), 64);
-            } else if (warp < stride && warp + stride < NW) {
-                named_bar_sync(17 - 2 * stride + warp, 64);
-                const float4* pb = reinterpret_cast<const float4*>(smem_dyn + (size_t)(warp + stride) * kMmaStages * kStageBytes);
-                const float4 pm = pb[8 * 32 + lane];
-                const float M0 = fmaxf(m_run[0], pm.x), M1 = fmaxf(m_run[1], pm.z);
-                const float M0s = M0 == -INFINITY ? 0.f : M0, M1s = M1 == -INFINITY ? 0.f : M1;
-                const float ea0 = exp2f(m_run[0] - M0s), eb0 = exp2f(pm.x - M0s);
-                const float ea1 = exp2f(m_run[1] - M1s), eb1 = exp2f(pm.z - M1s);
-                l_run[0] = fmaf(pm.y, eb0, l_run[0] * ea0), l_run[1] = fmaf(pm.w, eb1, l_run[1] * ea1);
-                m_run[0] = M0, m_run[1] = M1;
+        for (int w = 0; w < NW; ++w) q[w] = warp_buf(w)[8 * 32 + ln];
+        float M0 = -INFINITY, M1 = -INFINITY;
 #pragma unroll
-                for (int mt = 0; mt < 8; ++mt) {
-                    const float4 v = pb[mt * 32 + lane];
-                    o[mt][0] = fmaf(v.x, eb0, o[mt][0] * ea0), o[mt][1] = fmaf(v.y, eb1, o[mt][1] * ea1);
-                    o[mt][2] = fmaf(v.z, eb0, o[mt][2] * ea0), o[mt][3] = fmaf(v.w, eb1, o[mt][3] * ea1);
-                }
-            }
+        for (int w = 0; w < NW; ++w) M0 = fmaxf(M0, q[w].x), M1 = fmaxf(M1, q[w].z);
+        const float M0s = M0 == -INFINITY ? 0.f : M0, M1s = M1 == -INFINITY ? 0.f : M1;
+        float L0 = 0.f, L1 = 0.f;
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            const float e0 = exp2f(q[w].x - M0s), e1 = exp2f(q[w].z - M1s);
+            L0 = fmaf(q[w].y, e0, L0), L1 = fmaf(q[w].w, e1, L1);
+            const float4 v = warp_buf(w)[mt * 32 + ln];
+            acc.x = fmaf(v.x, e0, acc.x), acc.y = fmaf(v.y, e1, acc.y), acc.z = fmaf(v.z, e0, acc.z), acc.w = fmaf(v.w, e1, acc.w);
         }
-        attn_stamp(5);
+        stat = make_float4(M0, L0, M1, L1);
+    };
+    attn_stamp(5);
+    if (a.cluster_merge) {
         // Merge of the blocks' results inside the cluster, sliced by channels: the 128 channels are eight slices
-        // of 16 (one accumulator tile of the MMA layout each), slice j belongs to block j mod C.  Warp 0 of every
-        // block sends each slice of its (o) to the slice's owner and its (m, l) to every owner -- 4.5 KB per block
-        // in all --, one cluster barrier, and every owner merges its 16 channels of all heads from the C partials
-        // (blocks in rank order: bit-reproducible) and writes them out.  No single merging block: the work behind
-        // the barrier is C terms per output, not C x 8.
+        // of 16 (one accumulator tile each), slice j belongs to block j mod C.  The thread that folded a slot sends
+        // it to the slice's owner, the block's (m, l) go to every owner -- 4.5 KB per block in all --, one cluster
+        // barrier, and every owner merges its 16 channels of all heads from the C partials (blocks in rank order:
+        // bit-reproducible) and writes them out.  No single merging block: the work behind the barrier is C terms
+        // per output, not C x 8, and their loads are issued together.
         cg::cluster_group cluster = cg::this_cluster();
         const int rank = (int)cluster.block_rank(), C = (int)cluster.num_blocks();
         const int T = (8 + C - 1) / C;                               // slices per owner
         float4* area = reinterpret_cast<float4*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [T][C][32 lanes]
         float4* ml = area + (size_t)T * C * 32;                      // [C][4]: (m, l) of heads 2 tig, 2 tig + 1
-        if (warp == 0) {
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt)
-                cluster.map_shared_rank(area, mt % C)[((mt / C) * C + rank) * 32 + lane] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
-            if (gid < C) cluster.map_shared_rank(ml, gid)[rank * 4 + tig] = make_float4(m_run[0], l_run[0], m_run[1], l_run[1]);
+        for (int slot = tid; slot < 256; slot += NW * 32) {
+            const int mt = slot >> 5, ln = slot & 31;
+            float4 acc, stat;
+            fold_slot(mt, ln, acc, stat);
+            cluster.map_shared_rank(area, mt % C)[((mt / C) * C + rank) * 32 + ln] = acc;
+            if (mt == 0 && (ln >> 2) < C) cluster.map_shared_rank(ml, ln >> 2)[rank * 4 + (ln & 3)] = stat;
         }
         cluster.sync();
         if (rank < 8) {
+            constexpr int kMaxC = kAttnMaxCluster;
             for (int i = tid; i < T * 32; i += NW * 32) {
                 const int ts = i >> 5, ln = i & 31, tg = ln & 3, gd = ln >> 2;
                 const int j = ts * C + rank;                         // the slice
                 if (j >= 8) continue;
+                float4 q[kMaxC], v[kMaxC];
+#pragma unroll
+                for (int r = 0; r < kMaxC; ++r) {
+                    q[r] = r < C ? ml[r * 4 + tg] : make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
+                    v[r] = r < C ? area[(ts * C + r) * 32 + ln] : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
                 float M0 = -INFINITY, M1 = -INFINITY;
-                for (int r = 0; r < C; ++r) M0 = fmaxf(M0, ml[r * 4 + tg].x), M1 = fmaxf(M1, ml[r * 4 + tg].z);
+#pragma unroll
+                for (int r = 0; r < kMaxC; ++r) M0 = fmaxf(M0, q[r].x), M1 = fmaxf(M1, q[r].z);
                 const float M0s = M0 == -INFINITY ? 0.f : M0, M1s = M1 == -INFINITY ? 0.f : M1;
                 float ls0 = 0.f, ls1 = 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int r = 0; r < C; ++r) {
-                    const float4 q = ml[r * 4 + tg];
-                    const float e0 = exp2f(q.x - M0s), e1 = exp2f(q.z - M1s);
-                    ls0 = fmaf(q.y, e0, ls0), ls1 = fmaf(q.w, e1, ls1);
-                    const float4 v = area[(ts * C + r) * 32 + ln];
-                    acc.x = fmaf(v.x, e0, acc.x), acc.y = fmaf(v.y, e1, acc.y);
-                    acc.z = fmaf(v.z, e0, acc.z), acc.w = fmaf(v.w, e1, acc.w);
+#pragma unroll
+                for (int r = 0; r < kMaxC; ++r) {
+                    const float e0 = exp2f(q[r].x - M0s), e1 = exp2f(q[r].z - M1s);
+                    ls0 = fmaf(q[r].y, e0, ls0), ls1 = fmaf(q[r].w, e1, ls1);
+                    acc.x = fmaf(v[r].x, e0, acc.x), acc.y = fmaf(v[r].y, e1, acc.y);
+                    acc.z = fmaf(v[r].z, e0, acc.z), acc.w = fmaf(v[r].w, e1, acc.w);
                 }
                 const int u0 = 2 * tg, u1 = u0 + 1, ch = j * 16 + gd;
                 if (u0 < g) {
@@ -788,51 +798,21 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
             }
         }
     } else if constexpr (NW == kAttnWarps) {
-        // splits through the global workspace: flat combine into one channel per thread, then the sink
-        float* wo = reinterpret_cast<float*>(my_stage);                  // [8 heads][kMergePitch]
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt) {
-            wo[(2 * tig) * kMergePitch + mt * 16 + gid] = o[mt][0];          // pitch 132: the 32 lanes hit 32 banks
-            wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid] = o[mt][1];
-            wo[(2 * tig) * kMergePitch + mt * 16 + gid + 8] = o[mt][2];
-            wo[(2 * tig + 1) * kMergePitch + mt * 16 + gid + 8] = o[mt][3];
-        }
-        if (gid == 0) {
-            sh_m[warp][2 * tig] = m_run[0], sh_l[warp][2 * tig] = l_run[0];
-            sh_m[warp][2 * tig + 1] = m_run[1], sh_l[warp][2 * tig + 1] = l_run[1];
-        }
-        __syncthreads();
-        // weights 2^(m_w - M) of every (warp, head), computed once by NW*8 threads
-        __shared__ float sh_w[NW][kMaxGroup], sh_M[kMaxGroup];
-        if (tid < NW * kMaxGroup) {
-            const int w = tid / kMaxGroup, u = tid % kMaxGroup;
-            float M = -INFINITY;
-#pragma unroll
-            for (int x = 0; x < NW; ++x) M = fmaxf(M, sh_m[x][u]);
-            sh_w[w][u] = exp2f(sh_m[w][u] - (M == -INFINITY ? 0.f : M));
-            if (w == 0) sh_M[u] = M;
-        }
-        __syncthreads();
-        float cM[kMaxGroup], cL[kMaxGroup], cO[kMaxGroup];        // block result per head; cO: channel tid (tid < 128)
-#pragma unroll
-        for (int u = 0; u < kMaxGroup; ++u) {
-            cM[u] = -INFINITY, cL[u] = 0.f, cO[u] = 0.f;
-            if (u < g && tid < D) {
-                float lsum = 0.f, acc = 0.f;
-#pragma unroll
-                for (int w = 0; w < NW; ++w) {
-                    const float e = sh_w[w][u];
-                    lsum += sh_l[w][u] * e;
-                    acc = fmaf(reinterpret_cast<const float*>(smem_dyn + (size_t)w * kMmaStages * kStageBytes)[u * kMergePitch + tid], e, acc);
-                }
-                cM[u] = sh_M[u], cL[u] = lsum, cO[u] = acc;
+        // splits through the global workspace, merged by the last block to arrive
+        SplitSink sink{part_o, part_ml, counters, a.out, a.lse, hq0, lu, split, a.nsplit};
+        for (int slot = tid; slot < 256; slot += NW * 32) {
+            const int mt = slot >> 5, ln = slot & 31, u0 = 2 * (ln & 3), ch = mt * 16 + (ln >> 2);
+            float4 acc, stat;
+            fold_slot(mt, ln, acc, stat);
+            if (u0 < g) {
+                sink.publish_at(u0, ch, acc.x), sink.publish_at(u0, ch + 8, acc.z);
+                if (mt == 0 && ln < 4) sink.publish_stat(u0, stat.x, stat.y);
+            }
+            if (u0 + 1 < g) {
+                sink.publish_at(u0 + 1, ch, acc.y), sink.publish_at(u0 + 1, ch + 8, acc.w);
+                if (mt == 0 && ln < 4) sink.publish_stat(u0 + 1, stat.z, stat.w);
             }
         }
-        attn_stamp(5);
-        SplitSink sink{part_o, part_ml, counters, a.out, a.lse, hq0, lu, split, a.nsplit};
-#pragma unroll
-        for (int u = 0; u < kMaxGroup; ++u)
-            if (u < g) sink.publish(u, cM[u], cL[u], cO[u]);
         sink.merge_if_last(g, &sh_last);
     }
     attn_stamp(6);

@@ -6,6 +6,7 @@
 // softmax (m, l, o) per query head; the last block to arrive for a (sequence, KV head) merges the
 // splits in split order, so the result is bit-reproducible.
 #include <cooperative_groups.h>
+#include <type_traits>
 
 #include "tb_common.cuh"
 #include "tb_internal.h"
@@ -753,6 +754,28 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
         const int T = (8 + C - 1) / C;                               // slices per owner
         float4* area = reinterpret_cast<float4*>(smem_dyn + (size_t)NW * kMmaStages * kStageBytes);   // [T][C][32 lanes]
         float4* ml = area + (size_t)T * C * 32;                      // [C][4]: (m, l) of heads 2 tig, 2 tig + 1
+        // writes one merged piece: (acc, sums ls0 / ls1, maxima M0 / M1) of heads 2 tg, 2 tg + 1 at channels ch, ch + 8
+        auto write_piece = [&](int tg, int ch, const float4& acc, float M0, float ls0, float M1, float ls1) {
+            const int u0 = 2 * tg, u1 = u0 + 1;
+            if (u0 < g) {
+                a.out[(hq0 + u0) * D + ch] = acc.x / ls0, a.out[(hq0 + u0) * D + ch + 8] = acc.z / ls0;
+                if (a.lse && ch == 0) a.lse[hq0 + u0] = (M0 + log2f(ls0)) * kLn2;
+            }
+            if (u1 < g) {
+                a.out[(hq0 + u1) * D + ch] = acc.y / ls1, a.out[(hq0 + u1) * D + ch + 8] = acc.w / ls1;
+                if (a.lse && ch == 0) a.lse[hq0 + u1] = (M1 + log2f(ls1)) * kLn2;
+            }
+        };
+        if (C == 1) {                                                // the block's result is the problem's
+            for (int slot = tid; slot < 256; slot += NW * 32) {
+                const int mt = slot >> 5, ln = slot & 31;
+                float4 acc, stat;
+                fold_slot(mt, ln, acc, stat);
+                write_piece(ln & 3, mt * 16 + (ln >> 2), acc, stat.x, stat.y, stat.z, stat.w);
+            }
+            attn_stamp(6);
+            return;
+        }
         for (int slot = tid; slot < 256; slot += NW * 32) {
             const int mt = slot >> 5, ln = slot & 31;
             float4 acc, stat;
@@ -761,41 +784,39 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
             if (mt == 0 && (ln >> 2) < C) cluster.map_shared_rank(ml, ln >> 2)[rank * 4 + (ln & 3)] = stat;
         }
         cluster.sync();
-        if (rank < 8) {
-            constexpr int kMaxC = kAttnMaxCluster;
+        // the owners' merge, unrolled to a bound on the cluster size so that the loads go out together
+        auto owner_merge = [&](auto bound) {
+            constexpr int kC = decltype(bound)::value;
             for (int i = tid; i < T * 32; i += NW * 32) {
-                const int ts = i >> 5, ln = i & 31, tg = ln & 3, gd = ln >> 2;
+                const int ts = i >> 5, ln = i & 31, tg = ln & 3;
                 const int j = ts * C + rank;                         // the slice
                 if (j >= 8) continue;
-                float4 q[kMaxC], v[kMaxC];
+                float4 q[kC], v[kC];
 #pragma unroll
-                for (int r = 0; r < kMaxC; ++r) {
+                for (int r = 0; r < kC; ++r) {
                     q[r] = r < C ? ml[r * 4 + tg] : make_float4(-INFINITY, 0.f, -INFINITY, 0.f);
                     v[r] = r < C ? area[(ts * C + r) * 32 + ln] : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
                 float M0 = -INFINITY, M1 = -INFINITY;
 #pragma unroll
-                for (int r = 0; r < kMaxC; ++r) M0 = fmaxf(M0, q[r].x), M1 = fmaxf(M1, q[r].z);
+                for (int r = 0; r < kC; ++r) M0 = fmaxf(M0, q[r].x), M1 = fmaxf(M1, q[r].z);
                 const float M0s = M0 == -INFINITY ? 0.f : M0, M1s = M1 == -INFINITY ? 0.f : M1;
                 float ls0 = 0.f, ls1 = 0.f;
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int r = 0; r < kMaxC; ++r) {
+                for (int r = 0; r < kC; ++r) {
                     const float e0 = exp2f(q[r].x - M0s), e1 = exp2f(q[r].z - M1s);
                     ls0 = fmaf(q[r].y, e0, ls0), ls1 = fmaf(q[r].w, e1, ls1);
                     acc.x = fmaf(v[r].x, e0, acc.x), acc.y = fmaf(v[r].y, e1, acc.y);
                     acc.z = fmaf(v[r].z, e0, acc.z), acc.w = fmaf(v[r].w, e1, acc.w);
                 }
-                const int u0 = 2 * tg, u1 = u0 + 1, ch = j * 16 + gd;
-                if (u0 < g) {
-                    a.out[(hq0 + u0) * D + ch] = acc.x / ls0, a.out[(hq0 + u0) * D + ch + 8] = acc.z / ls0;
-                    if (a.lse && j == 0 && gd == 0) a.lse[hq0 + u0] = (M0 + log2f(ls0)) * kLn2;
-                }
-                if (u1 < g) {
-                    a.out[(hq0 + u1) * D + ch] = acc.y / ls1, a.out[(hq0 + u1) * D + ch + 8] = acc.w / ls1;
-                    if (a.lse && j == 0 && gd == 0) a.lse[hq0 + u1] = (M1 + log2f(ls1)) * kLn2;
-                }
+                write_piece(tg, j * 16 + (ln >> 2), acc, M0, ls0, M1, ls1);
             }
+        };
+        if (rank < 8) {
+            if (C <= 4) owner_merge(std::integral_constant<int, 4>{});
+            else if (C <= 9) owner_merge(std::integral_constant<int, 9>{});
+            else owner_merge(std::integral_constant<int, kAttnMaxCluster>{});
         }
     } else if constexpr (NW == kAttnWarps) {
         // splits through the global workspace, merged by the last block to arrive
@@ -933,7 +954,12 @@ cudaError_t launch_attention(const tb_ctx* c, const UnitTable& ut, const AttnArg
         const size_t merge_bytes = a.cluster_merge ? cluster_merge_bytes(a.nsplit) : 0;
         // three stages per warp when the 8-warp block still fits the SM with them
         const int nst = (nw == 8 && 8 * 3 * kStageBytes + merge_bytes <= 220 * 1024 && a.nsplit <= 8) ? 3 : 2;
-        const size_t smem = (size_t)nw * nst * kStageBytes + merge_bytes;
+        size_t smem = (size_t)nw * nst * kStageBytes + merge_bytes;
+        // The split count of the 4-warp launches is chosen for two blocks per SM; their 64 KB of stages would let
+        // a third one in, and the block scheduler then loads some SMs with three blocks and leaves others with one
+        // (batch 8 at 64K: 59 us per launch against 52.6).  Asking for a third of the SM's shared memory plus a
+        // little keeps it at two.
+        if (nw == 4 && smem < 76 * 1024) smem = 76 * 1024;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = grid;
         cfg.blockDim = dim3(nw * 32, 1, 1);

@@ -771,7 +771,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 
 #ifdef TB_PHASE_TIMING
     const unsigned long long tc0 = wave_now();
-#define CW_MARK(i) do { if (tid == 0) { const int bb = blockIdx.y * gridDim.x + blockIdx.x; if (bb < 1024) g_wave_ns[(i) & 3][bb] = ((i) < 4 ? 0 : 0) + wave_now() - ((i) == 0 ? 0 : tc0); } } while (0)
+#define CW_MARK(i) do { if (tid == 0) { const int bb = blockIdx.y * gridDim.x + blockIdx.x; if (bb < 1024) { g_wave_ns[(i) & 3][bb] = wave_now() - ((i) == 0 ? 0 : tc0); if ((i) == 0) { unsigned smid_; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_)); g_wave_smid[bb] = smid_; } } } } while (0)
 #else
 #define CW_MARK(i) do {} while (0)
 #endif
@@ -1012,6 +1012,7 @@ __global__ void __launch_bounds__(kThreads, 2)
 
     // ---- own digits -> bitmask; own rows of the threshold bin -> every peer's list ------------------------
     int my_take = 0;
+    int* my_slots = reinterpret_cast<int*>(list + (C + 1) * kCwListCap);       // own rows of the threshold bin (local row numbers)
     {
         const uint4* bins4 = reinterpret_cast<const uint4*>(bins);
         for (int v = tid; v < my_tiles * (kRows / 8); v += kThreads) {          // 8 digits per 16-byte load
@@ -1029,13 +1030,10 @@ __global__ void __launch_bounds__(kThreads, 2)
             word |= __shfl_xor_sync(0xffffffffu, word, 1);
             word |= __shfl_xor_sync(0xffffffffu, word, 2);
             if ((lane & 3) == 0) mask[v >> 2] = word;
-            while (eq) {                               // rare: a handful of rows per block
+            while (eq) {                               // a handful of rows per block: only their places are noted here
                 const int e = __ffs(eq) - 1;
                 eq &= eq - 1;
-                const int ls = v * 8 + e;
-                const int i = atomicAdd(&cs->my_n, 1);
-                const uint2 ent = make_uint2(__ldcg(keys_unit + slot0 + ls) - bin_base, (uint32_t)(slot0 + ls));
-                for (unsigned r = 0; r < C; ++r) peer_ptr(list, (int)r)[rank * kCwListCap + i] = ent;
+                my_slots[atomicAdd(&cs->my_n, 1)] = v * 8 + e;
             }
         }
     }
@@ -1043,7 +1041,16 @@ __global__ void __launch_bounds__(kThreads, 2)
         int total;
         wave_excl_scan(my_take, sm->warp_a, total);
         __syncthreads();
-        if (tid < (int)C) peer_ptr(cs, tid)->take[rank] = total, peer_ptr(cs, tid)->n_in[rank] = cs->my_n;
+        // The noted rows' parked keys come back from L2 in one round trip, a row per thread (fetched inside the
+        // loop above, every such row stalled its warp for that round trip: 2.5 us for the pass instead of 1.3),
+        // and go to every peer's list.
+        const int n_mine = cs->my_n;
+        if (tid < n_mine) {
+            const int ls = my_slots[tid];
+            const uint2 ent = make_uint2(__ldcg(keys_unit + slot0 + ls) - bin_base, (uint32_t)(slot0 + ls));
+            for (unsigned r = 0; r < C; ++r) peer_ptr(list, (int)r)[rank * kCwListCap + tid] = ent;
+        }
+        if (tid < (int)C) peer_ptr(cs, tid)->take[rank] = total, peer_ptr(cs, tid)->n_in[rank] = n_mine;
     }
     CW_PH(2);
     cluster_sync_all();                                // barrier 2: lists and counts are everywhere
@@ -1122,7 +1129,7 @@ cudaError_t launch_select_cw(const tb_ctx* c, const UnitTable& ut, const SelectA
     if (C < 1) C = 1;
     const int tiles_per_cta = (n_tiles + C - 1) / C > 0 ? (n_tiles + C - 1) / C : 1;
     const int tile_bytes = kRows * gm.dp * (gm.dtype == TB_BF16 ? 2 : 4);
-    const size_t ring_min = (size_t)(C + 1) * kCwListCap * sizeof(uint2);   // list regions + the entries side by side
+    const size_t ring_min = (size_t)(C + 1) * kCwListCap * sizeof(uint2) + kCwListCap * sizeof(int);   // list regions + the entries side by side + own rows' places
     const size_t budget = (size_t)(C * n_units > c->sm_count ? 113 : 224) * 1024;
     const size_t fixed_off = 1024 + kDigitBins * sizeof(int) + (size_t)tiles_per_cta * (kRows / 32) * 4 + sizeof(CwSmem);
     const size_t bins_bytes = (size_t)tiles_per_cta * kRows * 2;

@@ -39,10 +39,10 @@ UNIT = "tokens/s"
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
     ("cfg2_llama8b_32k", "select_kernel"): 67_221_760 + 848_896,   # profiles/select_kernel_cfg2_32k.md
-    ("cfg2_llama8b_32k", "attn_kernel"): 13_597_952,               # profiles/attn_mma_kernel_cfg2_32k.md
+    ("cfg2_llama8b_32k", "attn_kernel"): 13_598_208,               # profiles/attn_mma_kernel_cfg2_32k.md
     ("cfg3_batched_serving", "select_kernel"): 398_907_392 + 5_187_840,   # profiles/select_wave_kernel_cfg3_batched.md
     ("cfg4_long_context_128k", "select_kernel"): 268_011_264 + 3_980_544,  # profiles/select_cw_kernel_cfg4_128k.md
-    ("cfg5_interval_neighbors", "attn_kernel"): 309_482_496 + 3_839_488,   # profiles/attn_mma_kernel_cfg5_interval.md
+    ("cfg5_interval_neighbors", "attn_kernel"): 309_490_432 + 4_711_680,   # profiles/attn_mma_kernel_cfg5_interval.md
 }
 
 

@@ -77,8 +77,9 @@ struct AttnUnit {
     __device__ __forceinline__ AttnUnit(const Geom& gm, const UnitTable& ut, int ll, int s, int h) {
         const size_t pc = (size_t)(ut.layer_begin + ll) * gm.max_batch + ut.seq_id[s];
         const int pl = ll * ut.n_seq + s;
-        const int lh = (h * gm.Hl) / gm.Ha;
-        kv_c = pc * gm.Hkv + (h * gm.Hkv) / gm.Ha;
+        // (the usual scopes have Hl == Ha, and Hkv == Ha or Hl: no division on the way to the first load)
+        const int lh = gm.Hl == gm.Ha ? h : (h * gm.Hl) / gm.Ha;
+        kv_c = pc * gm.Hkv + (gm.Hkv == gm.Ha ? h : (h * gm.Hkv) / gm.Ha);
         list_c = pc * gm.Hl + lh;
         list_l = pl * gm.Hl + lh;
         lu = pl * gm.Ha + h;
@@ -417,15 +418,23 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     __shared__ int sh_last;
 
     attn_stamp(0);
-    // Dependency wait (see pdl_wait): up front when the lists or cache rows may come from the
-    // predecessor; otherwise only before the queries are read, so that the row map, the list fetch
-    // and the first gathers overlap the predecessor's tail.
-    if (!a.early_ok) pdl_wait();
-    pdl_launch_dependents();
+    // Dependency wait (see pdl_wait).  When the lists or cache rows may come from the predecessor: before the
+    // first read of anything it may have written -- the list entries, or already the lengths and list counts when
+    // those are read on the device; what comes from the kernel parameters alone (row map, split, addresses) runs
+    // beside the predecessor's tail.  Otherwise only before the queries are read, so that the list fetch and the
+    // first gathers overlap the predecessor as well.  The own dependent is released at the start in that case,
+    // else right after the wait (see tb_api.cu on why not before).
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int gid = lane >> 2, tig = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y;
-    const int ll = blockIdx.z / ut.n_seq, s = blockIdx.z % ut.n_seq;
+    const int ll = ut.layer_count == 1 ? 0 : blockIdx.z / ut.n_seq, s = blockIdx.z - ll * ut.n_seq;
+    bool waited = a.early_ok != 0;
+    if (waited) pdl_launch_dependents();
+    if (!waited && (ut.use_dev_len || (!a.dense && (a.idx != nullptr || a.known_cnt[ll * ut.n_seq + s] < 0)))) {
+        pdl_wait();
+        pdl_launch_dependents();
+        waited = true;
+    }
     const int L = unit_len(gm, ut, ll, s);
     const int g = gm.ga;
     const AttnUnit au(gm, ut, ll, s, h);
@@ -448,8 +457,11 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const int n_rows = a.dense ? L : rm.n_sink + n_list + (L - rm.w_begin);
 
     // rows of this split, dealt to the warps in whole tiles of 16
-    const int r_begin = (int)((long long)n_rows * split / a.nsplit);
-    const int r_end = (int)((long long)n_rows * (split + 1) / a.nsplit);
+    // (32-bit arithmetic whenever it is exact: a 64-bit division costs hundreds of cycles in a prologue that is
+    // on the critical path of the cluster that starts late)
+    const bool small = n_rows < (1 << 24);             // nsplit <= 32
+    const int r_begin = small ? (int)((unsigned)n_rows * (unsigned)split / (unsigned)a.nsplit) : (int)((long long)n_rows * split / a.nsplit);
+    const int r_end = small ? (int)((unsigned)n_rows * (unsigned)(split + 1) / (unsigned)a.nsplit) : (int)((long long)n_rows * (split + 1) / a.nsplit);
     const int tiles_all = (r_end - r_begin + kTileTok - 1) / kTileTok;
     // dealt evenly: no warp gets more than one tile above another (a tile beyond a warp's stages waits for
     // a stage to drain and then for its rows, a whole memory latency)
@@ -464,6 +476,10 @@ __global__ void __launch_bounds__(NW * 32) attn_mma_kernel(Geom gm, UnitTable ut
     const unsigned char* res_unit = reinterpret_cast<const unsigned char*>(a.res_rows) + au.kv_c * (size_t)(a.res_sinks + a.res_window) * 2 * D * 2;
     const unsigned char* imp_unit = reinterpret_cast<const unsigned char*>(a.imp_rows) + au.list_c * (size_t)gm.idx_cap * 2 * D * 2;
 
+    if (!waited) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
     bool any_bad = false;
     // Gather of one tile: the whole warp copies each 512-byte K|V row with one 16-byte cp.async per
     // lane (one warp instruction per row; the per-row TMA bulk copies this replaces queued up at the

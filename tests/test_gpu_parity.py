@@ -103,6 +103,17 @@ def test_cluster_path_long_sequence(H):
     full_pipeline_check(H, case, p)
 
 
+def test_attention_merge_shapes_with_eight_heads_per_group(H):
+    # Groups of eight query heads fill every lane of the accumulator layout (groups of four leave half of it as
+    # padding).  Three launch shapes of the bf16 attention kernel: a cluster of 16 blocks whose warps hold two
+    # tiles (taken as one 32-token tile) or one; a cluster of a few blocks with three tiles per warp; and one
+    # block per problem, which writes its result without the cluster exchange.
+    for lengths, budget, sinks, recent in (([40000], 3000, 5, 130), ([9000], 1100, 0, 40), ([2500, 2400, 2300, 2200], 300, 2, 9)):
+        w = wl.workload(2, n_layers=1, batch=len(lengths), n_q_heads=16, n_kv_heads=2, lengths=lengths, budget=budget,
+                        sinks=sinks, recent=recent)
+        full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, w.sinks, w.recent), dense_too=len(lengths) == 1 and lengths[0] < 10000)
+
+
 def test_imp_dim_16_and_fp32_gqa(H):
     w = wl.workload(1, n_q_heads=4, n_kv_heads=2, imp_dim=16, lengths=[1500], budget=100, sinks=2, recent=5)
     full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, w.sinks, w.recent))

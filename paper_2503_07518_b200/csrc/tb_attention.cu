@@ -325,8 +325,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_kernel(Geom gm, UnitTable u
 // bf16 path: tensor-core tiles of (16 gathered tokens) x (query heads padded to 8).
 //
 // Each warp owns a ring of shared-memory stages; a stage holds 16 gathered K|V row pairs (512 B each,
-// copied by the whole warp with 16-byte cp.async) at a 528-byte pitch so that ldmatrix reads are
-// bank-conflict free.  S = K Q^T (tokens x heads) and O^T += V^T P^T (channels x heads) run on
+// copied by the whole warp with 16-byte cp.async) at a 512-byte pitch with the 16-byte chunks of a row
+// permuted by the row number, so that ldmatrix reads are bank-conflict free.  S = K Q^T (tokens x heads) and O^T += V^T P^T (channels x heads) run on
 // mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the GQA group's heads as the N = 8 columns --
 // the one place where batch x group makes the contraction a real dense tile; P is split into a bf16
 // high and low part (two MMAs) so that the probabilities keep ~16 bits, and reaches the B operand

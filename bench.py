@@ -850,6 +850,8 @@ def main():
                     help="which heads share an index list (configs 1-4; default: one list per KV head)")
     ap.add_argument("--context", type=int, default=0,
                     help="override every sequence's context length (e.g. --config 4 --context 1048576 --layers 8)")
+    ap.add_argument("--budget", type=int, default=0,
+                    help="override the selection budget (e.g. --config 4 --budget 8192: the paper's latency setting, Sec. 4.3)")
     ap.add_argument("--list-layouts", action="store_true",
                     help="time the attention kernel on random / runs-of-3 / contiguous caller lists of the workload's shapes")
     ap.add_argument("--neighbors", default=None, choices=["dilate", "cluster"],
@@ -863,6 +865,8 @@ def main():
         w = w.scaled(lengths=[args.context] * w.batch, name="%s@%d" % (w.name, args.context))
     if args.neighbors:
         w = w.scaled(nmode=0 if args.neighbors == "dilate" else 1)
+    if args.budget:
+        w = w.scaled(budget=args.budget, name="%s,budget=%d" % (w.name, args.budget))
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -884,7 +888,7 @@ def main():
     if "profile_run" not in line:
         extra = default_run and not args.no_extra and not args.profile and world == 1 and not args.offload_kv and \
             not args.important_buffer and \
-            args.list_scope == "kv_head" and not args.layers and not args.context
+            args.list_scope == "kv_head" and not args.layers and not args.context and not args.budget
         if extra:
             line["workloads"] = {}
             for cfg in (3, 4, 5):

@@ -114,6 +114,31 @@ def test_attention_merge_shapes_with_eight_heads_per_group(H):
         full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, w.sinks, w.recent), dense_too=len(lengths) == 1 and lengths[0] < 10000)
 
 
+def _random_shapes(n, seed):
+    # seeded draws over group size, KV heads, batch, lengths (a few long ones), budget, sinks, window, neighbour rule:
+    # between them they reach every launch shape of the selection and attention kernels
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        g, hkv = int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2, 4]))
+        batch = int(rng.choice([1, 1, 1, 2, 3, 5, 24]))
+        top = 140000 if batch == 1 and i % 4 == 0 else 30000 if batch == 1 else 6000 if batch < 24 else 2500
+        lengths = [int(rng.integers(40, top)) for _ in range(batch)]
+        budget = int(rng.integers(8, max(9, min(3500, max(lengths)))))
+        cases.append((g, hkv, lengths, budget, int(rng.choice([0, 0, 1, 4, 16])), int(rng.choice([0, 0, 7, 64, 300])),
+                      int(rng.choice([0, 0, 0, 1, 2])), int(rng.choice([0, 1]))))
+    return cases
+
+
+@pytest.mark.parametrize("shape", _random_shapes(32, 20250307),
+                         ids=lambda c: "g%d_kv%d_b%d_L%d_B%d_s%d_w%d_r%d%s" % (c[0], c[1], len(c[2]), max(c[2]), c[3], c[4], c[5], c[6], "dc"[c[7]]))
+def test_random_shapes(H, shape):
+    g, hkv, lengths, budget, sinks, recent, radius, nmode = shape
+    w = wl.workload(2, n_layers=1, batch=len(lengths), n_q_heads=g * hkv, n_kv_heads=hkv, lengths=lengths, budget=budget,
+                    sinks=sinks, recent=recent, radius=radius, nmode=nmode)
+    full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, w.sinks, w.recent, radius, nmode))
+
+
 def test_imp_dim_16_and_fp32_gqa(H):
     w = wl.workload(1, n_q_heads=4, n_kv_heads=2, imp_dim=16, lengths=[1500], budget=100, sinks=2, recent=5)
     full_pipeline_check(H, H.Case(w), tb().select_params(w.budget, w.sinks, w.recent))
